@@ -1,0 +1,215 @@
+/*
+ * edgeshard.h — C ABI of the shard-execution library (sm_100a).
+ *
+ * EdgeShard cuts an LLM of N layers into contiguous shards and places each on one device
+ * (paper, Sec. "System Model" and Sec. "Optimize LLM Inference"): a shard runs layers i..m,
+ * takes the previous shard's activation (or the prompt's token ids if it holds the embedding
+ * layer) and emits the activation of its last layer (or, if it holds the output layer, the
+ * logits and the generated token).  Inference is a prefill over the prompt followed by
+ * one-token-at-a-time generation against a KV cache that is reserved on the device beforehand
+ * (Sec. "Generative LLM Inference", Sec. "Collaborative inference").  The partition algorithms
+ * consume a per-layer profile: execution time, activation size and memory (Sec. "Profiling").
+ *
+ * This library is the execution of ONE shard on ONE GPU.  The decoder is Llama-2 (RMSNorm,
+ * rotary position embedding on adjacent pairs (2i,2i+1), causal attention with grouped KV
+ * heads, SwiGLU feed-forward), fp16 weights / KV / intermediate activations, fp32 accumulation,
+ * fp32 residual stream (the activation that is handed off is fp32).
+ *
+ * Conventions
+ *  - Every function returns a status and never throws or aborts.  On error nothing has been
+ *    launched unless stated otherwise, out-parameters are untouched, and es_last_error()
+ *    returns a thread-local message.
+ *  - "dev" pointers are CUDA device pointers on the current device; "host" pointers are
+ *    ordinary host memory.  The library allocates no device memory: weights, KV pages and
+ *    scratch all belong to the caller and must outlive the shard.
+ *  - Work is enqueued on the stream given at creation; calls do not synchronise unless stated.
+ *  - Layer indices are decoder-layer indices in [0, n_layers_total).  The paper's layer 0
+ *    (embedding) belongs to the shard with layer_begin == 0 and its layer N-1 (output layer)
+ *    to the shard with layer_end == n_layers_total.
+ */
+#ifndef EDGESHARD_H_
+#define EDGESHARD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define ES_API __attribute__((visibility("default")))
+#else
+#define ES_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct es_shard es_shard_t; /* opaque, library-owned host object */
+
+typedef enum {
+  ES_OK = 0,
+  ES_ERR_INVALID_ARG = 1,    /* null pointer, non-positive size, both/neither of ids and hidden_in */
+  ES_ERR_SHAPE = 2,          /* model dimensions the kernels do not support */
+  ES_ERR_RANGE = 3,          /* layer range outside [0, n_layers_total], slot or length out of range */
+  ES_ERR_STATE = 4,          /* decode on a slot that was never prefilled, handoff before any pass */
+  ES_ERR_KV_FULL = 5,        /* the slot's context would exceed max_seq */
+  ES_ERR_WORKSPACE = 6,      /* a caller buffer is smaller than es_shard_workspace_bytes says */
+  ES_ERR_CUDA = 7,           /* a CUDA runtime call failed; message holds cudaGetErrorString */
+  ES_ERR_DEVICE_TIMEOUT = 8, /* a bounded device-side wait gave up (see es_shard_device_status) */
+  ES_ERR_UNSUPPORTED = 9
+} es_status_t;
+
+typedef enum { ES_DTYPE_F16 = 0, ES_DTYPE_F32 = 1, ES_DTYPE_I32 = 2 } es_dtype_t;
+
+/* Model and capacity description.  max_slots = number of sequences whose KV is kept at once;
+ * max_seq = longest context (prompt + generated) per slot; max_tokens = largest B*T of one
+ * prefill call; kv_page_tokens = tokens per KV page (power of two, >= 16; 64 is the default
+ * choice).  max_batch = largest B of one call (<= max_slots). */
+typedef struct {
+  int32_t n_layers_total, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  float rms_eps, rope_theta;
+  int32_t max_slots, max_seq, max_tokens, max_batch, kv_page_tokens;
+} es_model_desc_t;
+
+/* One decoder layer: dev pointers, fp16, matrices row-major [out, in].
+ *   attn_norm, ffn_norm [d_model]; wq [n_heads*head_dim, d_model]; wk, wv [n_kv_heads*head_dim, d_model];
+ *   wo [d_model, n_heads*head_dim]; w_gate, w_up [d_ffn, d_model]; w_down [d_model, d_ffn].
+ * All matrix pointers must be 16-byte aligned.  Borrowed for the shard's life. */
+typedef struct {
+  const void *attn_norm, *wq, *wk, *wv, *wo, *ffn_norm, *w_gate, *w_up, *w_down;
+} es_layer_weights_t;
+
+typedef struct {
+  const void *tok_embedding;         /* dev fp16 [vocab, d_model]; required iff layer_begin == 0 */
+  const void *final_norm, *lm_head;  /* dev fp16 [d_model], [vocab, d_model]; required iff layer_end == n_layers_total */
+  const es_layer_weights_t *layers;  /* host array of layer_end - layer_begin entries */
+} es_weights_t;
+
+/* A borrowed view of a device tensor, row-major, contiguous. */
+typedef struct {
+  void *data;
+  int32_t dtype; /* es_dtype_t */
+  int32_t rank;
+  int64_t shape[4];
+} es_tensor_t;
+
+/* One entry of the per-layer profile (the t_comp / O_i / Req_i traces of Sec. "Profiling").
+ * layer: -1 = embedding, n_layers_total = final norm + LM head, otherwise the decoder layer.
+ * avg_ms_per_token = (sum of prefill ms + sum of decode ms) / (n_prefill + n_decode): each
+ * prefill call and each decode step generates one token per sequence. */
+typedef struct {
+  int32_t layer;
+  int32_t n_prefill, n_decode;
+  float prefill_ms_mean, decode_ms_mean, avg_ms_per_token;
+  int64_t activation_bytes; /* output of this layer for one token: d_model * 4 (or vocab * 4 for the head) */
+  int64_t weight_bytes;     /* Req_i, parameters */
+  int64_t kv_bytes;         /* Req_i, reserved KV cache of this layer (all slots) */
+} es_layer_profile_t;
+
+/* Sizes of the two caller-owned device buffers a shard [layer_begin, layer_end) needs.
+ * Host-only; validates the description exactly as es_shard_create does. */
+ES_API es_status_t es_shard_workspace_bytes(const es_model_desc_t *desc, int32_t layer_begin, int32_t layer_end,
+                                     size_t *kv_bytes, size_t *scratch_bytes);
+
+/* Creates the shard for decoder layers [layer_begin, layer_end) (paper: layers i..m on device j).
+ * kv_buffer / scratch_buffer: dev, 256-byte aligned, at least the sizes reported above; the
+ * library initialises them (enqueued on `cuda_stream`, a cudaStream_t cast to void*, may be 0).
+ * KV pages of every slot are reserved here, before any inference call. */
+ES_API es_status_t es_shard_create(const es_model_desc_t *desc, int32_t layer_begin, int32_t layer_end,
+                            const es_weights_t *weights, void *kv_buffer, size_t kv_bytes,
+                            void *scratch_buffer, size_t scratch_bytes, void *cuda_stream, es_shard_t **out);
+
+/* Prefill: runs the shard over B prompts of T tokens each, filling the KV cache of the given slots
+ * from position 0 (earlier content of those slots is discarded).
+ *   ids        dev int32 [B, T]   — required iff the shard holds the embedding, else NULL
+ *   hidden_in  fp32 [B, T, d_model] view of the previous shard's handoff — required iff it does not
+ *   slots      host int32 [B], distinct, each in [0, max_slots)
+ * Result: es_shard_handoff() gives hidden [B, T, d_model]; with the output layer also logits of the
+ * LAST prompt position [B, vocab] and the greedy token [B] (lowest index wins ties). */
+ES_API es_status_t es_shard_prefill(es_shard_t *shard, const int32_t *ids, const es_tensor_t *hidden_in,
+                             int32_t B, int32_t T, const int32_t *slots);
+
+/* One autoregressive step for B sequences: each consumes one token (ids dev int32 [B]) or one
+ * activation row (hidden_in fp32 [B, d_model]) at its slot's next position and attends to the
+ * slot's cached keys/values.  ES_ERR_STATE if a slot has no prefilled context, ES_ERR_KV_FULL if
+ * it is at max_seq.  `ids` may be the next_ids pointer returned by es_shard_handoff (greedy
+ * feedback without leaving the device). */
+ES_API es_status_t es_shard_decode_step(es_shard_t *shard, const int32_t *ids, const es_tensor_t *hidden_in,
+                                 int32_t B, const int32_t *slots);
+
+/* The inter-shard activation of the most recent prefill/decode call: the residual stream after
+ * layer layer_end-1, fp32, [B, T, d_model] after a prefill and [B, 1, d_model] after a decode step
+ * (size O_i of the paper; on the same device the hand-over is this pointer, zero copy).  With the
+ * output layer, `logits` (fp32 [B, vocab]) and `next_ids` (int32 [B]) are filled as well, otherwise
+ * their data is NULL.  Any of the three out-pointers may be NULL.  Views stay valid, and their
+ * contents unchanged, until the next prefill/decode call on this shard. */
+ES_API es_status_t es_shard_handoff(es_shard_t *shard, es_tensor_t *hidden_out, es_tensor_t *logits,
+                             es_tensor_t *next_ids);
+
+/* Per-layer device time, activation size and memory.  Timing is collected only while profiling is
+ * switched on (es_shard_set_profiling), with one CUDA event pair per layer per call; this call
+ * synchronises the stream.  Writes min(capacity, entries) items to `out` and the number of entries
+ * (layers in the shard, plus embedding and/or head when present) to *n. */
+ES_API es_status_t es_layer_profile(es_shard_t *shard, es_layer_profile_t *out, int32_t capacity, int32_t *n);
+ES_API es_status_t es_shard_set_profiling(es_shard_t *shard, int32_t enabled);
+
+/* Forget the context of the given slots (host int32 [n]); NULL / n == 0 resets every slot. */
+ES_API es_status_t es_shard_reset_slots(es_shard_t *shard, const int32_t *slots, int32_t n);
+
+/* Replace the logical->physical KV page map: host int32 [max_slots * pages_per_slot], a permutation
+ * of 0..max_slots*pages_per_slot-1 (pages_per_slot = ceil(max_seq / kv_page_tokens)).  Resets all
+ * slots.  Results never depend on the map. */
+ES_API es_status_t es_shard_set_page_table(es_shard_t *shard, const int32_t *table);
+
+/* Run decode steps as replayed CUDA graphs (default on).  With graphs off every kernel is launched
+ * individually; results are identical. */
+ES_API es_status_t es_shard_set_graphs(es_shard_t *shard, int32_t enabled);
+
+/* Reads the device status word (synchronises): ES_OK, or ES_ERR_DEVICE_TIMEOUT if a bounded wait
+ * inside a kernel ran out since the last call. */
+ES_API es_status_t es_shard_device_status(es_shard_t *shard);
+
+/* Number of kernels this shard has launched (graph replays count their nodes). */
+ES_API int64_t es_shard_launch_count(const es_shard_t *shard);
+
+ES_API void es_shard_destroy(es_shard_t *shard);
+
+ES_API const char *es_last_error(void);
+ES_API const char *es_version(void);
+
+/* ---- single operations (the steps of the path, exposed for unit parity tests) -----------------
+ * All pointers dev unless marked host; `stream` is a cudaStream_t cast to void*.              */
+
+/* y[m,:] = x[m,:] * gain / sqrt(mean(x[m,:]^2) + eps);  x fp32 [M, d], gain fp16 [d], y fp16 [M, d]. */
+ES_API es_status_t es_op_rmsnorm(const float *x, const void *gain, void *y, int32_t M, int32_t d, float eps,
+                          void *stream);
+
+/* C = A * W^T (+ R):  A fp16 [M, K], W fp16 [N, K], C fp32 [M, N], R fp32 [M, N] or NULL.
+ * path: 0 = automatic, 1 = tensor-core (tcgen05) kernel, 2 = weight-streaming kernel (M <= 16),
+ * 3 = plain reference kernel. */
+ES_API es_status_t es_op_linear(const void *A, const void *W, const float *R, float *C, int32_t M, int32_t N,
+                         int32_t K, int32_t path, void *stream);
+
+/* Causal self-attention over a prompt.  q fp16 [B, T, Hq, hd] (already rotated); k, v fp16
+ * [B, T, Hkv, hd]; out fp16 [B, T, Hq*hd].  Query t sees keys 0..t; scale 1/sqrt(hd). */
+ES_API es_status_t es_op_prefill_attention(const void *q, const void *k, const void *v, void *out, int32_t B,
+                                    int32_t T, int32_t Hq, int32_t Hkv, int32_t hd, void *stream);
+
+/* Bytes of scratch es_op_decode_attention needs. */
+ES_API size_t es_op_decode_attention_scratch_bytes(int32_t B, int32_t Hq, int32_t hd, int32_t max_ctx,
+                                            int32_t page_tokens);
+
+/* Split-KV attention of one query row per (sequence, head) over a paged cache.
+ *   q fp16 [B, Hq, hd]; k_pages, v_pages fp16 [n_pages, Hkv, P, hd];
+ *   block_table int32 [B, pages_per_seq] (physical page of each logical page);
+ *   ctx_len int32 [B] (keys visible to the query, >= 1); out fp16 [B, Hq*hd];
+ *   scratch: dev, es_op_decode_attention_scratch_bytes(...) bytes. */
+ES_API es_status_t es_op_decode_attention(const void *q, const void *k_pages, const void *v_pages,
+                                   const int32_t *block_table, const int32_t *ctx_len, void *out,
+                                   int32_t B, int32_t Hq, int32_t Hkv, int32_t hd, int32_t page_tokens,
+                                   int32_t pages_per_seq, int32_t max_ctx, void *scratch, size_t scratch_bytes,
+                                   void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EDGESHARD_H_ */

@@ -1,0 +1,167 @@
+// Memory-bound helpers of the path: embedding gather, RMSNorm, greedy argmax, context counters.
+#include "es_internal.cuh"
+
+namespace es {
+
+namespace {
+
+// x[m, :] = table[ids[m], :] widened to fp32.  One CTA per row.
+__global__ void embed_kernel(const int* __restrict__ ids, const __half* __restrict__ table,
+                             float* __restrict__ x, int d, int vocab) {
+  const int m = blockIdx.x;
+  int id = ids[m];
+  id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);   // out-of-range ids are clamped, never dereferenced
+  const uint4* src = reinterpret_cast<const uint4*>(table + (int64_t)id * d);
+  float4* dst = reinterpret_cast<float4*>(x + (int64_t)m * d);
+  for (int c = threadIdx.x; c < d / 8; c += blockDim.x) {
+    const uint4 v = __ldg(src + c);
+    const __half2* h = reinterpret_cast<const __half2*>(&v);
+    const float2 a = __half22float2(h[0]), b = __half22float2(h[1]);
+    const float2 e = __half22float2(h[2]), f = __half22float2(h[3]);
+    dst[2 * c] = make_float4(a.x, a.y, b.x, b.y);
+    dst[2 * c + 1] = make_float4(e.x, e.y, f.x, f.y);
+  }
+}
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  const int nw = blockDim.x >> 5;
+  float t = (lane < nw) ? red[lane] : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  __syncthreads();
+  return t;
+}
+
+// One CTA per row; the row stays in registers between the two passes (up to 8 float4 per thread,
+// i.e. d <= 8192 at 256 threads); longer rows are re-read.
+constexpr int RMS_THREADS = 256;
+constexpr int RMS_REGS = 8;
+
+__global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const float* __restrict__ x,
+                                                              const __half* __restrict__ gain,
+                                                              __half* __restrict__ y, int d, float eps,
+                                                              int64_t row_stride, int64_t row_offset) {
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  const float4* src = reinterpret_cast<const float4*>(x + ((int64_t)r * row_stride + row_offset) * d);
+  const int n4 = d / 4;
+  float4 v[RMS_REGS];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < RMS_REGS; ++i) {
+    const int c = threadIdx.x + i * RMS_THREADS;
+    if (c < n4) {
+      v[i] = src[c];
+      ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+    }
+  }
+  for (int c = threadIdx.x + RMS_REGS * RMS_THREADS; c < n4; c += RMS_THREADS) {
+    const float4 t = src[c];
+    ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+  }
+  const float total = block_sum(ss, red);
+  const float inv = 1.0f / sqrtf(total / (float)d + eps);
+  __half2* dst = reinterpret_cast<__half2*>(y + (int64_t)r * d);
+  const __half2* g2 = reinterpret_cast<const __half2*>(gain);
+#pragma unroll
+  for (int i = 0; i < RMS_REGS; ++i) {
+    const int c = threadIdx.x + i * RMS_THREADS;
+    if (c < n4) {
+      const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
+      dst[2 * c] = __floats2half2_rn(v[i].x * inv * ga.x, v[i].y * inv * ga.y);
+      dst[2 * c + 1] = __floats2half2_rn(v[i].z * inv * gb.x, v[i].w * inv * gb.y);
+    }
+  }
+  for (int c = threadIdx.x + RMS_REGS * RMS_THREADS; c < n4; c += RMS_THREADS) {
+    const float4 t = src[c];
+    const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
+    dst[2 * c] = __floats2half2_rn(t.x * inv * ga.x, t.y * inv * ga.y);
+    dst[2 * c + 1] = __floats2half2_rn(t.z * inv * gb.x, t.w * inv * gb.y);
+  }
+}
+
+// Greedy token: index of the largest logit, the lowest index on ties.  One CTA per sequence.
+__global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ logits, int* __restrict__ out, int V) {
+  __shared__ float bv[8];
+  __shared__ int bi[8];
+  const float* row = logits + (int64_t)blockIdx.x * V;
+  float best = -INFINITY;
+  int idx = 0x7fffffff;
+  for (int i = threadIdx.x; i < V; i += blockDim.x) {
+    const float v = row[i];
+    if (v > best || (v == best && i < idx)) { best = v; idx = i; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+    if (ov > best || (ov == best && oi < idx)) { best = ov; idx = oi; }
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { bv[warp] = best; bi[warp] = idx; }
+  __syncthreads();
+  if (warp == 0) {
+    best = lane < 8 ? bv[lane] : -INFINITY;
+    idx = lane < 8 ? bi[lane] : 0x7fffffff;
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+      if (ov > best || (ov == best && oi < idx)) { best = ov; idx = oi; }
+    }
+    if (lane == 0) out[blockIdx.x] = (idx == 0x7fffffff) ? 0 : idx;
+  }
+}
+
+// ctx_len[slots[b]] = add ? ctx_len[..] + value : value
+__global__ void set_ctx_kernel(int* ctx_len, const int* slots, int B, int value, int add) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B) {
+    const int s = slots[b];
+    ctx_len[s] = add ? ctx_len[s] + value : value;
+  }
+}
+
+}  // namespace
+
+es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, int d, int vocab,
+                         cudaStream_t s, int64_t* launches) {
+  if (M <= 0) return ES_OK;
+  embed_kernel<<<M, 128, 0, s>>>(ids, table, x, d, vocab);
+  if (launches) ++*launches;
+  ES_CUDA_CHECK(cudaGetLastError());
+  return ES_OK;
+}
+
+es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M, int d, float eps,
+                           int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches) {
+  if (M <= 0) return ES_OK;
+  rmsnorm_kernel<<<M, RMS_THREADS, 0, s>>>(x, gain, y, d, eps, row_stride, row_offset);
+  if (launches) ++*launches;
+  ES_CUDA_CHECK(cudaGetLastError());
+  return ES_OK;
+}
+
+es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches) {
+  if (B <= 0) return ES_OK;
+  argmax_kernel<<<B, 256, 0, s>>>(logits, out, V);
+  if (launches) ++*launches;
+  ES_CUDA_CHECK(cudaGetLastError());
+  return ES_OK;
+}
+
+es_status_t launch_set_ctx(int* ctx_len, const int* slots, int B, int value, int add, cudaStream_t s,
+                           int64_t* launches) {
+  if (B <= 0) return ES_OK;
+  set_ctx_kernel<<<(B + 63) / 64, 64, 0, s>>>(ctx_len, slots, B, value, add);
+  if (launches) ++*launches;
+  ES_CUDA_CHECK(cudaGetLastError());
+  return ES_OK;
+}
+
+}  // namespace es

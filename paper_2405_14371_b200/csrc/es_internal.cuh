@@ -1,0 +1,124 @@
+// Internal declarations shared by the kernels and the host side of the shard library.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "edgeshard.h"
+
+namespace es {
+
+// ---- error plumbing -----------------------------------------------------------------------
+void set_error(const char* fmt, ...);
+es_status_t fail(es_status_t st, const char* fmt, ...);
+
+#define ES_CUDA_CHECK(expr)                                                                   \
+  do {                                                                                        \
+    cudaError_t _e = (expr);                                                                  \
+    if (_e != cudaSuccess)                                                                    \
+      return ::es::fail(ES_ERR_CUDA, "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(_e), \
+                        __FILE__, __LINE__);                                                  \
+  } while (0)
+
+#define ES_TRY(expr)                 \
+  do {                               \
+    es_status_t _s = (expr);         \
+    if (_s != ES_OK) return _s;      \
+  } while (0)
+
+// ---- the linear layer family ----------------------------------------------------------------
+// C[m, n] = sum_k A[m, k] * W[n, k], A fp16 [M, K] row-major (row stride lda), W fp16 row-major
+// [*, K].  The N output columns are a concatenation of up to three weight matrices ("segments",
+// used for Wq|Wk|Wv); with EPI_SWIGLU the kernel contracts against w[0] (gate) and w[1] (up) for
+// the same n and emits one column.
+
+enum Epilogue : int {
+  EPI_F32 = 0,     // out_f32[m, n] = acc (+ res[m, n])
+  EPI_SWIGLU = 1,  // out_f16[m, n] = silu(acc_gate) * acc_up
+  EPI_QKV = 2      // rotate q and k, q -> out_f16 [M, Nq], k/v -> paged cache
+};
+
+struct LinearParams {
+  const __half* A;
+  int64_t lda;
+  const __half* w[3];
+  int seg_rows[3];
+  int M, N, K;
+  // EPI_F32
+  float* out_f32;
+  const float* res;   // may alias out_f32 (same element read then written by one thread)
+  int64_t ldo;
+  // EPI_SWIGLU / EPI_QKV (q)
+  __half* out_f16;
+  // EPI_QKV
+  __half* k_cache;    // this layer's K pages [n_pages, Hkv, P, hd]
+  __half* v_cache;
+  const int* block_table;  // [max_slots, pages_per_slot]
+  const int* ctx_len;      // [max_slots], device-side context length of each slot
+  const int* slots;        // [B]
+  const float* rope_cos;   // [max_seq, hd/2]
+  const float* rope_sin;
+  int T;                   // rows per sequence: row m belongs to sequence m / T at prompt offset m % T
+  int is_decode;           // position = ctx_len[slot] instead of m % T
+  int Hq, Hkv, hd, P, pages_per_slot, max_seq;
+};
+
+// Kernel families.  Each returns after enqueuing; `launches` is incremented per kernel launched.
+es_status_t launch_linear_reference(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches);
+es_status_t launch_linear_stream(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches);   // M <= 16
+es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word);
+bool linear_tc_supported(const LinearParams& p, int epi);
+
+// ---- element-wise / reductions ---------------------------------------------------------------
+es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, int d, int vocab,
+                         cudaStream_t s, int64_t* launches);
+// row r of y = rmsnorm(row (r * row_stride + row_offset) of x)
+es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M, int d, float eps,
+                           int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches);
+es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches);
+es_status_t launch_set_ctx(int* ctx_len, const int* slots, int B, int value, int add, cudaStream_t s,
+                           int64_t* launches);
+
+// ---- attention -------------------------------------------------------------------------------
+// K/V addressing shared by both attention kernels: token t of sequence b, kv head g lives at
+//   base + page * page_stride + g * head_stride + (t % P) * tok_stride,
+//   page = block_table ? block_table[slot(b) * pages_per_slot + t / P] : b * pages_per_slot + t / P
+struct KvView {
+  const __half* k;
+  const __half* v;
+  const int* block_table;
+  const int* slots;       // [B] or nullptr (slot = b)
+  int64_t page_stride, head_stride, tok_stride;
+  int P, pages_per_slot;
+};
+
+__device__ __forceinline__ const __half* kv_addr(const KvView& kv, const __half* base, int slot, int t, int g) {
+  const int lp = t / kv.P;
+  const int page = kv.block_table ? kv.block_table[(int64_t)slot * kv.pages_per_slot + lp]
+                                  : slot * kv.pages_per_slot + lp;
+  return base + (int64_t)page * kv.page_stride + (int64_t)g * kv.head_stride + (int64_t)(t - lp * kv.P) * kv.tok_stride;
+}
+
+struct PrefillAttnParams {
+  const __half* q;   // [B, T, Hq, hd]
+  __half* out;       // [B, T, Hq*hd]
+  KvView kv;
+  int B, T, Hq, Hkv, hd;
+};
+es_status_t launch_prefill_attention(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches);
+
+struct DecodeAttnParams {
+  const __half* q;   // [B, Hq, hd]
+  __half* out;       // [B, Hq*hd]
+  KvView kv;
+  const int* ctx_len;     // indexed by slot (or by b when kv.slots == nullptr)
+  int ctx_add;            // keys visible = ctx_len[.] + ctx_add
+  float* part;            // scratch [B, Hq, n_splits, hd + 2]
+  int B, Hq, Hkv, hd;
+  int n_splits, pages_per_split;
+};
+size_t decode_attention_scratch_bytes(int B, int Hq, int hd, int n_splits);
+es_status_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t s, int64_t* launches);
+
+}  // namespace es

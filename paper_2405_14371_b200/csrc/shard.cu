@@ -1,0 +1,712 @@
+// Host side of the shard library: validation, buffer carving, KV page tables, the per-layer
+// launch sequence for prefill and decode, CUDA-graph replay of decode steps, per-layer event
+// timing, and the C ABI.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <map>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "es_internal.cuh"
+
+namespace es {
+
+// ---- thread-local error text ---------------------------------------------------------------
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+
+es_status_t fail(es_status_t st, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return st;
+}
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
+
+struct Layout {
+  int pages_per_slot, n_pages, n_splits, pages_per_split;
+  size_t page_elems;   // halves in one page of one of K / V
+  size_t kv_bytes;
+  size_t off_x, off_h, off_q, off_ao, off_act, off_logits, off_next, off_hlast, off_part, off_cos, off_sin,
+      off_table, off_ctx, off_slots, off_status;
+  size_t scratch_bytes;
+};
+
+void choose_splits(int max_ctx, int P, int B, int Hkv, int* n_splits, int* pages_per_split) {
+  const int pages = (max_ctx + P - 1) / P;
+  long long pps = (long long)pages * B * Hkv / (4 * 148);
+  if (pps < 1) pps = 1;
+  if (pps > pages) pps = pages;
+  *pages_per_split = (int)pps;
+  *n_splits = (pages + (int)pps - 1) / (int)pps;
+}
+
+es_status_t validate_desc(const es_model_desc_t* d, int begin, int end) {
+  if (!d) return fail(ES_ERR_INVALID_ARG, "desc is null");
+  if (d->n_layers_total <= 0 || d->d_model <= 0 || d->n_heads <= 0 || d->n_kv_heads <= 0 || d->head_dim <= 0 ||
+      d->d_ffn <= 0 || d->vocab <= 0 || d->max_slots <= 0 || d->max_seq <= 0 || d->max_tokens <= 0 ||
+      d->max_batch <= 0 || d->kv_page_tokens <= 0)
+    return fail(ES_ERR_INVALID_ARG, "model description has a non-positive field");
+  if (begin < 0 || end > d->n_layers_total || begin >= end)
+    return fail(ES_ERR_RANGE, "layer range [%d, %d) is not inside [0, %d] or is empty", begin, end, d->n_layers_total);
+  if (d->head_dim != 64 && d->head_dim != 128) return fail(ES_ERR_SHAPE, "head_dim must be 64 or 128");
+  if (d->n_heads % d->n_kv_heads != 0) return fail(ES_ERR_SHAPE, "n_heads must be a multiple of n_kv_heads");
+  const int grp = d->n_heads / d->n_kv_heads;
+  if (grp != 1 && grp != 2 && grp != 4 && grp != 8) return fail(ES_ERR_SHAPE, "n_heads / n_kv_heads must be 1, 2, 4 or 8");
+  if (d->d_model % 8 != 0 || d->d_ffn % 8 != 0) return fail(ES_ERR_SHAPE, "d_model and d_ffn must be multiples of 8");
+  if (d->kv_page_tokens < 16 || (d->kv_page_tokens & (d->kv_page_tokens - 1)))
+    return fail(ES_ERR_SHAPE, "kv_page_tokens must be a power of two >= 16");
+  if (d->max_batch > d->max_slots) return fail(ES_ERR_INVALID_ARG, "max_batch exceeds max_slots");
+  if (d->max_tokens < d->max_batch) return fail(ES_ERR_INVALID_ARG, "max_tokens is smaller than max_batch");
+  if (!(d->rms_eps >= 0.f) || !(d->rope_theta > 0.f)) return fail(ES_ERR_INVALID_ARG, "rms_eps / rope_theta out of range");
+  return ES_OK;
+}
+
+Layout make_layout(const es_model_desc_t& d, int begin, int end) {
+  Layout L{};
+  const int nl = end - begin;
+  const int P = d.kv_page_tokens;
+  L.pages_per_slot = (d.max_seq + P - 1) / P;
+  L.n_pages = L.pages_per_slot * d.max_slots;
+  L.page_elems = (size_t)d.n_kv_heads * P * d.head_dim;
+  L.kv_bytes = align_up((size_t)nl * 2 * L.n_pages * L.page_elems * sizeof(__half));
+  choose_splits(d.max_seq, P, d.max_batch, d.n_kv_heads, &L.n_splits, &L.pages_per_split);
+  const size_t M = d.max_tokens, B = d.max_batch, nq = (size_t)d.n_heads * d.head_dim;
+  const bool head = end == d.n_layers_total;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o += align_up(bytes); return at; };
+  L.off_x = take(M * d.d_model * 4);
+  L.off_h = take(M * d.d_model * 2);
+  L.off_q = take(M * nq * 2);
+  L.off_ao = take(M * nq * 2);
+  L.off_act = take(M * (size_t)d.d_ffn * 2);
+  L.off_logits = take(head ? B * (size_t)d.vocab * 4 : 0);
+  L.off_next = take(B * 4);
+  L.off_hlast = take(B * (size_t)d.d_model * 2);
+  L.off_part = take(decode_attention_scratch_bytes((int)B, d.n_heads, d.head_dim, L.n_splits));
+  L.off_cos = take((size_t)d.max_seq * (d.head_dim / 2) * 4);
+  L.off_sin = take((size_t)d.max_seq * (d.head_dim / 2) * 4);
+  L.off_table = take((size_t)L.n_pages * 4);
+  L.off_ctx = take((size_t)d.max_slots * 4);
+  L.off_slots = take(B * 4);
+  L.off_status = take(256);
+  L.scratch_bytes = o;
+  return L;
+}
+
+struct ProfileEntry {
+  int layer;
+  cudaEvent_t ev[2];
+  double prefill_ms = 0, decode_ms = 0;
+  int n_prefill = 0, n_decode = 0;
+};
+
+// A captured decode step is valid for one batch size and one pair of input pointers; slots and
+// positions are read from device memory at run time.
+struct GraphKey {
+  int B;
+  const void* ids;
+  const void* hidden;
+  bool operator<(const GraphKey& o) const {
+    if (B != o.B) return B < o.B;
+    if (ids != o.ids) return ids < o.ids;
+    return hidden < o.hidden;
+  }
+};
+
+struct GraphEntry {
+  cudaGraphExec_t exec = nullptr;
+  int64_t nodes = 0;
+};
+
+}  // namespace
+}  // namespace es
+
+using namespace es;
+
+struct es_shard {
+  es_model_desc_t d;
+  int begin, end, nl;
+  bool has_emb, has_head;
+  std::vector<es_layer_weights_t> lw;
+  const __half *emb = nullptr, *fnorm = nullptr, *lmh = nullptr;
+  cudaStream_t stream = nullptr;
+  Layout lay;
+  __half* kv = nullptr;
+  unsigned char* scratch = nullptr;
+  float* x;
+  __half *h, *q, *ao, *act, *h_last;
+  float *logits, *part, *rope_cos, *rope_sin;
+  int *next_ids, *block_table, *ctx_len, *slots_dev, *status;
+  std::vector<int> ctx;         // host mirror of ctx_len, -1 = never prefilled
+  std::vector<int> slots_host;  // slots currently uploaded to slots_dev
+  int last_B = 0, last_T = 0;
+  bool last_valid = false;
+  int64_t launches = 0;
+  bool profiling = false;
+  bool pending = false, pending_prefill = false;
+  std::vector<ProfileEntry> prof;
+  bool graphs = true;
+  std::map<GraphKey, GraphEntry> graph_cache;
+
+  __half* k_pages(int li) const { return kv + (size_t)(2 * li) * lay.n_pages * lay.page_elems; }
+  __half* v_pages(int li) const { return kv + (size_t)(2 * li + 1) * lay.n_pages * lay.page_elems; }
+};
+
+namespace es {
+namespace {
+
+es_status_t harvest_profile(es_shard* s) {
+  if (!s->pending) return ES_OK;
+  ES_CUDA_CHECK(cudaStreamSynchronize(s->stream));
+  for (auto& e : s->prof) {
+    float ms = 0.f;
+    ES_CUDA_CHECK(cudaEventElapsedTime(&ms, e.ev[0], e.ev[1]));
+    if (s->pending_prefill) { e.prefill_ms += ms; e.n_prefill++; }
+    else { e.decode_ms += ms; e.n_decode++; }
+  }
+  s->pending = false;
+  return ES_OK;
+}
+
+es_status_t upload_slots(es_shard* s, const int32_t* slots, int B) {
+  if ((int)s->slots_host.size() == B && memcmp(s->slots_host.data(), slots, B * sizeof(int)) == 0) return ES_OK;
+  s->slots_host.assign(slots, slots + B);
+  ES_CUDA_CHECK(cudaMemcpyAsync(s->slots_dev, s->slots_host.data(), B * sizeof(int), cudaMemcpyHostToDevice, s->stream));
+  return ES_OK;
+}
+
+es_status_t check_tensor(const es_tensor_t* t, int64_t rows, int64_t d, const char* what) {
+  if (!t->data) return fail(ES_ERR_INVALID_ARG, "%s: data is null", what);
+  if (t->dtype != ES_DTYPE_F32) return fail(ES_ERR_INVALID_ARG, "%s: must be fp32", what);
+  int64_t n = 1;
+  if (t->rank < 1 || t->rank > 4) return fail(ES_ERR_INVALID_ARG, "%s: bad rank", what);
+  for (int i = 0; i < t->rank; ++i) n *= t->shape[i];
+  if (n != rows * d || t->shape[t->rank - 1] != d)
+    return fail(ES_ERR_SHAPE, "%s: expected %lld x %lld elements", what, (long long)rows, (long long)d);
+  return ES_OK;
+}
+
+es_status_t run_linear(es_shard* s, const LinearParams& p, int epi) {
+  if (p.M <= 16) return launch_linear_stream(p, epi, s->stream, &s->launches);
+  if (linear_tc_supported(p, epi)) return launch_linear_tc(p, epi, s->stream, &s->launches, s->status);
+  return launch_linear_reference(p, epi, s->stream, &s->launches);
+}
+
+LinearParams base_params(const es_shard* s, int M, int T, bool decode) {
+  LinearParams p{};
+  p.M = M;
+  p.T = T;
+  p.is_decode = decode ? 1 : 0;
+  p.block_table = s->block_table;
+  p.ctx_len = s->ctx_len;
+  p.slots = s->slots_dev;
+  p.rope_cos = s->rope_cos;
+  p.rope_sin = s->rope_sin;
+  p.Hq = s->d.n_heads;
+  p.Hkv = s->d.n_kv_heads;
+  p.hd = s->d.head_dim;
+  p.P = s->d.kv_page_tokens;
+  p.pages_per_slot = s->lay.pages_per_slot;
+  p.max_seq = s->d.max_seq;
+  return p;
+}
+
+inline void prof_mark(es_shard* s, int idx, int which) {
+  if (s->profiling) cudaEventRecord(s->prof[idx].ev[which], s->stream);
+}
+
+// The launch sequence of one pass (prefill: T tokens per sequence; decode: T == 1 at each slot's
+// next position).  Everything is enqueued on s->stream.
+es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in, int B, int T, bool decode) {
+  const es_model_desc_t& d = s->d;
+  const int M = B * T;
+  const int nq = d.n_heads * d.head_dim, nkv = d.n_kv_heads * d.head_dim;
+  int pi = 0;
+  const float* xin = s->x;
+  if (s->has_emb) {
+    prof_mark(s, pi, 0);
+    ES_TRY(launch_embed(ids, s->emb, s->x, M, d.d_model, d.vocab, s->stream, &s->launches));
+    prof_mark(s, pi, 1);
+    ++pi;
+  } else {
+    xin = hidden_in;
+  }
+  for (int li = 0; li < s->nl; ++li, ++pi) {
+    const es_layer_weights_t& w = s->lw[li];
+    prof_mark(s, pi, 0);
+    ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches));
+    {
+      LinearParams p = base_params(s, M, T, decode);
+      p.A = s->h; p.lda = d.d_model; p.K = d.d_model; p.N = nq + 2 * nkv;
+      p.w[0] = (const __half*)w.wq; p.w[1] = (const __half*)w.wk; p.w[2] = (const __half*)w.wv;
+      p.seg_rows[0] = nq; p.seg_rows[1] = nkv; p.seg_rows[2] = nkv;
+      p.out_f16 = s->q; p.k_cache = s->k_pages(li); p.v_cache = s->v_pages(li);
+      ES_TRY(run_linear(s, p, EPI_QKV));
+    }
+    KvView kvv{};
+    kvv.k = s->k_pages(li); kvv.v = s->v_pages(li);
+    kvv.block_table = s->block_table; kvv.slots = s->slots_dev;
+    kvv.page_stride = (int64_t)s->lay.page_elems; kvv.head_stride = (int64_t)d.kv_page_tokens * d.head_dim;
+    kvv.tok_stride = d.head_dim; kvv.P = d.kv_page_tokens; kvv.pages_per_slot = s->lay.pages_per_slot;
+    if (decode) {
+      DecodeAttnParams a{};
+      a.q = s->q; a.out = s->ao; a.kv = kvv; a.ctx_len = s->ctx_len; a.ctx_add = 1; a.part = s->part;
+      a.B = B; a.Hq = d.n_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim;
+      a.n_splits = s->lay.n_splits; a.pages_per_split = s->lay.pages_per_split;
+      ES_TRY(launch_decode_attention(a, s->stream, &s->launches));
+    } else {
+      PrefillAttnParams a{};
+      a.q = s->q; a.out = s->ao; a.kv = kvv; a.B = B; a.T = T; a.Hq = d.n_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim;
+      ES_TRY(launch_prefill_attention(a, s->stream, &s->launches));
+    }
+    {
+      LinearParams p = base_params(s, M, T, decode);
+      p.A = s->ao; p.lda = nq; p.K = nq; p.N = d.d_model;
+      p.w[0] = (const __half*)w.wo; p.seg_rows[0] = d.d_model;
+      p.out_f32 = s->x; p.res = xin; p.ldo = d.d_model;
+      ES_TRY(run_linear(s, p, EPI_F32));
+    }
+    xin = s->x;
+    ES_TRY(launch_rmsnorm(s->x, (const __half*)w.ffn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches));
+    {
+      LinearParams p = base_params(s, M, T, decode);
+      p.A = s->h; p.lda = d.d_model; p.K = d.d_model; p.N = d.d_ffn;
+      p.w[0] = (const __half*)w.w_gate; p.w[1] = (const __half*)w.w_up; p.seg_rows[0] = d.d_ffn;
+      p.out_f16 = s->act; p.ldo = d.d_ffn;
+      ES_TRY(run_linear(s, p, EPI_SWIGLU));
+    }
+    {
+      LinearParams p = base_params(s, M, T, decode);
+      p.A = s->act; p.lda = d.d_ffn; p.K = d.d_ffn; p.N = d.d_model;
+      p.w[0] = (const __half*)w.w_down; p.seg_rows[0] = d.d_model;
+      p.out_f32 = s->x; p.res = s->x; p.ldo = d.d_model;
+      ES_TRY(run_linear(s, p, EPI_F32));
+    }
+    prof_mark(s, pi, 1);
+  }
+  if (s->has_head) {
+    prof_mark(s, pi, 0);
+    // last position of every sequence only
+    ES_TRY(launch_rmsnorm(s->x, s->fnorm, s->h_last, B, d.d_model, d.rms_eps, T, T - 1, s->stream, &s->launches));
+    for (int b0 = 0; b0 < B; b0 += 16) {
+      LinearParams p = base_params(s, (B - b0 < 16 ? B - b0 : 16), 1, decode);
+      p.A = s->h_last + (size_t)b0 * d.d_model; p.lda = d.d_model; p.K = d.d_model; p.N = d.vocab;
+      p.w[0] = s->lmh; p.seg_rows[0] = d.vocab;
+      p.out_f32 = s->logits + (size_t)b0 * d.vocab; p.res = nullptr; p.ldo = d.vocab;
+      ES_TRY(launch_linear_stream(p, EPI_F32, s->stream, &s->launches));
+    }
+    ES_TRY(launch_argmax(s->logits, s->next_ids, B, d.vocab, s->stream, &s->launches));
+    prof_mark(s, pi, 1);
+  }
+  // the slots' contexts now hold T (prefill) or one more (decode) position
+  ES_TRY(launch_set_ctx(s->ctx_len, s->slots_dev, B, decode ? 1 : T, decode ? 1 : 0, s->stream, &s->launches));
+  return ES_OK;
+}
+
+es_status_t check_slots(const es_shard* s, const int32_t* slots, int B) {
+  if (!slots) return fail(ES_ERR_INVALID_ARG, "slots is null");
+  for (int b = 0; b < B; ++b) {
+    if (slots[b] < 0 || slots[b] >= s->d.max_slots)
+      return fail(ES_ERR_RANGE, "slot %d (batch row %d) outside [0, %d)", slots[b], b, s->d.max_slots);
+    for (int c = 0; c < b; ++c)
+      if (slots[c] == slots[b]) return fail(ES_ERR_INVALID_ARG, "slot %d appears twice in the batch", slots[b]);
+  }
+  return ES_OK;
+}
+
+es_status_t check_inputs(const es_shard* s, const int32_t* ids, const es_tensor_t* hidden_in, int64_t rows,
+                         const float** hin) {
+  *hin = nullptr;
+  if (s->has_emb) {
+    if (!ids || hidden_in) return fail(ES_ERR_INVALID_ARG, "this shard holds the embedding: pass ids, not hidden_in");
+  } else {
+    if (ids || !hidden_in) return fail(ES_ERR_INVALID_ARG, "this shard starts at layer %d: pass hidden_in, not ids", s->begin);
+    ES_TRY(check_tensor(hidden_in, rows, s->d.d_model, "hidden_in"));
+    *hin = (const float*)hidden_in->data;
+  }
+  return ES_OK;
+}
+
+}  // namespace
+}  // namespace es
+
+// =============================================================================================
+// C ABI
+
+extern "C" {
+
+const char* es_last_error(void) { return es::g_err; }
+const char* es_version(void) { return "edgeshard-b200 0.1 (sm_100a)"; }
+
+es_status_t es_shard_workspace_bytes(const es_model_desc_t* desc, int32_t layer_begin, int32_t layer_end,
+                                     size_t* kv_bytes, size_t* scratch_bytes) {
+  ES_TRY(validate_desc(desc, layer_begin, layer_end));
+  const Layout L = make_layout(*desc, layer_begin, layer_end);
+  if (kv_bytes) *kv_bytes = L.kv_bytes;
+  if (scratch_bytes) *scratch_bytes = L.scratch_bytes;
+  return ES_OK;
+}
+
+es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, int32_t layer_end,
+                            const es_weights_t* weights, void* kv_buffer, size_t kv_bytes, void* scratch_buffer,
+                            size_t scratch_bytes, void* cuda_stream, es_shard_t** out) {
+  ES_TRY(validate_desc(desc, layer_begin, layer_end));
+  if (!weights || !weights->layers || !kv_buffer || !scratch_buffer || !out)
+    return fail(ES_ERR_INVALID_ARG, "null argument");
+  const Layout L = make_layout(*desc, layer_begin, layer_end);
+  if (kv_bytes < L.kv_bytes) return fail(ES_ERR_WORKSPACE, "kv buffer: %zu bytes given, %zu needed", kv_bytes, L.kv_bytes);
+  if (scratch_bytes < L.scratch_bytes)
+    return fail(ES_ERR_WORKSPACE, "scratch buffer: %zu bytes given, %zu needed", scratch_bytes, L.scratch_bytes);
+  if (((uintptr_t)kv_buffer | (uintptr_t)scratch_buffer) % ALIGN)
+    return fail(ES_ERR_INVALID_ARG, "kv / scratch buffers must be %zu-byte aligned", ALIGN);
+  const bool has_emb = layer_begin == 0, has_head = layer_end == desc->n_layers_total;
+  if (has_emb && !weights->tok_embedding) return fail(ES_ERR_INVALID_ARG, "tok_embedding is required when layer_begin == 0");
+  if (has_head && (!weights->final_norm || !weights->lm_head))
+    return fail(ES_ERR_INVALID_ARG, "final_norm and lm_head are required when layer_end == n_layers_total");
+  const int nl = layer_end - layer_begin;
+  for (int i = 0; i < nl; ++i) {
+    const es_layer_weights_t& w = weights->layers[i];
+    const void* ptrs[9] = {w.attn_norm, w.wq, w.wk, w.wv, w.wo, w.ffn_norm, w.w_gate, w.w_up, w.w_down};
+    for (int j = 0; j < 9; ++j) {
+      if (!ptrs[j]) return fail(ES_ERR_INVALID_ARG, "layer %d: weight pointer %d is null", layer_begin + i, j);
+      if ((uintptr_t)ptrs[j] % 16) return fail(ES_ERR_INVALID_ARG, "layer %d: weight pointer %d is not 16-byte aligned", layer_begin + i, j);
+    }
+  }
+  es_shard* s = new (std::nothrow) es_shard();
+  if (!s) return fail(ES_ERR_INVALID_ARG, "out of host memory");
+  s->d = *desc;
+  s->begin = layer_begin; s->end = layer_end; s->nl = nl;
+  s->has_emb = has_emb; s->has_head = has_head;
+  s->lw.assign(weights->layers, weights->layers + nl);
+  s->emb = (const __half*)weights->tok_embedding;
+  s->fnorm = (const __half*)weights->final_norm;
+  s->lmh = (const __half*)weights->lm_head;
+  s->stream = (cudaStream_t)cuda_stream;
+  s->lay = L;
+  s->kv = (__half*)kv_buffer;
+  unsigned char* sb = (unsigned char*)scratch_buffer;
+  s->scratch = sb;
+  s->x = (float*)(sb + L.off_x);
+  s->h = (__half*)(sb + L.off_h);
+  s->q = (__half*)(sb + L.off_q);
+  s->ao = (__half*)(sb + L.off_ao);
+  s->act = (__half*)(sb + L.off_act);
+  s->logits = (float*)(sb + L.off_logits);
+  s->next_ids = (int*)(sb + L.off_next);
+  s->h_last = (__half*)(sb + L.off_hlast);
+  s->part = (float*)(sb + L.off_part);
+  s->rope_cos = (float*)(sb + L.off_cos);
+  s->rope_sin = (float*)(sb + L.off_sin);
+  s->block_table = (int*)(sb + L.off_table);
+  s->ctx_len = (int*)(sb + L.off_ctx);
+  s->slots_dev = (int*)(sb + L.off_slots);
+  s->status = (int*)(sb + L.off_status);
+  s->ctx.assign(desc->max_slots, -1);
+
+  auto bail = [&](es_status_t st) { delete s; return st; };
+  // rotary table: angle = pos * theta^(-2i/hd), evaluated in double, stored as fp32
+  {
+    const int half_hd = desc->head_dim / 2;
+    std::vector<float> c((size_t)desc->max_seq * half_hd), sn(c.size());
+    for (int i = 0; i < half_hd; ++i) {
+      const double inv = pow((double)desc->rope_theta, -2.0 * i / desc->head_dim);
+      for (int p = 0; p < desc->max_seq; ++p) {
+        c[(size_t)p * half_hd + i] = (float)cos(p * inv);
+        sn[(size_t)p * half_hd + i] = (float)sin(p * inv);
+      }
+    }
+    std::vector<int> table(L.n_pages);
+    for (int i = 0; i < L.n_pages; ++i) table[i] = i;
+    cudaError_t e = cudaMemcpyAsync(s->rope_cos, c.data(), c.size() * 4, cudaMemcpyHostToDevice, s->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(s->rope_sin, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice, s->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(s->block_table, table.data(), table.size() * 4, cudaMemcpyHostToDevice, s->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(s->ctx_len, 0, (size_t)desc->max_slots * 4, s->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(s->status, 0, 256, s->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(s->kv, 0, L.kv_bytes, s->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);
+    if (e != cudaSuccess) return bail(fail(ES_ERR_CUDA, "shard initialisation failed: %s", cudaGetErrorString(e)));
+  }
+  // profile entries: [embedding] layers... [head]
+  auto add_entry = [&](int layer) {
+    ProfileEntry pe;
+    pe.layer = layer;
+    cudaEventCreate(&pe.ev[0]);
+    cudaEventCreate(&pe.ev[1]);
+    s->prof.push_back(pe);
+  };
+  if (has_emb) add_entry(-1);
+  for (int i = layer_begin; i < layer_end; ++i) add_entry(i);
+  if (has_head) add_entry(desc->n_layers_total);
+  if (cudaGetLastError() != cudaSuccess) return bail(fail(ES_ERR_CUDA, "event creation failed"));
+  *out = s;
+  return ES_OK;
+}
+
+void es_shard_destroy(es_shard_t* s) {
+  if (!s) return;
+  cudaStreamSynchronize(s->stream);
+  for (auto& e : s->prof) { cudaEventDestroy(e.ev[0]); cudaEventDestroy(e.ev[1]); }
+  for (auto& g : s->graph_cache) if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
+  delete s;
+}
+
+es_status_t es_shard_prefill(es_shard_t* s, const int32_t* ids, const es_tensor_t* hidden_in, int32_t B, int32_t T,
+                             const int32_t* slots) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  if (B <= 0 || T <= 0) return fail(ES_ERR_INVALID_ARG, "B and T must be positive");
+  if (B > s->d.max_batch) return fail(ES_ERR_RANGE, "B = %d exceeds max_batch = %d", B, s->d.max_batch);
+  if ((int64_t)B * T > s->d.max_tokens) return fail(ES_ERR_RANGE, "B*T = %lld exceeds max_tokens = %d", (long long)B * T, s->d.max_tokens);
+  if (T > s->d.max_seq) return fail(ES_ERR_KV_FULL, "prompt of %d tokens exceeds max_seq = %d", T, s->d.max_seq);
+  ES_TRY(check_slots(s, slots, B));
+  const float* hin;
+  ES_TRY(check_inputs(s, ids, hidden_in, (int64_t)B * T, &hin));
+  if (s->profiling) ES_TRY(harvest_profile(s));
+  ES_TRY(upload_slots(s, slots, B));
+  s->last_valid = false;
+  ES_TRY(enqueue_pass(s, ids, hin, B, T, false));
+  for (int b = 0; b < B; ++b) s->ctx[slots[b]] = T;
+  s->last_B = B; s->last_T = T; s->last_valid = true;
+  if (s->profiling) { s->pending = true; s->pending_prefill = true; }
+  return ES_OK;
+}
+
+es_status_t es_shard_decode_step(es_shard_t* s, const int32_t* ids, const es_tensor_t* hidden_in, int32_t B,
+                                 const int32_t* slots) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  if (B <= 0) return fail(ES_ERR_INVALID_ARG, "B must be positive");
+  if (B > s->d.max_batch) return fail(ES_ERR_RANGE, "B = %d exceeds max_batch = %d", B, s->d.max_batch);
+  ES_TRY(check_slots(s, slots, B));
+  for (int b = 0; b < B; ++b) {
+    const int c = s->ctx[slots[b]];
+    if (c <= 0) return fail(ES_ERR_STATE, "slot %d has no prefilled context", slots[b]);
+    if (c + 1 > s->d.max_seq) return fail(ES_ERR_KV_FULL, "slot %d is full (%d of %d positions)", slots[b], c, s->d.max_seq);
+  }
+  const float* hin;
+  ES_TRY(check_inputs(s, ids, hidden_in, B, &hin));
+  if (s->profiling) ES_TRY(harvest_profile(s));
+  ES_TRY(upload_slots(s, slots, B));
+  s->last_valid = false;
+
+  const bool use_graph = s->graphs && !s->profiling;
+  if (!use_graph) {
+    ES_TRY(enqueue_pass(s, ids, hin, B, 1, true));
+  } else {
+    GraphKey key{B, ids, hin};
+    auto it = s->graph_cache.find(key);
+    if (it == s->graph_cache.end()) {
+      // capture the step once; positions live in device memory, so the same graph serves every step
+      if (s->graph_cache.size() >= 64) {
+        for (auto& g : s->graph_cache) if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
+        s->graph_cache.clear();
+      }
+      ES_CUDA_CHECK(cudaStreamSynchronize(s->stream));
+      const int64_t before = s->launches;
+      ES_CUDA_CHECK(cudaStreamBeginCapture(s->stream, cudaStreamCaptureModeThreadLocal));
+      es_status_t st = enqueue_pass(s, ids, hin, B, 1, true);
+      cudaGraph_t graph = nullptr;
+      cudaError_t e = cudaStreamEndCapture(s->stream, &graph);
+      const int64_t nodes = s->launches - before;
+      s->launches = before;
+      if (st != ES_OK) { if (graph) cudaGraphDestroy(graph); return st; }
+      if (e != cudaSuccess) return fail(ES_ERR_CUDA, "graph capture failed: %s", cudaGetErrorString(e));
+      GraphEntry ge;
+      e = cudaGraphInstantiate(&ge.exec, graph, 0);
+      cudaGraphDestroy(graph);
+      if (e != cudaSuccess) return fail(ES_ERR_CUDA, "graph instantiation failed: %s", cudaGetErrorString(e));
+      ge.nodes = nodes;
+      it = s->graph_cache.emplace(key, ge).first;
+    }
+    ES_CUDA_CHECK(cudaGraphLaunch(it->second.exec, s->stream));
+    s->launches += it->second.nodes;
+  }
+  for (int b = 0; b < B; ++b) s->ctx[slots[b]] += 1;
+  s->last_B = B; s->last_T = 1; s->last_valid = true;
+  if (s->profiling) { s->pending = true; s->pending_prefill = false; }
+  return ES_OK;
+}
+
+es_status_t es_shard_handoff(es_shard_t* s, es_tensor_t* hidden_out, es_tensor_t* logits, es_tensor_t* next_ids) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  if (!s->last_valid) return fail(ES_ERR_STATE, "no completed prefill/decode call to hand off");
+  if (hidden_out) {
+    hidden_out->data = s->x; hidden_out->dtype = ES_DTYPE_F32; hidden_out->rank = 3;
+    hidden_out->shape[0] = s->last_B; hidden_out->shape[1] = s->last_T; hidden_out->shape[2] = s->d.d_model; hidden_out->shape[3] = 1;
+  }
+  if (logits) {
+    logits->data = s->has_head ? s->logits : nullptr; logits->dtype = ES_DTYPE_F32; logits->rank = 2;
+    logits->shape[0] = s->last_B; logits->shape[1] = s->d.vocab; logits->shape[2] = logits->shape[3] = 1;
+  }
+  if (next_ids) {
+    next_ids->data = s->has_head ? s->next_ids : nullptr; next_ids->dtype = ES_DTYPE_I32; next_ids->rank = 1;
+    next_ids->shape[0] = s->last_B; next_ids->shape[1] = next_ids->shape[2] = next_ids->shape[3] = 1;
+  }
+  return ES_OK;
+}
+
+es_status_t es_shard_set_profiling(es_shard_t* s, int32_t enabled) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  if (!enabled && s->profiling) ES_TRY(harvest_profile(s));
+  s->profiling = enabled != 0;
+  return ES_OK;
+}
+
+es_status_t es_layer_profile(es_shard_t* s, es_layer_profile_t* out, int32_t capacity, int32_t* n) {
+  if (!s || !n) return fail(ES_ERR_INVALID_ARG, "null argument");
+  if (capacity > 0 && !out) return fail(ES_ERR_INVALID_ARG, "out is null");
+  ES_TRY(harvest_profile(s));
+  const es_model_desc_t& d = s->d;
+  const int64_t nq = (int64_t)d.n_heads * d.head_dim, nkv = (int64_t)d.n_kv_heads * d.head_dim;
+  const int64_t layer_w = 2 * (2 * (int64_t)d.d_model + nq * d.d_model + 2 * nkv * d.d_model + d.d_model * nq + 3 * (int64_t)d.d_model * d.d_ffn);
+  const int64_t layer_kv = 2 * (int64_t)s->lay.n_pages * s->lay.page_elems * 2;
+  int i = 0;
+  for (const auto& e : s->prof) {
+    if (i < capacity) {
+      es_layer_profile_t& o = out[i];
+      o.layer = e.layer;
+      o.n_prefill = e.n_prefill; o.n_decode = e.n_decode;
+      o.prefill_ms_mean = e.n_prefill ? (float)(e.prefill_ms / e.n_prefill) : 0.f;
+      o.decode_ms_mean = e.n_decode ? (float)(e.decode_ms / e.n_decode) : 0.f;
+      const int tok = e.n_prefill + e.n_decode;
+      o.avg_ms_per_token = tok ? (float)((e.prefill_ms + e.decode_ms) / tok) : 0.f;
+      if (e.layer == -1) { o.activation_bytes = (int64_t)d.d_model * 4; o.weight_bytes = 2 * (int64_t)d.vocab * d.d_model; o.kv_bytes = 0; }
+      else if (e.layer == d.n_layers_total) { o.activation_bytes = (int64_t)d.vocab * 4; o.weight_bytes = 2 * ((int64_t)d.vocab * d.d_model + d.d_model); o.kv_bytes = 0; }
+      else { o.activation_bytes = (int64_t)d.d_model * 4; o.weight_bytes = layer_w; o.kv_bytes = layer_kv; }
+    }
+    ++i;
+  }
+  *n = i;
+  return ES_OK;
+}
+
+es_status_t es_shard_reset_slots(es_shard_t* s, const int32_t* slots, int32_t n) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  if (!slots || n <= 0) {
+    std::fill(s->ctx.begin(), s->ctx.end(), -1);
+    ES_CUDA_CHECK(cudaMemsetAsync(s->ctx_len, 0, (size_t)s->d.max_slots * 4, s->stream));
+    return ES_OK;
+  }
+  for (int i = 0; i < n; ++i)
+    if (slots[i] < 0 || slots[i] >= s->d.max_slots) return fail(ES_ERR_RANGE, "slot %d out of range", slots[i]);
+  for (int i = 0; i < n; ++i) {
+    s->ctx[slots[i]] = -1;
+    ES_CUDA_CHECK(cudaMemsetAsync(s->ctx_len + slots[i], 0, 4, s->stream));
+  }
+  return ES_OK;
+}
+
+es_status_t es_shard_set_page_table(es_shard_t* s, const int32_t* table) {
+  if (!s || !table) return fail(ES_ERR_INVALID_ARG, "null argument");
+  const int n = s->lay.n_pages;
+  std::vector<char> seen(n, 0);
+  for (int i = 0; i < n; ++i) {
+    if (table[i] < 0 || table[i] >= n || seen[table[i]]) return fail(ES_ERR_INVALID_ARG, "page table is not a permutation of 0..%d", n - 1);
+    seen[table[i]] = 1;
+  }
+  ES_CUDA_CHECK(cudaStreamSynchronize(s->stream));
+  ES_CUDA_CHECK(cudaMemcpy(s->block_table, table, (size_t)n * 4, cudaMemcpyHostToDevice));
+  return es_shard_reset_slots(s, nullptr, 0);
+}
+
+es_status_t es_shard_set_graphs(es_shard_t* s, int32_t enabled) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  s->graphs = enabled != 0;
+  return ES_OK;
+}
+
+es_status_t es_shard_device_status(es_shard_t* s) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  int host[2] = {0, 0};
+  ES_CUDA_CHECK(cudaStreamSynchronize(s->stream));
+  ES_CUDA_CHECK(cudaMemcpy(host, s->status, sizeof(host), cudaMemcpyDeviceToHost));
+  if (host[0] != 0) {
+    cudaMemset(s->status, 0, 256);
+    return fail(ES_ERR_DEVICE_TIMEOUT, "a device-side wait ran out (code %d, detail %d)", host[0], host[1]);
+  }
+  return ES_OK;
+}
+
+int64_t es_shard_launch_count(const es_shard_t* s) { return s ? s->launches : 0; }
+
+// ---- single operations -----------------------------------------------------------------------
+
+es_status_t es_op_rmsnorm(const float* x, const void* gain, void* y, int32_t M, int32_t d, float eps, void* stream) {
+  if (!x || !gain || !y) return fail(ES_ERR_INVALID_ARG, "null argument");
+  if (M < 0 || d <= 0 || d % 8) return fail(ES_ERR_SHAPE, "d must be a positive multiple of 8");
+  return launch_rmsnorm(x, (const __half*)gain, (__half*)y, M, d, eps, 1, 0, (cudaStream_t)stream, nullptr);
+}
+
+es_status_t es_op_linear(const void* A, const void* W, const float* R, float* C, int32_t M, int32_t N, int32_t K,
+                         int32_t path, void* stream) {
+  if (!A || !W || !C) return fail(ES_ERR_INVALID_ARG, "null argument");
+  if (M < 0 || N <= 0 || K <= 0 || K % 8) return fail(ES_ERR_SHAPE, "N, K must be positive and K a multiple of 8");
+  LinearParams p{};
+  p.A = (const __half*)A; p.lda = K; p.w[0] = (const __half*)W; p.seg_rows[0] = N;
+  p.M = M; p.N = N; p.K = K; p.out_f32 = C; p.res = R; p.ldo = N; p.T = 1;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (path == 0) path = (M <= 16) ? 2 : (linear_tc_supported(p, EPI_F32) ? 1 : 3);
+  switch (path) {
+    case 1:
+      if (!linear_tc_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "tensor-core kernel does not take this shape");
+      return launch_linear_tc(p, EPI_F32, st, nullptr, nullptr);
+    case 2: return launch_linear_stream(p, EPI_F32, st, nullptr);
+    case 3: return launch_linear_reference(p, EPI_F32, st, nullptr);
+    default: return fail(ES_ERR_INVALID_ARG, "unknown path %d", path);
+  }
+}
+
+es_status_t es_op_prefill_attention(const void* q, const void* k, const void* v, void* out, int32_t B, int32_t T,
+                                    int32_t Hq, int32_t Hkv, int32_t hd, void* stream) {
+  if (!q || !k || !v || !out) return fail(ES_ERR_INVALID_ARG, "null argument");
+  if (B < 0 || T < 0 || Hq <= 0 || Hkv <= 0) return fail(ES_ERR_INVALID_ARG, "bad sizes");
+  PrefillAttnParams p{};
+  p.q = (const __half*)q; p.out = (__half*)out; p.B = B; p.T = T; p.Hq = Hq; p.Hkv = Hkv; p.hd = hd;
+  p.kv.k = (const __half*)k; p.kv.v = (const __half*)v; p.kv.block_table = nullptr; p.kv.slots = nullptr;
+  p.kv.page_stride = (int64_t)T * Hkv * hd; p.kv.head_stride = hd; p.kv.tok_stride = (int64_t)Hkv * hd;
+  p.kv.P = T > 0 ? T : 1; p.kv.pages_per_slot = 1;
+  return launch_prefill_attention(p, (cudaStream_t)stream, nullptr);
+}
+
+size_t es_op_decode_attention_scratch_bytes(int32_t B, int32_t Hq, int32_t hd, int32_t max_ctx, int32_t page_tokens) {
+  if (B <= 0 || Hq <= 0 || hd <= 0 || max_ctx <= 0 || page_tokens <= 0) return 0;
+  // worst case over the KV-head count: one page per split
+  return decode_attention_scratch_bytes(B, Hq, hd, (max_ctx + page_tokens - 1) / page_tokens);
+}
+
+es_status_t es_op_decode_attention(const void* q, const void* k_pages, const void* v_pages, const int32_t* block_table,
+                                   const int32_t* ctx_len, void* out, int32_t B, int32_t Hq, int32_t Hkv, int32_t hd,
+                                   int32_t page_tokens, int32_t pages_per_seq, int32_t max_ctx, void* scratch,
+                                   size_t scratch_bytes, void* stream) {
+  if (!q || !k_pages || !v_pages || !block_table || !ctx_len || !out || !scratch) return fail(ES_ERR_INVALID_ARG, "null argument");
+  if (B <= 0 || Hq <= 0 || Hkv <= 0 || page_tokens <= 0 || pages_per_seq <= 0 || max_ctx <= 0)
+    return fail(ES_ERR_INVALID_ARG, "bad sizes");
+  if (max_ctx > page_tokens * pages_per_seq) return fail(ES_ERR_RANGE, "max_ctx exceeds the block table");
+  DecodeAttnParams p{};
+  p.q = (const __half*)q; p.out = (__half*)out; p.ctx_len = ctx_len; p.ctx_add = 0; p.part = (float*)scratch;
+  p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.hd = hd;
+  p.kv.k = (const __half*)k_pages; p.kv.v = (const __half*)v_pages; p.kv.block_table = block_table; p.kv.slots = nullptr;
+  p.kv.page_stride = (int64_t)Hkv * page_tokens * hd; p.kv.head_stride = (int64_t)page_tokens * hd; p.kv.tok_stride = hd;
+  p.kv.P = page_tokens; p.kv.pages_per_slot = pages_per_seq;
+  choose_splits(max_ctx, page_tokens, B, Hkv, &p.n_splits, &p.pages_per_split);
+  if (scratch_bytes < decode_attention_scratch_bytes(B, Hq, hd, p.n_splits))
+    return fail(ES_ERR_WORKSPACE, "scratch: %zu bytes given, %zu needed", scratch_bytes,
+                decode_attention_scratch_bytes(B, Hq, hd, p.n_splits));
+  return launch_decode_attention(p, (cudaStream_t)stream, nullptr);
+}
+
+}  // extern "C"

@@ -1,0 +1,33 @@
+"""Shared test plumbing: device weights from the seeded generator, shard construction, and the
+oracle run over the same inputs.  The oracle is only ever called from here and from the tests."""
+from __future__ import annotations
+
+import torch
+
+from workload import shard_weights
+
+
+def device_weights(cfg: int, model, layer_begin: int, layer_end: int):
+    """(weights on cuda, the same weights on the host) — generated on the GPU, copied back."""
+    w = shard_weights(cfg, model, layer_begin, layer_end, device="cuda")
+    host = {k: v.cpu() for k, v in w.items() if k != "layers"}
+    host["layers"] = [{k: v.cpu() for k, v in lw.items()} for lw in w["layers"]]
+    return w, host
+
+
+def slice_weights(w: dict, model, begin: int, end: int, base: int = 0) -> dict:
+    """Weights of the sub-shard [begin, end) out of a dict that starts at layer `base`."""
+    out = {"layers": w["layers"][begin - base:end - base]}
+    if begin == 0:
+        out["tok_embedding"] = w["tok_embedding"]
+    if end == model.n_layers:
+        out["final_norm"] = w["final_norm"]
+        out["lm_head"] = w["lm_head"]
+    return out
+
+
+def rel_err(got: torch.Tensor, want: torch.Tensor) -> float:
+    """max|got - want| / max|want| over the whole tensor (the stated parity metric)."""
+    got = got.detach().double().cpu()
+    want = want.detach().double().cpu()
+    return float((got - want).abs().max() / want.abs().max())

@@ -1,0 +1,107 @@
+"""Per-kernel parity against the oracle's definitions, on small and ragged shapes (through the C ABI)."""
+import math
+
+import pytest
+import torch
+
+from oracle import decoder as O
+from tests.helpers import rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2405_14371_b200 import binding
+    return binding
+
+
+def _randn(*shape, seed=0, scale=1.0, dtype=torch.float16):
+    g = torch.Generator().manual_seed(seed)
+    return (torch.randn(*shape, generator=g) * scale).to(dtype)
+
+
+@pytest.mark.parametrize("M,d", [(1, 256), (5, 4096), (3, 8192), (2, 16384), (7, 688), (0, 256)])
+def test_rmsnorm(B, M, d):
+    x = _randn(M, d, seed=1, scale=3.0, dtype=torch.float32)
+    g = (1 + 0.1 * _randn(d, seed=2, dtype=torch.float32)).half()
+    y = B.es_op_rmsnorm(x.cuda(), g.cuda(), 1e-5)
+    torch.cuda.synchronize()
+    if M == 0:
+        return
+    want = O.rmsnorm(x.double(), g.double(), 1e-5)
+    assert rel_err(y, want) < 2e-3
+
+
+@pytest.mark.parametrize("path", [2, 3])
+@pytest.mark.parametrize("M,N,K", [(1, 256, 256), (1, 1000, 256), (3, 300, 688), (16, 768, 256), (8, 129, 1032),
+                                   (13, 4096, 4096), (1, 11008, 4096)])
+def test_linear_skinny_and_reference(B, path, M, N, K):
+    A = _randn(M, K, seed=3)
+    W = _randn(N, K, seed=4, scale=0.05)
+    R = _randn(M, N, seed=5, dtype=torch.float32)
+    want = A.double() @ W.double().T
+    got = B.es_op_linear(A.cuda(), W.cuda(), None, path)
+    assert rel_err(got, want) < 1e-5
+    got = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), path)
+    assert rel_err(got, want + R.double()) < 1e-5
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 128, 64), (100, 200, 136), (257, 1000, 688), (512, 4096, 4096)])
+def test_linear_reference_large(B, M, N, K):
+    A = _randn(M, K, seed=6)
+    W = _randn(N, K, seed=7, scale=0.05)
+    got = B.es_op_linear(A.cuda(), W.cuda(), None, 3)
+    assert rel_err(got, A.double() @ W.double().T) < 1e-5
+
+
+def test_linear_rejects_bad_shapes(B):
+    A = _randn(17, 64).cuda()
+    W = _randn(32, 64).cuda()
+    with pytest.raises(B.EsError) as e:
+        B.es_op_linear(A, W, None, 2)          # weight-streaming kernel takes <= 16 rows
+    assert e.value.status == 9
+    with pytest.raises(B.EsError) as e:
+        B.es_op_linear(_randn(2, 12).cuda(), _randn(4, 12).cuda(), None, 0)   # K % 8
+    assert e.value.status == 2
+
+
+@pytest.mark.parametrize("Bn,T,Hq,Hkv,hd", [(1, 1, 4, 4, 64), (2, 16, 4, 4, 64), (1, 37, 4, 2, 128), (2, 130, 8, 1, 128),
+                                            (1, 200, 2, 2, 64)])
+def test_prefill_attention(B, Bn, T, Hq, Hkv, hd):
+    q = _randn(Bn, T, Hq, hd, seed=8)
+    k = _randn(Bn, T, Hkv, hd, seed=9)
+    v = _randn(Bn, T, Hkv, hd, seed=10)
+    got = B.es_op_prefill_attention(q.cuda(), k.cuda(), v.cuda())
+    for b in range(Bn):
+        want = O.causal_attention_matrix(q[b].double(), k[b].double(), v[b].double()).reshape(T, Hq * hd)
+        assert rel_err(got[b], want) < 2e-3
+
+
+@pytest.mark.parametrize("Bn,Hq,Hkv,hd,P,ctxs", [
+    (1, 4, 4, 64, 16, [1]), (2, 4, 4, 64, 16, [16, 17]), (3, 8, 2, 128, 64, [5, 64, 200]),
+    (2, 8, 1, 128, 64, [300, 1]), (4, 32, 32, 128, 64, [128, 129, 255, 256]), (16, 64, 8, 128, 64, list(range(1000, 1016))),
+])
+def test_decode_attention_paged(B, Bn, Hq, Hkv, hd, P, ctxs):
+    max_ctx = max(ctxs)
+    pps = (max_ctx + P - 1) // P + 1
+    n_pages = Bn * pps
+    g = torch.Generator().manual_seed(11)
+    perm = torch.randperm(n_pages, generator=g).to(torch.int32).reshape(Bn, pps)   # scattered physical pages
+    kp = torch.zeros(n_pages, Hkv, P, hd, dtype=torch.float16)
+    vp = torch.zeros_like(kp)
+    q = _randn(Bn, Hq, hd, seed=12)
+    ks, vs = [], []
+    for b in range(Bn):
+        k = _randn(ctxs[b], Hkv, hd, seed=20 + b)
+        v = _randn(ctxs[b], Hkv, hd, seed=40 + b)
+        ks.append(k); vs.append(v)
+        for t in range(ctxs[b]):
+            pg = int(perm[b, t // P])
+            kp[pg, :, t % P, :] = k[t]
+            vp[pg, :, t % P, :] = v[t]
+    got = B.es_op_decode_attention(q.cuda(), kp.cuda(), vp.cuda(), perm.cuda(),
+                                   torch.tensor(ctxs, dtype=torch.int32).cuda(), max_ctx)
+    for b in range(Bn):
+        want = O.causal_attention_matrix(q[b:b + 1].double(), ks[b].double(), vs[b].double(), q_pos0=ctxs[b] - 1)
+        assert rel_err(got[b], want.reshape(-1)) < 2e-3

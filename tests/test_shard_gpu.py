@@ -1,0 +1,212 @@
+"""End-to-end parity of the CUDA shard against the CPU oracle on the tiny configuration, plus the
+invariants of the path (split points, batch rows, page map, graphs) and the error paths."""
+import os
+
+import pytest
+import torch
+
+from oracle import decoder as O
+from tests.helpers import device_weights, slice_weights, rel_err
+from workload import TINY, WORKLOADS, prompt_ids, forced_decode_ids
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2          # max|gpu - oracle| / max|oracle| on hidden states and logits
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2405_14371_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    return device_weights(0, TINY, 0, TINY.n_layers)
+
+
+def _golden_cfg0():
+    path = os.path.join(os.path.dirname(__file__), "golden", "cfg0_greedy.txt")
+    out = {}
+    for line in open(path):
+        if not line.startswith("#"):
+            k, *v = line.split()
+            out[k] = v
+    return int(out["seed"][0]), [int(t) for t in out["tokens"]]
+
+
+def test_cfg0_greedy_generation_matches_oracle(B, tiny):
+    wd, wh = tiny
+    wl = WORKLOADS["cfg0"]
+    seed, golden_tokens = _golden_cfg0()
+    ids = prompt_ids(0, 1, wl.prompt_len, TINY.vocab, seed=seed)
+    toks, logits, hidden = O.generate_greedy(TINY, wh, ids[0], wl.decode_steps)
+    assert toks.tolist() == golden_tokens
+
+    sh = B.Shard(TINY, 0, 2, wd, max_slots=1, max_seq=32, max_tokens=16)
+    sh.es_shard_prefill(ids.cuda(), None, 1, wl.prompt_len, [0])
+    h, l, n = sh.es_shard_handoff()
+    assert h.shape == (1, 16, 256) and l.shape == (1, 1000) and n.shape == (1,)
+    assert rel_err(h[0], hidden[:16]) < TOL
+    assert rel_err(l[0], logits[0]) < TOL
+    got = [int(n[0])]
+    for s in range(wl.decode_steps):
+        sh.es_shard_decode_step(n, None, 1, [0])       # greedy feedback stays on the device
+        h, l, n = sh.es_shard_handoff()
+        assert h.shape == (1, 1, 256)
+        assert rel_err(h[0, 0], hidden[16 + s]) < TOL
+        assert rel_err(l[0], logits[1 + s]) < TOL
+        got.append(int(n[0]))
+    assert got == golden_tokens
+    sh.es_shard_device_status()
+    assert sh.es_shard_launch_count() > 0
+    sh.close()
+
+
+@pytest.mark.parametrize("k", [1])
+def test_split_point_equals_single_shard(B, tiny, k):
+    """[0,k) then [k,L) on the GPU equals [0,L) bitwise (same kernels, same order of operations)."""
+    wd, _ = tiny
+    ids = prompt_ids(0, 2, 12, TINY.vocab).cuda()
+    nxt = forced_decode_ids(0, 2, 3, TINY.vocab).cuda()
+    full = B.Shard(TINY, 0, 2, wd, max_slots=2, max_seq=32, max_tokens=24)
+    a = B.Shard(TINY, 0, k, slice_weights(wd, TINY, 0, k), max_slots=2, max_seq=32, max_tokens=24)
+    b = B.Shard(TINY, k, 2, slice_weights(wd, TINY, k, 2), max_slots=2, max_seq=32, max_tokens=24)
+    full.es_shard_prefill(ids, None, 2, 12, [0, 1])
+    a.es_shard_prefill(ids, None, 2, 12, [0, 1])
+    ha, la, _ = a.es_shard_handoff()
+    assert la is None
+    b.es_shard_prefill(None, ha, 2, 12, [0, 1])
+    hf, lf, nf = full.es_shard_handoff()
+    hb, lb, nb = b.es_shard_handoff()
+    assert torch.equal(hf, hb) and torch.equal(lf, lb) and torch.equal(nf, nb)
+    for s in range(3):
+        full.es_shard_decode_step(nxt[s], None, 2, [0, 1])
+        a.es_shard_decode_step(nxt[s], None, 2, [0, 1])
+        ha, _, _ = a.es_shard_handoff()
+        b.es_shard_decode_step(None, ha, 2, [0, 1])
+        hf, lf, _ = full.es_shard_handoff()
+        hb, lb, _ = b.es_shard_handoff()
+        assert torch.equal(hf, hb) and torch.equal(lf, lb)
+    for s_ in (full, a, b):
+        s_.close()
+
+
+def test_batch_rows_independent_and_match_oracle(B, tiny):
+    wd, wh = tiny
+    T, S, Bn = 9, 4, 3
+    ids = prompt_ids(0, Bn, T, TINY.vocab, seed=5)
+    nxt = forced_decode_ids(0, Bn, S, TINY.vocab, seed=5)
+    sh = B.Shard(TINY, 0, 2, wd, max_slots=4, max_seq=16, max_tokens=Bn * T, kv_page_tokens=16)
+    sh.es_shard_prefill(ids.cuda(), None, Bn, T, [2, 0, 3])
+    h, l, _ = sh.es_shard_handoff()
+    hs, ls = [h.clone()], [l.clone()]
+    for s in range(S):
+        sh.es_shard_decode_step(nxt[s].cuda(), None, Bn, [2, 0, 3])
+        h, l, _ = sh.es_shard_handoff()
+        hs.append(h.clone()); ls.append(l.clone())
+    for b in range(Bn):
+        seq = torch.cat([ids[b], nxt[:, b]])
+        want_h, _ = O.shard_forward_full(TINY, wh, 0, 2, ids=seq)
+        assert rel_err(hs[0][b], want_h[:T]) < TOL
+        for s in range(S):
+            assert rel_err(hs[1 + s][b, 0], want_h[T + s]) < TOL
+            _, want_l = O.shard_forward_full(TINY, wh, 0, 2, ids=seq[:T + s + 1])
+            assert rel_err(ls[1 + s][b], want_l) < TOL
+    # the same sequence alone, in another slot, gives the same bits as inside the batch
+    sh.es_shard_prefill(ids[1:2].cuda(), None, 1, T, [1])
+    h1, l1, _ = sh.es_shard_handoff()
+    assert torch.equal(h1[0], hs[0][1]) and torch.equal(l1[0], ls[0][1])
+    sh.close()
+
+
+def test_page_map_and_graphs_do_not_change_results(B, tiny):
+    wd, _ = tiny
+    ids = prompt_ids(0, 2, 20, TINY.vocab, seed=9).cuda()
+    nxt = forced_decode_ids(0, 2, 6, TINY.vocab, seed=9).cuda()
+
+    def run(permute, graphs):
+        sh = B.Shard(TINY, 0, 2, wd, max_slots=2, max_seq=48, max_tokens=40, kv_page_tokens=16)
+        if permute:
+            g = torch.Generator().manual_seed(3)
+            sh.es_shard_set_page_table(torch.randperm(sh.n_pages, generator=g).tolist())
+        sh.es_shard_set_graphs(graphs)
+        sh.es_shard_prefill(ids, None, 2, 20, [0, 1])
+        outs = [t.clone() for t in sh.es_shard_handoff()[:2]]
+        for s in range(6):
+            sh.es_shard_decode_step(nxt[s], None, 2, [0, 1])
+            outs += [t.clone() for t in sh.es_shard_handoff()[:2]]
+        sh.close()
+        return outs
+
+    ref = run(False, False)
+    for permute, graphs in ((True, False), (False, True), (True, True)):
+        got = run(permute, graphs)
+        assert all(torch.equal(a, b) for a, b in zip(ref, got)), (permute, graphs)
+
+
+def test_profile_reports_every_layer(B, tiny):
+    wd, _ = tiny
+    ids = prompt_ids(0, 1, 16, TINY.vocab).cuda()
+    sh = B.Shard(TINY, 0, 2, wd, max_slots=1, max_seq=32, max_tokens=16)
+    sh.es_shard_set_profiling(True)
+    sh.es_shard_prefill(ids, None, 1, 16, [0])
+    _, _, n = sh.es_shard_handoff()
+    for _ in range(3):
+        sh.es_shard_decode_step(n, None, 1, [0])
+    prof = sh.es_layer_profile()
+    assert [p["layer"] for p in prof] == [-1, 0, 1, 2]
+    for p in prof:
+        assert p["n_prefill"] == 1 and p["n_decode"] == 3
+        assert p["prefill_ms_mean"] > 0 and p["decode_ms_mean"] > 0
+        want = (p["prefill_ms_mean"] + 3 * p["decode_ms_mean"]) / 4
+        assert abs(p["avg_ms_per_token"] - want) < 1e-3 * want + 1e-6
+    layer = prof[1]
+    assert layer["activation_bytes"] == 256 * 4
+    assert layer["weight_bytes"] == 2 * TINY.layer_params()
+    assert layer["kv_bytes"] == sh.kv_bytes // 2
+    assert prof[0]["weight_bytes"] == 2 * 1000 * 256 and prof[3]["activation_bytes"] == 4000
+    sh.close()
+
+
+def test_error_paths_launch_nothing(B, tiny):
+    wd, _ = tiny
+    ids = prompt_ids(0, 1, 8, TINY.vocab).cuda()
+    sh = B.Shard(TINY, 0, 2, wd, max_slots=2, max_seq=10, max_tokens=8, max_batch=1)
+    E = B.EsError
+    with pytest.raises(E) as e:
+        sh.es_shard_handoff()
+    assert e.value.status == 4
+    with pytest.raises(E) as e:
+        sh.es_shard_decode_step(ids[0, :1], None, 1, [0])          # never prefilled
+    assert e.value.status == 4
+    with pytest.raises(E) as e:
+        sh.es_shard_prefill(ids, None, 1, 8, [2])                   # slot out of range
+    assert e.value.status == 3
+    with pytest.raises(E) as e:
+        sh.es_shard_prefill(None, torch.zeros(1, 8, 256, device="cuda"), 1, 8, [0])   # needs ids
+    assert e.value.status == 1
+    with pytest.raises(E) as e:
+        sh.es_shard_prefill(ids.repeat(2, 1), None, 2, 8, [0, 1])   # B > max_batch
+    assert e.value.status == 3
+    n0 = sh.es_shard_launch_count()
+    assert n0 == 0
+    sh.es_shard_prefill(ids, None, 1, 8, [0])
+    _, _, n = sh.es_shard_handoff()
+    sh.es_shard_decode_step(n, None, 1, [0])
+    sh.es_shard_decode_step(n, None, 1, [0])
+    with pytest.raises(E) as e:
+        sh.es_shard_decode_step(n, None, 1, [0])                    # context 10 == max_seq
+    assert e.value.status == 5
+    sh.es_shard_reset_slots([0])
+    with pytest.raises(E) as e:
+        sh.es_shard_decode_step(n, None, 1, [0])
+    assert e.value.status == 4
+    b = B.Shard(TINY, 1, 2, slice_weights(wd, TINY, 1, 2), max_slots=1, max_seq=10, max_tokens=8)
+    with pytest.raises(E) as e:
+        b.es_shard_prefill(ids, None, 1, 8, [0])                    # needs hidden_in
+    assert e.value.status == 1
+    with pytest.raises(E) as e:
+        b.es_shard_prefill(None, torch.zeros(1, 8, 128, device="cuda"), 1, 8, [0])    # wrong width
+    assert e.value.status == 2
+    sh.es_shard_device_status()
+    sh.close(); b.close()
