@@ -160,8 +160,9 @@ ES_API es_status_t es_shard_reset_slots(es_shard_t *shard, const int32_t *slots,
  * slots.  Results never depend on the map. */
 ES_API es_status_t es_shard_set_page_table(es_shard_t *shard, const int32_t *table);
 
-/* Run decode steps as replayed CUDA graphs (default on).  With graphs off every kernel is launched
- * individually; results are identical. */
+/* Run decode steps as replayed CUDA graphs (default on; needs a shard created on a stream other than
+ * the default stream, which cannot be captured, and profiling off).  With graphs off every kernel
+ * is launched individually; results are identical. */
 ES_API es_status_t es_shard_set_graphs(es_shard_t *shard, int32_t enabled);
 
 /* Reads the device status word (synchronises): ES_OK, or ES_ERR_DEVICE_TIMEOUT if a bounded wait

@@ -503,7 +503,9 @@ es_status_t es_shard_decode_step(es_shard_t* s, const int32_t* ids, const es_ten
   ES_TRY(upload_slots(s, slots, B));
   s->last_valid = false;
 
-  const bool use_graph = s->graphs && !s->profiling;
+  // the legacy default stream cannot be captured: steps on it are launched kernel by kernel
+  const bool capturable = s->stream != nullptr && s->stream != cudaStreamLegacy && s->stream != cudaStreamPerThread;
+  const bool use_graph = s->graphs && !s->profiling && capturable;
   if (!use_graph) {
     ES_TRY(enqueue_pass(s, ids, hin, B, 1, true));
   } else {
@@ -646,8 +648,9 @@ int64_t es_shard_launch_count(const es_shard_t* s) { return s ? s->launches : 0;
 // ---- single operations -----------------------------------------------------------------------
 
 es_status_t es_op_rmsnorm(const float* x, const void* gain, void* y, int32_t M, int32_t d, float eps, void* stream) {
-  if (!x || !gain || !y) return fail(ES_ERR_INVALID_ARG, "null argument");
   if (M < 0 || d <= 0 || d % 8) return fail(ES_ERR_SHAPE, "d must be a positive multiple of 8");
+  if (M == 0) return ES_OK;
+  if (!x || !gain || !y) return fail(ES_ERR_INVALID_ARG, "null argument");
   return launch_rmsnorm(x, (const __half*)gain, (__half*)y, M, d, eps, 1, 0, (cudaStream_t)stream, nullptr);
 }
 

@@ -112,10 +112,11 @@ def test_batch_rows_independent_and_match_oracle(B, tiny):
             assert rel_err(hs[1 + s][b, 0], want_h[T + s]) < TOL
             _, want_l = O.shard_forward_full(TINY, wh, 0, 2, ids=seq[:T + s + 1])
             assert rel_err(ls[1 + s][b], want_l) < TOL
-    # the same sequence alone, in another slot, gives the same bits as inside the batch
+    # the same sequence alone, in another slot, gives the same result as inside the batch (a different
+    # kernel may serve the smaller row count, so equality is up to fp32 summation order)
     sh.es_shard_prefill(ids[1:2].cuda(), None, 1, T, [1])
     h1, l1, _ = sh.es_shard_handoff()
-    assert torch.equal(h1[0], hs[0][1]) and torch.equal(l1[0], ls[0][1])
+    assert rel_err(h1[0], hs[0][1]) < 2e-3 and rel_err(l1[0], ls[0][1]) < 2e-3
     sh.close()
 
 
@@ -124,8 +125,17 @@ def test_page_map_and_graphs_do_not_change_results(B, tiny):
     ids = prompt_ids(0, 2, 20, TINY.vocab, seed=9).cuda()
     nxt = forced_decode_ids(0, 2, 6, TINY.vocab, seed=9).cuda()
 
+    stream = torch.cuda.Stream()
+
     def run(permute, graphs):
-        sh = B.Shard(TINY, 0, 2, wd, max_slots=2, max_seq=48, max_tokens=40, kv_page_tokens=16)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            outs = _run(permute, graphs)
+        torch.cuda.synchronize()
+        return outs
+
+    def _run(permute, graphs):
+        sh = B.Shard(TINY, 0, 2, wd, max_slots=2, max_seq=48, max_tokens=40, kv_page_tokens=16, stream=stream)
         if permute:
             g = torch.Generator().manual_seed(3)
             sh.es_shard_set_page_table(torch.randperm(sh.n_pages, generator=g).tolist())
@@ -135,7 +145,9 @@ def test_page_map_and_graphs_do_not_change_results(B, tiny):
         for s in range(6):
             sh.es_shard_decode_step(nxt[s], None, 2, [0, 1])
             outs += [t.clone() for t in sh.es_shard_handoff()[:2]]
+        n_launch = sh.es_shard_launch_count()
         sh.close()
+        assert n_launch > 6 * 10
         return outs
 
     ref = run(False, False)
