@@ -169,6 +169,15 @@ ES_API es_status_t es_shard_set_graphs(es_shard_t *shard, int32_t enabled);
  * inside a kernel ran out since the last call. */
 ES_API es_status_t es_shard_device_status(es_shard_t *shard);
 
+/* Launch-by-launch timing of the linear-layer kernels (the weight-streaming and tensor-core
+ * products that dominate a pass): while on, every such launch is bracketed by a CUDA event pair on
+ * the shard's stream and decode steps are not replayed as graphs.  Switching it on or off clears
+ * the record.  es_shard_kernel_timing synchronises and reports the summed event time, the weight
+ * bytes those launches had to read (N*K*2 each) and their number. */
+ES_API es_status_t es_shard_set_kernel_timing(es_shard_t *shard, int32_t enabled);
+ES_API es_status_t es_shard_kernel_timing(es_shard_t *shard, double *total_ms, double *weight_bytes,
+                                          int64_t *launches);
+
 /* Number of kernels this shard has launched (graph replays count their nodes). */
 ES_API int64_t es_shard_launch_count(const es_shard_t *shard);
 

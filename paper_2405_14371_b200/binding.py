@@ -77,6 +77,8 @@ def _load() -> C.CDLL:
         "es_shard_set_graphs": (i32, [vp, i32]),
         "es_shard_device_status": (i32, [vp]),
         "es_shard_launch_count": (C.c_int64, [vp]),
+        "es_shard_set_kernel_timing": (i32, [vp, i32]),
+        "es_shard_kernel_timing": (i32, [vp, P(C.c_double), P(C.c_double), P(C.c_int64)]),
         "es_shard_destroy": (None, [vp]),
         "es_last_error": (C.c_char_p, []),
         "es_version": (C.c_char_p, []),
@@ -96,7 +98,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ("es_shard_workspace_bytes es_shard_create es_shard_prefill es_shard_decode_step es_shard_handoff "
            "es_layer_profile es_shard_set_profiling es_shard_reset_slots es_shard_set_page_table es_shard_set_graphs "
-           "es_shard_device_status es_shard_launch_count es_shard_destroy es_last_error es_version es_op_rmsnorm "
+           "es_shard_device_status es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_destroy es_last_error es_version es_op_rmsnorm "
            "es_op_linear es_op_prefill_attention es_op_decode_attention_scratch_bytes es_op_decode_attention").split()
 
 
@@ -236,6 +238,14 @@ class Shard:
 
     def es_shard_launch_count(self) -> int:
         return int(lib.es_shard_launch_count(self._handle))
+
+    def es_shard_set_kernel_timing(self, enabled: bool) -> None:
+        _check(lib.es_shard_set_kernel_timing(self._handle, int(enabled)))
+
+    def es_shard_kernel_timing(self) -> dict:
+        ms, by, n = C.c_double(0), C.c_double(0), C.c_int64(0)
+        _check(lib.es_shard_kernel_timing(self._handle, C.byref(ms), C.byref(by), C.byref(n)))
+        return {"ms": ms.value, "bytes": by.value, "launches": n.value}
 
     @property
     def n_pages(self) -> int:

@@ -163,6 +163,11 @@ struct es_shard {
   std::vector<ProfileEntry> prof;
   bool graphs = true;
   std::map<GraphKey, GraphEntry> graph_cache;
+  // launch-by-launch timing of the linear-layer kernels (off by default)
+  bool kernel_timing = false;
+  std::vector<cudaEvent_t> kt_events;   // pairs
+  size_t kt_used = 0;
+  double kt_bytes = 0;
 
   __half* k_pages(int li) const { return kv + (size_t)(2 * li) * lay.n_pages * lay.page_elems; }
   __half* v_pages(int li) const { return kv + (size_t)(2 * li + 1) * lay.n_pages * lay.page_elems; }
@@ -202,10 +207,27 @@ es_status_t check_tensor(const es_tensor_t* t, int64_t rows, int64_t d, const ch
   return ES_OK;
 }
 
-es_status_t run_linear(es_shard* s, const LinearParams& p, int epi) {
+es_status_t dispatch_linear(es_shard* s, const LinearParams& p, int epi) {
   if (p.M <= 16) return launch_linear_stream(p, epi, s->stream, &s->launches);
   if (linear_tc_supported(p, epi)) return launch_linear_tc(p, epi, s->stream, &s->launches, s->status);
   return launch_linear_reference(p, epi, s->stream, &s->launches);
+}
+
+es_status_t run_linear(es_shard* s, const LinearParams& p, int epi) {
+  if (!s->kernel_timing) return dispatch_linear(s, p, epi);
+  if (s->kt_used + 2 > s->kt_events.size()) {
+    cudaEvent_t a, b;
+    ES_CUDA_CHECK(cudaEventCreate(&a));
+    ES_CUDA_CHECK(cudaEventCreate(&b));
+    s->kt_events.push_back(a);
+    s->kt_events.push_back(b);
+  }
+  ES_CUDA_CHECK(cudaEventRecord(s->kt_events[s->kt_used], s->stream));
+  ES_TRY(dispatch_linear(s, p, epi));
+  ES_CUDA_CHECK(cudaEventRecord(s->kt_events[s->kt_used + 1], s->stream));
+  s->kt_used += 2;
+  s->kt_bytes += (double)p.N * p.K * 2.0 * (epi == EPI_SWIGLU ? 2.0 : 1.0);
+  return ES_OK;
 }
 
 LinearParams base_params(const es_shard* s, int M, int T, bool decode) {
@@ -309,7 +331,7 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       p.A = s->h_last + (size_t)b0 * d.d_model; p.lda = d.d_model; p.K = d.d_model; p.N = d.vocab;
       p.w[0] = s->lmh; p.seg_rows[0] = d.vocab;
       p.out_f32 = s->logits + (size_t)b0 * d.vocab; p.res = nullptr; p.ldo = d.vocab;
-      ES_TRY(launch_linear_stream(p, EPI_F32, s->stream, &s->launches));
+      ES_TRY(run_linear(s, p, EPI_F32));
     }
     ES_TRY(launch_argmax(s->logits, s->next_ids, B, d.vocab, s->stream, &s->launches));
     prof_mark(s, pi, 1);
@@ -463,6 +485,7 @@ void es_shard_destroy(es_shard_t* s) {
   cudaStreamSynchronize(s->stream);
   for (auto& e : s->prof) { cudaEventDestroy(e.ev[0]); cudaEventDestroy(e.ev[1]); }
   for (auto& g : s->graph_cache) if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
+  for (auto& e : s->kt_events) cudaEventDestroy(e);
   delete s;
 }
 
@@ -505,7 +528,7 @@ es_status_t es_shard_decode_step(es_shard_t* s, const int32_t* ids, const es_ten
 
   // the legacy default stream cannot be captured: steps on it are launched kernel by kernel
   const bool capturable = s->stream != nullptr && s->stream != cudaStreamLegacy && s->stream != cudaStreamPerThread;
-  const bool use_graph = s->graphs && !s->profiling && capturable;
+  const bool use_graph = s->graphs && !s->profiling && !s->kernel_timing && capturable;
   if (!use_graph) {
     ES_TRY(enqueue_pass(s, ids, hin, B, 1, true));
   } else {
@@ -644,6 +667,29 @@ es_status_t es_shard_device_status(es_shard_t* s) {
 }
 
 int64_t es_shard_launch_count(const es_shard_t* s) { return s ? s->launches : 0; }
+
+es_status_t es_shard_set_kernel_timing(es_shard_t* s, int32_t enabled) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  s->kernel_timing = enabled != 0;
+  s->kt_used = 0;
+  s->kt_bytes = 0;
+  return ES_OK;
+}
+
+es_status_t es_shard_kernel_timing(es_shard_t* s, double* total_ms, double* weight_bytes, int64_t* launches) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  ES_CUDA_CHECK(cudaStreamSynchronize(s->stream));
+  double ms = 0;
+  for (size_t i = 0; i + 1 < s->kt_used; i += 2) {
+    float t = 0.f;
+    ES_CUDA_CHECK(cudaEventElapsedTime(&t, s->kt_events[i], s->kt_events[i + 1]));
+    ms += t;
+  }
+  if (total_ms) *total_ms = ms;
+  if (weight_bytes) *weight_bytes = s->kt_bytes;
+  if (launches) *launches = (int64_t)(s->kt_used / 2);
+  return ES_OK;
+}
 
 // ---- single operations -----------------------------------------------------------------------
 
