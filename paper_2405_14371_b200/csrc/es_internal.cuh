@@ -39,7 +39,11 @@ enum Epilogue : int {
   EPI_QKV = 2      // rotate q and k, q -> out_f16 [M, Nq], k/v -> paged cache
 };
 
+// Four TMA tensor maps (A and up to three weight segments) of one tensor-core launch; opaque here.
+struct alignas(64) TcMaps { unsigned char bytes[512]; };
+
 struct LinearParams {
+  const TcMaps* tc_maps;   // host pointer to pre-encoded maps (rows of A >= M), or nullptr: encode per launch
   const __half* A;
   int64_t lda;
   const __half* w[3];
@@ -69,6 +73,8 @@ es_status_t launch_linear_reference(const LinearParams& p, int epi, cudaStream_t
 es_status_t launch_linear_stream(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches);   // M <= 16
 es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word);
 bool linear_tc_supported(const LinearParams& p, int epi);
+// Encodes the tensor maps for p's operands; the A map covers a_rows rows (the buffer's capacity).
+es_status_t tc_build_maps(const LinearParams& p, int epi, int64_t a_rows, TcMaps* out);
 
 // ---- element-wise / reductions ---------------------------------------------------------------
 es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, int d, int vocab,

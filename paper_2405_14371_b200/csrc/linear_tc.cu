@@ -1,12 +1,416 @@
-// Tensor-core (tcgen05 / TMEM / TMA) kernel of the linear-layer family.  Placeholder: not yet built.
-#include "es_internal.cuh"
+// Tensor-core kernel of the linear-layer family for sm_100a: C[M,N] = A[M,K] * W[N,K]^T with the
+// fused epilogues, for M > 16 (prefill).
+//
+// One CTA computes a 128 x BN output tile.  A single elected thread feeds a ring of shared-memory
+// stages with TMA (128-byte-swizzled K-major tiles of A and W, 64 K-elements deep); a second
+// elected thread issues tcgen05.mma (M=128, N=BN, K=16, fp16 in, fp32 accumulate) into a TMEM
+// accumulator and releases each stage with tcgen05.commit; four epilogue warps read the
+// accumulator back with tcgen05.ld (each warp its own 32-lane quarter) and run the epilogue.
+// Ragged M, N and K are handled by TMA zero fill on the way in and by guards on the way out.
+// Every wait is bounded: if a barrier does not flip within about a second the CTA records an
+// error code in the status word and leaves through the normal teardown (TMEM freed).
+#include <cuda.h>
+#include <string.h>
+
+#include "epilogue.cuh"
 
 namespace es {
 
-bool linear_tc_supported(const LinearParams&, int) { return false; }
+namespace {
 
-es_status_t launch_linear_tc(const LinearParams&, int, cudaStream_t, int64_t*, int*) {
-  return fail(ES_ERR_UNSUPPORTED, "tensor-core kernel not built");
+constexpr int BM = 128, BK = 64, UMMA_K = 16;
+constexpr int W_BOX_ROWS = 32;
+constexpr int TC_THREADS = 192;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+
+template <int BN> struct TileCfg {
+  static constexpr int B_STAGE_BYTES = BN * BK * 2;
+  static constexpr int STAGES = (BN >= 128) ? 6 : 8;
+  static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+  static constexpr size_t SMEM = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
+};
+
+struct TmapSet {
+  CUtensorMap a;
+  CUtensorMap w[3];
+};
+static_assert(sizeof(TmapSet) == sizeof(TcMaps), "TcMaps must hold four tensor maps");
+
+// ---- PTX wrappers ----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait: false if the CTA is aborting or the barrier did not flip within ~1 s.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 63u) == 0) {
+      if (*abort_flag) return false;
+      if (global_timer_ns() - t0 > 1000000000ull) {
+        *abort_flag = 1;
+        if (status) { atomicCAS(status, 0, code); status[1] = (int)blockIdx.x; }
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor for a K-major tile stored with the 128-byte swizzle: rows are
+// 128 bytes apart, groups of 8 rows 1024 bytes apart (stride byte offset), descriptor version 1.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major), 16 B units
+  d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset
+  d |= (uint64_t)1 << 46;                 // descriptor version
+  d |= (uint64_t)2 << 61;                 // layout: 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor, kind::f16: fp32 accumulator, fp16 A and B, both K-major, M x N tile.
+__host__ __device__ constexpr uint32_t umma_idesc_f16(int m, int n) {
+  return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 consecutive fp32 accumulator columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ---- the kernel --------------------------------------------------------------------------------
+template <int EPI, int BN>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int* status, int m_tiles, int n_tiles) {
+  using Cfg = TileCfg<BN>;
+  constexpr int STAGES = Cfg::STAGES;
+  constexpr int BN_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;   // output columns per tile
+
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  unsigned char* a_tiles = smem;
+  unsigned char* b_tiles = smem + (size_t)STAGES * A_STAGE_BYTES;
+  uint64_t* bars = (uint64_t*)(b_tiles + (size_t)STAGES * Cfg::B_STAGE_BYTES);
+  uint64_t* full_bar = bars;
+  uint64_t* empty_bar = bars + STAGES;
+  uint64_t* acc_bar = bars + 2 * STAGES;
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * STAGES + 1);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // tile order: groups of up to 16 row tiles share each column tile while it is hot in L2
+  constexpr int GM = 16;
+  const int tile = blockIdx.x;
+  const int per_group = GM * n_tiles;
+  const int first_m = (tile / per_group) * GM;
+  const int gsz = min(GM, m_tiles - first_m);
+  const int mt = first_m + (tile % per_group) % gsz;
+  const int nt = (tile % per_group) / gsz;
+  const int m0 = mt * BM;
+  const int n0 = nt * BN_OUT;
+  const int num_kb = (p.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&maps.a);
+    prefetch_tmap(&maps.w[0]);
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    mbar_init(smem_u32(acc_bar), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), Cfg::TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---- TMA producer ----
+      // the B stage is BN rows of W, fetched 32 rows per copy; with SwiGLU the first half of the
+      // rows comes from the gate matrix and the second half from the up matrix (same row range)
+      constexpr int N_LOADS = BN / W_BOX_ROWS;
+      const CUtensorMap* wmap[N_LOADS];
+      int wrow[N_LOADS];
+      if (EPI == EPI_SWIGLU) {
+#pragma unroll
+        for (int i = 0; i < N_LOADS; ++i) {
+          const bool up = i >= N_LOADS / 2;
+          wmap[i] = up ? &maps.w[1] : &maps.w[0];
+          wrow[i] = n0 + (up ? i - N_LOADS / 2 : i) * W_BOX_ROWS;
+        }
+      } else {
+        int n = n0, seg = 0;
+        while (seg < 2 && n >= p.seg_rows[seg]) { n -= p.seg_rows[seg]; ++seg; }
+#pragma unroll
+        for (int i = 0; i < N_LOADS; ++i) { wmap[i] = &maps.w[seg]; wrow[i] = n + i * W_BOX_ROWS; }
+      }
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, abort_flag, status, 1)) break;
+        const uint32_t fb = smem_u32(&full_bar[s]);
+        mbar_expect_tx(fb, A_STAGE_BYTES + Cfg::B_STAGE_BYTES);
+        tma_load_2d(smem_u32(a_tiles + (size_t)s * A_STAGE_BYTES), &maps.a, kb * BK, m0, fb);
+        const uint32_t bdst = smem_u32(b_tiles + (size_t)s * Cfg::B_STAGE_BYTES);
+#pragma unroll
+        for (int i = 0; i < N_LOADS; ++i)
+          tma_load_2d(bdst + i * W_BOX_ROWS * (BK * 2), wmap[i], kb * BK, wrow[i], fb);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---- MMA issuer ----
+      constexpr uint32_t idesc = umma_idesc_f16(BM, BN);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb && ok; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        ok = mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag, status, 2);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a0 = smem_u32(a_tiles + (size_t)s * A_STAGE_BYTES);
+        const uint32_t b0 = smem_u32(b_tiles + (size_t)s * Cfg::B_STAGE_BYTES);
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; ++k)
+          umma_f16(tmem_base, umma_desc_sw128(a0 + k * UMMA_K * 2), umma_desc_sw128(b0 + k * UMMA_K * 2), idesc,
+                   (kb > 0 || k > 0) ? 1u : 0u);
+        umma_commit(smem_u32(&empty_bar[s]));      // frees the stage once these MMAs have read it
+      }
+      if (ok) umma_commit(smem_u32(acc_bar));      // accumulator complete
+    }
+  } else {
+    // ---- epilogue warps: TMEM lane quarter = warp % 4 ----
+    const int quarter = warp & 3;
+    const bool ok = mbar_wait(smem_u32(acc_bar), 0, abort_flag, status, 3);
+    tc_fence_after();
+    if (ok) {
+      const int m = m0 + quarter * 32 + lane;
+      const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      if (EPI == EPI_SWIGLU) {
+#pragma unroll 1
+        for (int c = 0; c < BN_OUT; c += 32) {
+          float g[32], u[32];
+          tmem_ld32(trow + c, g);
+          tmem_ld32(trow + BN_OUT + c, u);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) epi_swiglu(p, m, n0 + c + j, g[j], u[j]);
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          float v[32];
+          tmem_ld32(trow + c, v);
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) epi_pair<EPI>(p, m, n0 + c + j, v[j], v[j + 1]);
+        }
+      }
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    if (*abort_flag) __nanosleep(100000);     // let copies still in flight land before the CTA's memory is released
+    tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+  }
+}
+
+// ---- host side -----------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)f;
+  }
+  return fn;
+}
+
+// fp16 row-major [rows, K] matrix, box = 64 K-elements x box_rows rows, 128-byte swizzle, zero fill
+es_status_t encode_2d(CUtensorMap* map, const void* base, int64_t rows, int64_t K, int64_t ld, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return fail(ES_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ES_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+  return ES_OK;
+}
+
+int pick_bn(const LinearParams& p, int epi) {
+  // widest tile that still fills the machine; segments must be whole tiles
+  const int m_tiles = (p.M + BM - 1) / BM;
+  const int cands[3] = {128, 64, 32};
+  int best = 0;
+  for (int bn : cands) {
+    const int out = (epi == EPI_SWIGLU) ? bn / 2 : bn;
+    bool fits = !(epi == EPI_SWIGLU && bn < 2 * W_BOX_ROWS);
+    if (epi == EPI_QKV)
+      for (int s = 0; s < 3; ++s) if (p.seg_rows[s] % out) fits = false;
+    if (!fits) continue;
+    if (best == 0) best = bn;
+    const long long tiles = (long long)m_tiles * ((p.N + out - 1) / out);
+    if (tiles >= 148) return bn;
+    best = bn;
+  }
+  return best;
+}
+
+template <int EPI, int BN>
+es_status_t launch_bn(const TmapSet& maps, const LinearParams& p, int* status, cudaStream_t s) {
+  constexpr int out = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
+  const int m_tiles = (p.M + BM - 1) / BM, n_tiles = (p.N + out - 1) / out;
+  auto kern = linear_tc_kernel<EPI, BN>;
+  static bool configured = false;
+  if (!configured) {
+    ES_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TileCfg<BN>::SMEM));
+    configured = true;
+  }
+  kern<<<m_tiles * n_tiles, TC_THREADS, TileCfg<BN>::SMEM, s>>>(maps, p, status, m_tiles, n_tiles);
+  ES_CUDA_CHECK(cudaGetLastError());
+  return ES_OK;
+}
+
+template <int EPI>
+es_status_t launch_epi(const TmapSet& maps, const LinearParams& p, int bn, int* status, cudaStream_t s) {
+  switch (bn) {
+    case 128: return launch_bn<EPI, 128>(maps, p, status, s);
+    case 64: return launch_bn<EPI, 64>(maps, p, status, s);
+    case 32: return launch_bn<EPI, 32>(maps, p, status, s);
+  }
+  return fail(ES_ERR_UNSUPPORTED, "no tile width for this shape");
+}
+
+}  // namespace
+
+bool linear_tc_supported(const LinearParams& p, int epi) {
+  if (p.M <= 0 || p.N <= 0 || p.K <= 0) return false;
+  if (p.K % 8 != 0 || p.lda % 8 != 0) return false;                 // TMA strides are multiples of 16 bytes
+  if (((uintptr_t)p.A | (uintptr_t)p.w[0]) % 16) return false;
+  if (epi == EPI_QKV && (((uintptr_t)p.w[1] | (uintptr_t)p.w[2]) % 16)) return false;
+  if (epi == EPI_SWIGLU && ((uintptr_t)p.w[1] % 16)) return false;
+  return pick_bn(p, epi) != 0 && encode_fn() != nullptr;
+}
+
+es_status_t tc_build_maps(const LinearParams& p, int epi, int64_t a_rows, TcMaps* out) {
+  TmapSet* t = reinterpret_cast<TmapSet*>(out);
+  memset(t, 0, sizeof(*t));
+  ES_TRY(encode_2d(&t->a, p.A, a_rows, p.K, p.lda, BM));
+  const int nseg = (epi == EPI_QKV) ? 3 : (epi == EPI_SWIGLU ? 2 : 1);
+  for (int s = 0; s < nseg; ++s) {
+    const int64_t rows = (epi == EPI_SWIGLU) ? p.N : p.seg_rows[s];
+    ES_TRY(encode_2d(&t->w[s], p.w[s], rows, p.K, p.K, W_BOX_ROWS));
+  }
+  return ES_OK;
+}
+
+es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word) {
+  if (!linear_tc_supported(p, epi)) return fail(ES_ERR_UNSUPPORTED, "tensor-core kernel does not take this shape");
+  TcMaps local;
+  const TcMaps* maps = p.tc_maps;
+  if (!maps) {
+    ES_TRY(tc_build_maps(p, epi, p.M, &local));
+    maps = &local;
+  }
+  const TmapSet& t = *reinterpret_cast<const TmapSet*>(maps);
+  const int bn = pick_bn(p, epi);
+  es_status_t st;
+  switch (epi) {
+    case EPI_F32: st = launch_epi<EPI_F32>(t, p, bn, status_word, s); break;
+    case EPI_SWIGLU: st = launch_epi<EPI_SWIGLU>(t, p, bn, status_word, s); break;
+    case EPI_QKV: st = launch_epi<EPI_QKV>(t, p, bn, status_word, s); break;
+    default: return fail(ES_ERR_INVALID_ARG, "unknown epilogue %d", epi);
+  }
+  if (st == ES_OK && launches) ++*launches;
+  return st;
 }
 
 }  // namespace es

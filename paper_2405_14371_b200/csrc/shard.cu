@@ -163,6 +163,9 @@ struct es_shard {
   std::vector<ProfileEntry> prof;
   bool graphs = true;
   std::map<GraphKey, GraphEntry> graph_cache;
+  // tensor maps of the prefill GEMMs, encoded once: [layer][qkv, o, gate/up, down]
+  std::vector<TcMaps> tmaps;
+  bool tmaps_valid = false;
   // launch-by-launch timing of the linear-layer kernels (off by default)
   bool kernel_timing = false;
   std::vector<cudaEvent_t> kt_events;   // pairs
@@ -249,6 +252,43 @@ LinearParams base_params(const es_shard* s, int M, int T, bool decode) {
   return p;
 }
 
+// Parameters of the four linear layers of decoder layer li (kind: 0 qkv, 1 o, 2 gate/up, 3 down).
+LinearParams layer_linear(const es_shard* s, int li, int kind, int M, int T, bool decode, const float* xin, int* epi) {
+  const es_model_desc_t& d = s->d;
+  const es_layer_weights_t& w = s->lw[li];
+  const int nq = d.n_heads * d.head_dim, nkv = d.n_kv_heads * d.head_dim;
+  LinearParams p = base_params(s, M, T, decode);
+  switch (kind) {
+    case 0:
+      p.A = s->h; p.lda = d.d_model; p.K = d.d_model; p.N = nq + 2 * nkv;
+      p.w[0] = (const __half*)w.wq; p.w[1] = (const __half*)w.wk; p.w[2] = (const __half*)w.wv;
+      p.seg_rows[0] = nq; p.seg_rows[1] = nkv; p.seg_rows[2] = nkv;
+      p.out_f16 = s->q; p.k_cache = s->k_pages(li); p.v_cache = s->v_pages(li);
+      *epi = EPI_QKV;
+      break;
+    case 1:
+      p.A = s->ao; p.lda = nq; p.K = nq; p.N = d.d_model;
+      p.w[0] = (const __half*)w.wo; p.seg_rows[0] = d.d_model;
+      p.out_f32 = s->x; p.res = xin; p.ldo = d.d_model;
+      *epi = EPI_F32;
+      break;
+    case 2:
+      p.A = s->h; p.lda = d.d_model; p.K = d.d_model; p.N = d.d_ffn;
+      p.w[0] = (const __half*)w.w_gate; p.w[1] = (const __half*)w.w_up; p.seg_rows[0] = d.d_ffn;
+      p.out_f16 = s->act; p.ldo = d.d_ffn;
+      *epi = EPI_SWIGLU;
+      break;
+    default:
+      p.A = s->act; p.lda = d.d_ffn; p.K = d.d_ffn; p.N = d.d_model;
+      p.w[0] = (const __half*)w.w_down; p.seg_rows[0] = d.d_model;
+      p.out_f32 = s->x; p.res = s->x; p.ldo = d.d_model;
+      *epi = EPI_F32;
+      break;
+  }
+  if (s->tmaps_valid && M > 16) p.tc_maps = &s->tmaps[(size_t)li * 4 + kind];
+  return p;
+}
+
 inline void prof_mark(es_shard* s, int idx, int which) {
   if (s->profiling) cudaEventRecord(s->prof[idx].ev[which], s->stream);
 }
@@ -258,7 +298,6 @@ inline void prof_mark(es_shard* s, int idx, int which) {
 es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in, int B, int T, bool decode) {
   const es_model_desc_t& d = s->d;
   const int M = B * T;
-  const int nq = d.n_heads * d.head_dim, nkv = d.n_kv_heads * d.head_dim;
   int pi = 0;
   const float* xin = s->x;
   if (s->has_emb) {
@@ -273,13 +312,10 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     const es_layer_weights_t& w = s->lw[li];
     prof_mark(s, pi, 0);
     ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches));
+    int epi = 0;
     {
-      LinearParams p = base_params(s, M, T, decode);
-      p.A = s->h; p.lda = d.d_model; p.K = d.d_model; p.N = nq + 2 * nkv;
-      p.w[0] = (const __half*)w.wq; p.w[1] = (const __half*)w.wk; p.w[2] = (const __half*)w.wv;
-      p.seg_rows[0] = nq; p.seg_rows[1] = nkv; p.seg_rows[2] = nkv;
-      p.out_f16 = s->q; p.k_cache = s->k_pages(li); p.v_cache = s->v_pages(li);
-      ES_TRY(run_linear(s, p, EPI_QKV));
+      LinearParams p = layer_linear(s, li, 0, M, T, decode, xin, &epi);
+      ES_TRY(run_linear(s, p, epi));
     }
     KvView kvv{};
     kvv.k = s->k_pages(li); kvv.v = s->v_pages(li);
@@ -298,27 +334,18 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       ES_TRY(launch_prefill_attention(a, s->stream, &s->launches));
     }
     {
-      LinearParams p = base_params(s, M, T, decode);
-      p.A = s->ao; p.lda = nq; p.K = nq; p.N = d.d_model;
-      p.w[0] = (const __half*)w.wo; p.seg_rows[0] = d.d_model;
-      p.out_f32 = s->x; p.res = xin; p.ldo = d.d_model;
-      ES_TRY(run_linear(s, p, EPI_F32));
+      LinearParams p = layer_linear(s, li, 1, M, T, decode, xin, &epi);
+      ES_TRY(run_linear(s, p, epi));
     }
     xin = s->x;
     ES_TRY(launch_rmsnorm(s->x, (const __half*)w.ffn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches));
     {
-      LinearParams p = base_params(s, M, T, decode);
-      p.A = s->h; p.lda = d.d_model; p.K = d.d_model; p.N = d.d_ffn;
-      p.w[0] = (const __half*)w.w_gate; p.w[1] = (const __half*)w.w_up; p.seg_rows[0] = d.d_ffn;
-      p.out_f16 = s->act; p.ldo = d.d_ffn;
-      ES_TRY(run_linear(s, p, EPI_SWIGLU));
+      LinearParams p = layer_linear(s, li, 2, M, T, decode, xin, &epi);
+      ES_TRY(run_linear(s, p, epi));
     }
     {
-      LinearParams p = base_params(s, M, T, decode);
-      p.A = s->act; p.lda = d.d_ffn; p.K = d.d_ffn; p.N = d.d_model;
-      p.w[0] = (const __half*)w.w_down; p.seg_rows[0] = d.d_model;
-      p.out_f32 = s->x; p.res = s->x; p.ldo = d.d_model;
-      ES_TRY(run_linear(s, p, EPI_F32));
+      LinearParams p = layer_linear(s, li, 3, M, T, decode, xin, &epi);
+      ES_TRY(run_linear(s, p, epi));
     }
     prof_mark(s, pi, 1);
   }
@@ -463,6 +490,18 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
     if (e == cudaSuccess) e = cudaMemsetAsync(s->kv, 0, L.kv_bytes, s->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);
     if (e != cudaSuccess) return bail(fail(ES_ERR_CUDA, "shard initialisation failed: %s", cudaGetErrorString(e)));
+  }
+  // tensor maps of the prefill GEMMs (A buffers are fixed, so one encoding serves every call)
+  if (desc->max_tokens > 16) {
+    s->tmaps.resize((size_t)nl * 4);
+    bool ok = true;
+    for (int li = 0; li < nl && ok; ++li)
+      for (int kind = 0; kind < 4 && ok; ++kind) {
+        int epi = 0;
+        LinearParams p = layer_linear(s, li, kind, desc->max_tokens, 1, false, s->x, &epi);
+        ok = linear_tc_supported(p, epi) && tc_build_maps(p, epi, desc->max_tokens, &s->tmaps[(size_t)li * 4 + kind]) == ES_OK;
+      }
+    s->tmaps_valid = ok;
   }
   // profile entries: [embedding] layers... [head]
   auto add_entry = [&](int layer) {

@@ -55,6 +55,22 @@ def test_linear_reference_large(B, M, N, K):
     assert rel_err(got, A.double() @ W.double().T) < 1e-5
 
 
+@pytest.mark.parametrize("M,N,K", [(17, 32, 64), (128, 128, 64), (100, 200, 136), (257, 1000, 688), (512, 4096, 4096),
+                                   (300, 96, 4096), (128, 4096, 11008), (1024, 640, 256), (2100, 384, 1024)])
+def test_linear_tensor_core(B, M, N, K):
+    """tcgen05 path: several tile widths, ragged M / N / K, long K, and agreement with the plain kernel."""
+    A = _randn(M, K, seed=13)
+    W = _randn(N, K, seed=14, scale=0.05)
+    R = _randn(M, N, seed=15, dtype=torch.float32)
+    want = A.double() @ W.double().T
+    got = B.es_op_linear(A.cuda(), W.cuda(), None, 1)
+    assert rel_err(got, want) < 1e-5
+    got_r = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), 1)
+    assert rel_err(got_r, want + R.double()) < 1e-5
+    ref = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), 3)
+    assert rel_err(got_r, ref) < 1e-5
+
+
 def test_linear_rejects_bad_shapes(B):
     A = _randn(17, 64).cuda()
     W = _randn(32, 64).cuda()
