@@ -64,11 +64,11 @@ def test_linear_tensor_core(B, M, N, K):
     R = _randn(M, N, seed=15, dtype=torch.float32)
     want = A.double() @ W.double().T
     got = B.es_op_linear(A.cuda(), W.cuda(), None, 1)
-    assert rel_err(got, want) < 1e-5
+    assert rel_err(got, want) < 5e-5   # fp32 tensor-core accumulation over K up to 11008
     got_r = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), 1)
-    assert rel_err(got_r, want + R.double()) < 1e-5
+    assert rel_err(got_r, want + R.double()) < 5e-5   # fp32 tensor-core accumulation over K up to 11008
     ref = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), 3)
-    assert rel_err(got_r, ref) < 1e-5
+    assert rel_err(got_r, ref) < 5e-5   # fp32 tensor-core accumulation over K up to 11008
 
 
 def test_linear_rejects_bad_shapes(B):
