@@ -219,6 +219,27 @@ ES_API es_status_t es_op_decode_attention(const void *q, const void *k_pages, co
                                    int32_t pages_per_seq, int32_t max_ctx, void *scratch, size_t scratch_bytes,
                                    void *stream);
 
+/* The same operation as es_op_decode_attention for callers that must not allocate device memory
+ * and have no buffer to lend — for instance code running under a memory pool that forbids
+ * cudaMalloc, inside a region where allocation would synchronise the device, or a plug-in that
+ * is only ever given its inputs and outputs.  (The paper has no counterpart; this is a
+ * convenience of the library.)  The split-KV partials go to an array built into the library
+ * image, es_op_decode_attention_static_capacity() bytes (8 MiB) on every GPU that loads the
+ * library, held until the process exits.  The call performs no allocation of any kind.
+ *   - A call whose partials do not fit returns ES_ERR_WORKSPACE and launches nothing; use
+ *     es_op_decode_attention with your own buffer for such sizes.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before starting any stream capture.
+ *   - All calls share the one array.  Each call overwrites what it later reads, so stale contents
+ *     are harmless, but two calls that overlap on the GPU (different streams) race: order them.
+ * Arguments and result are those of es_op_decode_attention, without scratch / scratch_bytes. */
+ES_API size_t es_op_decode_attention_static_capacity(void);
+ES_API es_status_t es_op_decode_attention_static(const void *q, const void *k_pages, const void *v_pages,
+                                                 const int32_t *block_table, const int32_t *ctx_len, void *out,
+                                                 int32_t B, int32_t Hq, int32_t Hkv, int32_t hd,
+                                                 int32_t page_tokens, int32_t pages_per_seq, int32_t max_ctx,
+                                                 void *stream);
+
 #ifdef __cplusplus
 }
 #endif

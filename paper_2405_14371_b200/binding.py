@@ -87,6 +87,8 @@ def _load() -> C.CDLL:
         "es_op_prefill_attention": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]),
         "es_op_decode_attention_scratch_bytes": (sz, [i32, i32, i32, i32, i32]),
         "es_op_decode_attention": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp]),
+        "es_op_decode_attention_static_capacity": (sz, []),
+        "es_op_decode_attention_static": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -99,7 +101,8 @@ lib = _load()
 EXPORTS = ("es_shard_workspace_bytes es_shard_create es_shard_prefill es_shard_decode_step es_shard_handoff "
            "es_layer_profile es_shard_set_profiling es_shard_reset_slots es_shard_set_page_table es_shard_set_graphs "
            "es_shard_device_status es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_destroy es_last_error es_version es_op_rmsnorm "
-           "es_op_linear es_op_prefill_attention es_op_decode_attention_scratch_bytes es_op_decode_attention").split()
+           "es_op_linear es_op_prefill_attention es_op_decode_attention_scratch_bytes es_op_decode_attention "
+           "es_op_decode_attention_static_capacity es_op_decode_attention_static").split()
 
 
 def es_last_error() -> str:
@@ -321,4 +324,24 @@ def es_op_decode_attention(q: torch.Tensor, k_pages: torch.Tensor, v_pages: torc
     _check(lib.es_op_decode_attention(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table), _ptr(ctx_len),
                                       _ptr(out), B, Hq, Hkv, hd, P, pages_per_seq, max_ctx, _ptr(scratch),
                                       scratch.numel(), _stream_ptr(stream)))
+    return out
+
+
+def es_op_decode_attention_static_capacity() -> int:
+    return int(lib.es_op_decode_attention_static_capacity())
+
+
+def es_op_decode_attention_static(q: torch.Tensor, k_pages: torch.Tensor, v_pages: torch.Tensor,
+                                  block_table: torch.Tensor, ctx_len: torch.Tensor, max_ctx: int,
+                                  out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Decode attention whose split-KV partials live in the library's built-in array: the call itself
+    allocates nothing (pass `out` to keep the binding from allocating the result either).  Calls that
+    overlap on the GPU race on that array; sizes beyond its capacity raise ES_ERR_WORKSPACE."""
+    B, Hq, hd = q.shape
+    _, Hkv, P, _ = k_pages.shape
+    if out is None:
+        out = torch.empty(B, Hq * hd, dtype=torch.float16, device=q.device)
+    _check(lib.es_op_decode_attention_static(_ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(block_table), _ptr(ctx_len),
+                                             _ptr(out), B, Hq, Hkv, hd, P, block_table.shape[1], max_ctx,
+                                             _stream_ptr(stream)))
     return out

@@ -33,6 +33,17 @@ es_status_t fail(es_status_t st, const char* fmt, ...) {
   return st;
 }
 
+// How the context of a decode-attention call is cut into splits: enough CTAs to fill the machine,
+// never less than one KV page per split.
+void choose_splits(int max_ctx, int P, int B, int Hkv, int* n_splits, int* pages_per_split) {
+  const int pages = (max_ctx + P - 1) / P;
+  long long pps = (long long)pages * B * Hkv / (4 * 148);
+  if (pps < 1) pps = 1;
+  if (pps > pages) pps = pages;
+  *pages_per_split = (int)pps;
+  *n_splits = (pages + (int)pps - 1) / (int)pps;
+}
+
 namespace {
 
 constexpr size_t ALIGN = 256;
@@ -46,15 +57,6 @@ struct Layout {
       off_table, off_ctx, off_slots, off_status;
   size_t scratch_bytes;
 };
-
-void choose_splits(int max_ctx, int P, int B, int Hkv, int* n_splits, int* pages_per_split) {
-  const int pages = (max_ctx + P - 1) / P;
-  long long pps = (long long)pages * B * Hkv / (4 * 148);
-  if (pps < 1) pps = 1;
-  if (pps > pages) pps = pages;
-  *pages_per_split = (int)pps;
-  *n_splits = (pages + (int)pps - 1) / (int)pps;
-}
 
 es_status_t validate_desc(const es_model_desc_t* d, int begin, int end) {
   if (!d) return fail(ES_ERR_INVALID_ARG, "desc is null");
