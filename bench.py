@@ -157,7 +157,7 @@ def run_ours(args):
     rank, local, world = _dist_setup(args.gpus)
     wl = WORKLOADS[args.workload]
     m = wl.model
-    Bn, T, S = wl.batch, wl.prompt_len, wl.decode_steps
+    Bn, T, S = wl.batch, wl.prompt_len, (args.decode_steps or wl.decode_steps)
     dev = torch.device("cuda", local)
     stream = torch.cuda.Stream(device=dev)
     weights = shard_weights(wl.cfg, m, wl.layer_begin, wl.layer_end, device=dev)
@@ -203,7 +203,8 @@ def run_ours(args):
 
         for _ in range(args.warmup):
             one_step(False)
-            one_step(True)
+            if not args.profile:
+                one_step(True)
         stream.synchronize()
 
         def timed(e2e: bool):
@@ -223,6 +224,15 @@ def run_ours(args):
         if rank == 0:
             sampler.start()
         pre, dec, launches = timed(False)
+        if args.profile:
+            # short run for a profiler capture: one timed pass, nothing else (not a bench value)
+            sampler.stop()
+            stream.synchronize()
+            if rank == 0:
+                print(json.dumps({"profile_run": True, "workload": args.workload, "decode_steps": S,
+                                  "prefill_ms": sum(pre) / len(pre), "decode_ms_per_step": sum(dec) / (S * len(dec)),
+                                  "gpu_launches": int(launches)}))
+            return None
         pre_e, dec_e, _ = timed(True)
         clocks = sampler.stop() if rank == 0 else None
 
@@ -362,8 +372,14 @@ def main():
     ap.add_argument("--workload", default="cfg1", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="short run for an ncu capture: 1 warm-up pass, 1 timed pass, no e2e / kernel-timing / CPU legs")
+    ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (profile runs)")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.profile:
+        args.warmup, args.steps = 1, 1
+    else:
+        args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     if args.impl == "reference":
         out = run_reference(args)

@@ -1,75 +1,136 @@
 // Split-KV decode attention over the paged cache: one query row per (sequence, head).
+//
 // A CTA takes one split (a run of KV pages) of one KV head and serves all query heads of that
-// group, so K and V are read from HBM once per group.  Inside a warp the head dimension is spread
-// over the lanes; scores are reduced with warp shuffles, the softmax is the running (max, sum)
-// form.  Each split writes an unnormalised partial (o, max, sum); a second kernel merges the
-// partials of a row in split order, so the result does not depend on scheduling.
+// group, so K and V are read from HBM once per group.  Its warps take 32 tokens at a time:
+//   * scores: one token per lane — the lane reads its token's whole K row with 16-byte loads and
+//     forms the dot products with the query rows held in shared memory (no cross-lane traffic);
+//   * softmax: running (max, sum) per head, updated once per 32 tokens with warp shuffles;
+//   * values: the head dimension is spread over the lanes (coalesced V rows), the 32
+//     probabilities are broadcast lane by lane with shuffles.
+// The warps of a CTA are merged through shared memory in warp order.  With a single split the
+// CTA writes the final output; otherwise it writes an unnormalised partial (o, max, sum) and a
+// second kernel merges the partials of a row in split order, so results never depend on
+// scheduling.
 #include "es_internal.cuh"
+#include "launch.cuh"
 
 namespace es {
 
 namespace {
 
-constexpr int DWARPS = 4;
-
-template <int E>
-__device__ __forceinline__ void load_vec(const __half* p, float (&f)[E]) {
-  if (E == 4) {
-    const uint2 u = *reinterpret_cast<const uint2*>(p);
-    const __half2* h = reinterpret_cast<const __half2*>(&u);
-    const float2 a = __half22float2(h[0]), b = __half22float2(h[1]);
-    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
-  } else {
-    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(p));
-    f[0] = a.x; f[1] = a.y;
-  }
-}
+constexpr int DWARPS = 8;
 
 template <int HD, int G>
 __global__ void __launch_bounds__(DWARPS * 32) decode_attn_split_kernel(const DecodeAttnParams p) {
+  pdl_launch_dependents();
   constexpr int E = HD / 32;
+  __shared__ __align__(16) float q_s[G][HD];
   __shared__ float sm_o[DWARPS][G][HD];
   __shared__ float sm_m[DWARPS][G];
   __shared__ float sm_l[DWARPS][G];
 
   const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_wait();
   const int slot = p.kv.slots ? p.kv.slots[b] : b;
   const int ctx = p.ctx_len[slot] + p.ctx_add;
   const int tokens_per_split = p.pages_per_split * p.kv.P;
   const int t_begin = split * tokens_per_split;
   if (t_begin >= ctx) return;
   const int t_end = min(ctx, t_begin + tokens_per_split);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const float scale = rsqrtf((float)HD);
 
-  float q[G][E], acc[G][E], m[G], l[G];
+  for (int i = threadIdx.x; i < G * HD; i += DWARPS * 32) {
+    const int j = i / HD, c = i - j * HD;
+    q_s[j][c] = __half2float(p.q[((int64_t)b * p.Hq + (g * G + j)) * HD + c]) * scale;
+  }
+  __syncthreads();
+
+  float acc[G][E], m[G], l[G];
 #pragma unroll
   for (int j = 0; j < G; ++j) {
-    load_vec<E>(p.q + ((int64_t)b * p.Hq + (g * G + j)) * HD + lane * E, q[j]);
 #pragma unroll
-    for (int e = 0; e < E; ++e) { q[j][e] *= scale; acc[j][e] = 0.f; }
+    for (int e = 0; e < E; ++e) acc[j][e] = 0.f;
     m[j] = -INFINITY;
     l[j] = 0.f;
   }
 
-  for (int t = t_begin + warp; t < t_end; t += DWARPS) {
-    float kf[E], vf[E];
-    load_vec<E>(kv_addr(p.kv, p.kv.k, slot, t, g) + lane * E, kf);
-    load_vec<E>(kv_addr(p.kv, p.kv.v, slot, t, g) + lane * E, vf);
+  for (int t0 = t_begin + warp * 32; t0 < t_end; t0 += DWARPS * 32) {
+    const int t = t0 + lane;
+    const bool valid = t < t_end;
+    // offset of this lane's token row (same for K and V), in 16-byte units
+    uint32_t off16 = 0;
+    float s[G];
+#pragma unroll
+    for (int j = 0; j < G; ++j) s[j] = 0.f;
+    if (valid) {
+      const __half* kr = kv_addr(p.kv, p.kv.k, slot, t, g);
+      off16 = (uint32_t)((kr - p.kv.k) >> 3);
+      const uint4* k4 = reinterpret_cast<const uint4*>(kr);
+      // all 16-byte pieces of the row are requested up front when registers allow (small groups)
+      constexpr int KU = (G <= 2) ? HD / 8 : 4;
+#pragma unroll KU
+      for (int c = 0; c < HD / 8; ++c) {
+        const uint4 u = k4[c];
+        const __half2* h2 = reinterpret_cast<const __half2*>(&u);
+        float kf[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __half22float2(h2[i]);
+          kf[2 * i] = f.x;
+          kf[2 * i + 1] = f.y;
+        }
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+          const float4 qa = *reinterpret_cast<const float4*>(&q_s[j][c * 8]);
+          const float4 qb = *reinterpret_cast<const float4*>(&q_s[j][c * 8 + 4]);
+          s[j] = fmaf(qa.x, kf[0], s[j]); s[j] = fmaf(qa.y, kf[1], s[j]);
+          s[j] = fmaf(qa.z, kf[2], s[j]); s[j] = fmaf(qa.w, kf[3], s[j]);
+          s[j] = fmaf(qb.x, kf[4], s[j]); s[j] = fmaf(qb.y, kf[5], s[j]);
+          s[j] = fmaf(qb.z, kf[6], s[j]); s[j] = fmaf(qb.w, kf[7], s[j]);
+        }
+      }
+    }
+    float pr[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) {
-      float s = 0.f;
+      float cm = valid ? s[j] : -INFINITY;
 #pragma unroll
-      for (int e = 0; e < E; ++e) s = fmaf(q[j][e], kf[e], s);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      const float mn = fmaxf(m[j], s);
+      for (int o = 16; o > 0; o >>= 1) cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, o));
+      const float mn = fmaxf(m[j], cm);          // finite: lane 0 of every block is valid
       const float alpha = __expf(m[j] - mn);
-      const float pj = __expf(s - mn);
-      l[j] = l[j] * alpha + pj;
+      pr[j] = valid ? __expf(s[j] - mn) : 0.f;
+      float ps = pr[j];
 #pragma unroll
-      for (int e = 0; e < E; ++e) acc[j][e] = acc[j][e] * alpha + pj * vf[e];
+      for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xffffffffu, ps, o);
+      l[j] = l[j] * alpha + ps;
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[j][e] *= alpha;
       m[j] = mn;
+    }
+    // value rows of the 32 tokens; lanes past the end carry probability 0 and a valid (repeated) offset
+    const int cnt = min(32, t_end - t0);
+    constexpr int VU = (G <= 2) ? 16 : 8;
+#pragma unroll VU
+    for (int jj = 0; jj < 32; ++jj) {
+      const uint32_t o16 = __shfl_sync(0xffffffffu, off16, jj < cnt ? jj : 0);
+      const __half* vr = p.kv.v + ((int64_t)o16 << 3) + lane * E;
+      float vf[E];
+      if (E == 4) {
+        const uint2 u = *reinterpret_cast<const uint2*>(vr);
+        const __half2* h2 = reinterpret_cast<const __half2*>(&u);
+        const float2 a = __half22float2(h2[0]), c2 = __half22float2(h2[1]);
+        vf[0] = a.x; vf[1] = a.y; vf[E - 2] = c2.x; vf[E - 1] = c2.y;
+      } else {
+        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(vr));
+        vf[0] = a.x; vf[1] = a.y;
+      }
+#pragma unroll
+      for (int j = 0; j < G; ++j) {
+        const float pv = __shfl_sync(0xffffffffu, pr[j], jj);
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[j][e] = fmaf(pv, vf[e], acc[j][e]);
+      }
     }
   }
 
@@ -93,15 +154,22 @@ __global__ void __launch_bounds__(DWARPS * 32) decode_attn_split_kernel(const De
       o += sm_o[w][j][c] * f;
       ll += sm_l[w][j] * f;
     }
-    float* dst = p.part + (((int64_t)b * p.Hq + (g * G + j)) * p.n_splits + split) * (HD + 2);
-    dst[c] = o;
-    if (c == 0) { dst[HD] = mm; dst[HD + 1] = ll; }
+    const int64_t row = (int64_t)b * p.Hq + (g * G + j);
+    if (p.n_splits == 1) {
+      p.out[row * HD + c] = __float2half_rn(o / ll);
+    } else {
+      float* dst = p.part + (row * p.n_splits + split) * (HD + 2);
+      dst[c] = o;
+      if (c == 0) { dst[HD] = mm; dst[HD + 1] = ll; }
+    }
   }
 }
 
 template <int HD>
 __global__ void __launch_bounds__(HD) decode_attn_merge_kernel(const DecodeAttnParams p) {
+  pdl_launch_dependents();
   const int h = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+  pdl_wait();
   const int slot = p.kv.slots ? p.kv.slots[b] : b;
   const int ctx = p.ctx_len[slot] + p.ctx_add;
   const int tokens_per_split = p.pages_per_split * p.kv.P;
@@ -119,19 +187,28 @@ __global__ void __launch_bounds__(HD) decode_attn_merge_kernel(const DecodeAttnP
   p.out[((int64_t)b * p.Hq + h) * HD + c] = __float2half_rn(active > 0 ? o / ll : 0.f);
 }
 
+template <int HD, int G>
+es_status_t launch_g(const DecodeAttnParams& p, cudaStream_t s, bool pdl) {
+  ES_CUDA_CHECK(launch_kernel(decode_attn_split_kernel<HD, G>, dim3(p.n_splits, p.Hkv, p.B), dim3(DWARPS * 32), 0, s, pdl, p));
+  return ES_OK;
+}
+
 template <int HD>
-es_status_t launch_hd(const DecodeAttnParams& p, cudaStream_t s) {
-  const dim3 grid(p.n_splits, p.Hkv, p.B);
+es_status_t launch_hd(const DecodeAttnParams& p, cudaStream_t s, bool pdl, int64_t* launches) {
+  es_status_t st;
   switch (p.Hq / p.Hkv) {
-    case 1: decode_attn_split_kernel<HD, 1><<<grid, DWARPS * 32, 0, s>>>(p); break;
-    case 2: decode_attn_split_kernel<HD, 2><<<grid, DWARPS * 32, 0, s>>>(p); break;
-    case 4: decode_attn_split_kernel<HD, 4><<<grid, DWARPS * 32, 0, s>>>(p); break;
-    case 8: decode_attn_split_kernel<HD, 8><<<grid, DWARPS * 32, 0, s>>>(p); break;
+    case 1: st = launch_g<HD, 1>(p, s, pdl); break;
+    case 2: st = launch_g<HD, 2>(p, s, pdl); break;
+    case 4: st = launch_g<HD, 4>(p, s, pdl); break;
+    case 8: st = launch_g<HD, 8>(p, s, pdl); break;
     default: return fail(ES_ERR_SHAPE, "query heads per KV head must be 1, 2, 4 or 8");
   }
-  ES_CUDA_CHECK(cudaGetLastError());
-  decode_attn_merge_kernel<HD><<<dim3(p.Hq, p.B), HD, 0, s>>>(p);
-  ES_CUDA_CHECK(cudaGetLastError());
+  ES_TRY(st);
+  if (launches) ++*launches;
+  if (p.n_splits > 1) {
+    ES_CUDA_CHECK(launch_kernel(decode_attn_merge_kernel<HD>, dim3(p.Hq, p.B), dim3(HD), 0, s, pdl, p));
+    if (launches) ++*launches;
+  }
   return ES_OK;
 }
 
@@ -141,15 +218,12 @@ size_t decode_attention_scratch_bytes(int B, int Hq, int hd, int n_splits) {
   return (size_t)B * Hq * n_splits * (hd + 2) * sizeof(float);
 }
 
-es_status_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t s, int64_t* launches) {
+es_status_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t s, int64_t* launches, bool pdl) {
   if (p.B <= 0) return ES_OK;
   if (p.Hq % p.Hkv != 0) return fail(ES_ERR_SHAPE, "n_heads %% n_kv_heads != 0");
-  es_status_t st;
-  if (p.hd == 128) st = launch_hd<128>(p, s);
-  else if (p.hd == 64) st = launch_hd<64>(p, s);
-  else return fail(ES_ERR_SHAPE, "head_dim must be 64 or 128, got %d", p.hd);
-  if (st == ES_OK && launches) *launches += 2;
-  return st;
+  if (p.hd == 128) return launch_hd<128>(p, s, pdl, launches);
+  if (p.hd == 64) return launch_hd<64>(p, s, pdl, launches);
+  return fail(ES_ERR_SHAPE, "head_dim must be 64 or 128, got %d", p.hd);
 }
 
 }  // namespace es

@@ -1,5 +1,6 @@
 // Memory-bound helpers of the path: embedding gather, RMSNorm, greedy argmax, context counters.
 #include "es_internal.cuh"
+#include "launch.cuh"
 
 namespace es {
 
@@ -8,6 +9,8 @@ namespace {
 // x[m, :] = table[ids[m], :] widened to fp32.  One CTA per row.
 __global__ void embed_kernel(const int* __restrict__ ids, const __half* __restrict__ table,
                              float* __restrict__ x, int d, int vocab) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int m = blockIdx.x;
   int id = ids[m];
   id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);   // out-of-range ids are clamped, never dereferenced
@@ -47,6 +50,8 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const float* __res
                                                               __half* __restrict__ y, int d, float eps,
                                                               int64_t row_stride, int64_t row_offset) {
   __shared__ float red[32];
+  pdl_launch_dependents();
+  pdl_wait();
   const int r = blockIdx.x;
   const float4* src = reinterpret_cast<const float4*>(x + ((int64_t)r * row_stride + row_offset) * d);
   const int n4 = d / 4;
@@ -89,6 +94,8 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const float* __res
 __global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ logits, int* __restrict__ out, int V) {
   __shared__ float bv[8];
   __shared__ int bi[8];
+  pdl_launch_dependents();
+  pdl_wait();
   const float* row = logits + (int64_t)blockIdx.x * V;
   float best = -INFINITY;
   int idx = 0x7fffffff;
@@ -120,6 +127,8 @@ __global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ l
 
 // ctx_len[slots[b]] = add ? ctx_len[..] + value : value
 __global__ void set_ctx_kernel(int* ctx_len, const int* slots, int B, int value, int add) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < B) {
     const int s = slots[b];
@@ -130,37 +139,33 @@ __global__ void set_ctx_kernel(int* ctx_len, const int* slots, int B, int value,
 }  // namespace
 
 es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, int d, int vocab,
-                         cudaStream_t s, int64_t* launches) {
+                         cudaStream_t s, int64_t* launches, bool pdl) {
   if (M <= 0) return ES_OK;
-  embed_kernel<<<M, 128, 0, s>>>(ids, table, x, d, vocab);
+  ES_CUDA_CHECK(launch_kernel(embed_kernel, dim3(M), dim3(128), 0, s, pdl, ids, table, x, d, vocab));
   if (launches) ++*launches;
-  ES_CUDA_CHECK(cudaGetLastError());
   return ES_OK;
 }
 
 es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M, int d, float eps,
-                           int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches) {
+                           int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches, bool pdl) {
   if (M <= 0) return ES_OK;
-  rmsnorm_kernel<<<M, RMS_THREADS, 0, s>>>(x, gain, y, d, eps, row_stride, row_offset);
+  ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel, dim3(M), dim3(RMS_THREADS), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset));
   if (launches) ++*launches;
-  ES_CUDA_CHECK(cudaGetLastError());
   return ES_OK;
 }
 
-es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches) {
+es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches, bool pdl) {
   if (B <= 0) return ES_OK;
-  argmax_kernel<<<B, 256, 0, s>>>(logits, out, V);
+  ES_CUDA_CHECK(launch_kernel(argmax_kernel, dim3(B), dim3(256), 0, s, pdl, logits, out, V));
   if (launches) ++*launches;
-  ES_CUDA_CHECK(cudaGetLastError());
   return ES_OK;
 }
 
 es_status_t launch_set_ctx(int* ctx_len, const int* slots, int B, int value, int add, cudaStream_t s,
-                           int64_t* launches) {
+                           int64_t* launches, bool pdl) {
   if (B <= 0) return ES_OK;
-  set_ctx_kernel<<<(B + 63) / 64, 64, 0, s>>>(ctx_len, slots, B, value, add);
+  ES_CUDA_CHECK(launch_kernel(set_ctx_kernel, dim3((B + 63) / 64), dim3(64), 0, s, pdl, ctx_len, slots, B, value, add));
   if (launches) ++*launches;
-  ES_CUDA_CHECK(cudaGetLastError());
   return ES_OK;
 }
 

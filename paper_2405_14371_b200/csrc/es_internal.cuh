@@ -27,6 +27,15 @@ es_status_t fail(es_status_t st, const char* fmt, ...);
     if (_s != ES_OK) return _s;      \
   } while (0)
 
+// ---- tuning knobs (read once from the environment; defaults are the measured best) -----------
+struct Tunables {
+  int stream_prefetch_row_bytes;   // ES_STREAM_PREFETCH: bytes of each first row pair prefetched into L2 before the dependency wait
+  int stream_ctas_per_sm;          // ES_STREAM_CTAS: cap on resident CTAs per SM of the weight-streaming kernel (0 = occupancy limit)
+  int stream_deep;                 // ES_STREAM_DEEP: -1 auto, 0 never, 1 always use the deeper (U = 4) chunking
+  int pdl;                         // ES_PDL: programmatic dependent launch in decode steps (1) or plain stream order (0)
+};
+const Tunables& tunables();
+
 // ---- the linear layer family ----------------------------------------------------------------
 // C[m, n] = sum_k A[m, k] * W[n, k], A fp16 [M, K] row-major (row stride lda), W fp16 row-major
 // [*, K].  The N output columns are a concatenation of up to three weight matrices ("segments",
@@ -46,6 +55,12 @@ struct LinearParams {
   const TcMaps* tc_maps;   // host pointer to pre-encoded maps (rows of A >= M), or nullptr: encode per launch
   const __half* A;
   int64_t lda;
+  // optional fused RMSNorm (weight-streaming kernel, M <= 2): A = rmsnorm(norm_x rows; norm_gain)
+  int prefetch_row_bytes;  // weight-streaming kernel: L2 prefetch per first row (0 = none)
+  const float* norm_x;     // fp32 [M, K], row stride norm_ldx; nullptr = read A
+  int64_t norm_ldx;
+  const __half* norm_gain;
+  float norm_eps;
   const __half* w[3];
   int seg_rows[3];
   int M, N, K;
@@ -70,7 +85,8 @@ struct LinearParams {
 
 // Kernel families.  Each returns after enqueuing; `launches` is incremented per kernel launched.
 es_status_t launch_linear_reference(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches);
-es_status_t launch_linear_stream(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches);   // M <= 16
+es_status_t launch_linear_stream(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl = false);   // M <= 16
+bool linear_stream_can_fuse_norm(int M);
 es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word);
 bool linear_tc_supported(const LinearParams& p, int epi);
 // Encodes the tensor maps for p's operands; the A map covers a_rows rows (the buffer's capacity).
@@ -78,13 +94,15 @@ es_status_t tc_build_maps(const LinearParams& p, int epi, int64_t a_rows, TcMaps
 
 // ---- element-wise / reductions ---------------------------------------------------------------
 es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, int d, int vocab,
-                         cudaStream_t s, int64_t* launches);
+                         cudaStream_t s, int64_t* launches, bool pdl = false);
 // row r of y = rmsnorm(row (r * row_stride + row_offset) of x)
 es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M, int d, float eps,
-                           int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches);
-es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches);
+                           int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches,
+                           bool pdl = false);
+es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches,
+                          bool pdl = false);
 es_status_t launch_set_ctx(int* ctx_len, const int* slots, int B, int value, int add, cudaStream_t s,
-                           int64_t* launches);
+                           int64_t* launches, bool pdl = false);
 
 // ---- attention -------------------------------------------------------------------------------
 // K/V addressing shared by both attention kernels: token t of sequence b, kv head g lives at
@@ -126,6 +144,6 @@ struct DecodeAttnParams {
 };
 size_t decode_attention_scratch_bytes(int B, int Hq, int hd, int n_splits);
 void choose_splits(int max_ctx, int P, int B, int Hkv, int* n_splits, int* pages_per_split);
-es_status_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t s, int64_t* launches);
+es_status_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t s, int64_t* launches, bool pdl = false);
 
 }  // namespace es

@@ -4,6 +4,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <map>
@@ -33,12 +34,24 @@ es_status_t fail(es_status_t st, const char* fmt, ...) {
   return st;
 }
 
+static int env_int(const char* name, int dflt) {
+  const char* v = getenv(name);
+  return (v && *v) ? atoi(v) : dflt;
+}
+
+const Tunables& tunables() {
+  static const Tunables t = {env_int("ES_STREAM_PREFETCH", 0), env_int("ES_STREAM_CTAS", 0), env_int("ES_STREAM_DEEP", -1),
+                             env_int("ES_PDL", 1)};
+  return t;
+}
+
 // How the context of a decode-attention call is cut into splits: enough CTAs to fill the machine,
 // never less than one KV page per split.
 void choose_splits(int max_ctx, int P, int B, int Hkv, int* n_splits, int* pages_per_split) {
   const int pages = (max_ctx + P - 1) / P;
   long long pps = (long long)pages * B * Hkv / (4 * 148);
-  if (pps < 1) pps = 1;
+  const int min_pps = 256 / P > 1 ? 256 / P : 1;      // at least 256 tokens per split
+  if (pps < min_pps) pps = min_pps;
   if (pps > pages) pps = pages;
   *pages_per_split = (int)pps;
   *n_splits = (pages + (int)pps - 1) / (int)pps;
@@ -164,6 +177,7 @@ struct es_shard {
   bool pending = false, pending_prefill = false;
   std::vector<ProfileEntry> prof;
   bool graphs = true;
+  bool pdl_now = false;   // the pass being enqueued uses programmatic dependent launch (decode steps)
   std::map<GraphKey, GraphEntry> graph_cache;
   // tensor maps of the prefill GEMMs, encoded once: [layer][qkv, o, gate/up, down]
   std::vector<TcMaps> tmaps;
@@ -213,7 +227,7 @@ es_status_t check_tensor(const es_tensor_t* t, int64_t rows, int64_t d, const ch
 }
 
 es_status_t dispatch_linear(es_shard* s, const LinearParams& p, int epi) {
-  if (p.M <= 16) return launch_linear_stream(p, epi, s->stream, &s->launches);
+  if (p.M <= 16) return launch_linear_stream(p, epi, s->stream, &s->launches, s->pdl_now);
   if (linear_tc_supported(p, epi)) return launch_linear_tc(p, epi, s->stream, &s->launches, s->status);
   return launch_linear_reference(p, epi, s->stream, &s->launches);
 }
@@ -302,9 +316,12 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   const int M = B * T;
   int pi = 0;
   const float* xin = s->x;
+  const bool pdl = decode && tunables().pdl != 0;
+  s->pdl_now = pdl;
+  const bool fuse_norm = M <= 16 && linear_stream_can_fuse_norm(M);
   if (s->has_emb) {
     prof_mark(s, pi, 0);
-    ES_TRY(launch_embed(ids, s->emb, s->x, M, d.d_model, d.vocab, s->stream, &s->launches));
+    ES_TRY(launch_embed(ids, s->emb, s->x, M, d.d_model, d.vocab, s->stream, &s->launches, pdl));
     prof_mark(s, pi, 1);
     ++pi;
   } else {
@@ -313,10 +330,12 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   for (int li = 0; li < s->nl; ++li, ++pi) {
     const es_layer_weights_t& w = s->lw[li];
     prof_mark(s, pi, 0);
-    ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches));
+    if (!fuse_norm)
+      ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl));
     int epi = 0;
     {
       LinearParams p = layer_linear(s, li, 0, M, T, decode, xin, &epi);
+      if (fuse_norm) { p.norm_x = xin; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.attn_norm; p.norm_eps = d.rms_eps; }
       ES_TRY(run_linear(s, p, epi));
     }
     KvView kvv{};
@@ -329,7 +348,7 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       a.q = s->q; a.out = s->ao; a.kv = kvv; a.ctx_len = s->ctx_len; a.ctx_add = 1; a.part = s->part;
       a.B = B; a.Hq = d.n_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim;
       a.n_splits = s->lay.n_splits; a.pages_per_split = s->lay.pages_per_split;
-      ES_TRY(launch_decode_attention(a, s->stream, &s->launches));
+      ES_TRY(launch_decode_attention(a, s->stream, &s->launches, pdl));
     } else {
       PrefillAttnParams a{};
       a.q = s->q; a.out = s->ao; a.kv = kvv; a.B = B; a.T = T; a.Hq = d.n_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim;
@@ -340,9 +359,11 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       ES_TRY(run_linear(s, p, epi));
     }
     xin = s->x;
-    ES_TRY(launch_rmsnorm(s->x, (const __half*)w.ffn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches));
+    if (!fuse_norm)
+      ES_TRY(launch_rmsnorm(s->x, (const __half*)w.ffn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl));
     {
       LinearParams p = layer_linear(s, li, 2, M, T, decode, xin, &epi);
+      if (fuse_norm) { p.norm_x = s->x; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.ffn_norm; p.norm_eps = d.rms_eps; }
       ES_TRY(run_linear(s, p, epi));
     }
     {
@@ -354,19 +375,26 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   if (s->has_head) {
     prof_mark(s, pi, 0);
     // last position of every sequence only
-    ES_TRY(launch_rmsnorm(s->x, s->fnorm, s->h_last, B, d.d_model, d.rms_eps, T, T - 1, s->stream, &s->launches));
+    const bool fuse_head = linear_stream_can_fuse_norm(B);
+    if (!fuse_head)
+      ES_TRY(launch_rmsnorm(s->x, s->fnorm, s->h_last, B, d.d_model, d.rms_eps, T, T - 1, s->stream, &s->launches, pdl));
     for (int b0 = 0; b0 < B; b0 += 16) {
       LinearParams p = base_params(s, (B - b0 < 16 ? B - b0 : 16), 1, decode);
       p.A = s->h_last + (size_t)b0 * d.d_model; p.lda = d.d_model; p.K = d.d_model; p.N = d.vocab;
       p.w[0] = s->lmh; p.seg_rows[0] = d.vocab;
       p.out_f32 = s->logits + (size_t)b0 * d.vocab; p.res = nullptr; p.ldo = d.vocab;
+      if (fuse_head) {
+        p.norm_x = s->x + (size_t)(T - 1) * d.d_model; p.norm_ldx = (int64_t)T * d.d_model;
+        p.norm_gain = s->fnorm; p.norm_eps = d.rms_eps;
+      }
       ES_TRY(run_linear(s, p, EPI_F32));
     }
-    ES_TRY(launch_argmax(s->logits, s->next_ids, B, d.vocab, s->stream, &s->launches));
+    ES_TRY(launch_argmax(s->logits, s->next_ids, B, d.vocab, s->stream, &s->launches, pdl));
     prof_mark(s, pi, 1);
   }
   // the slots' contexts now hold T (prefill) or one more (decode) position
-  ES_TRY(launch_set_ctx(s->ctx_len, s->slots_dev, B, decode ? 1 : T, decode ? 1 : 0, s->stream, &s->launches));
+  ES_TRY(launch_set_ctx(s->ctx_len, s->slots_dev, B, decode ? 1 : T, decode ? 1 : 0, s->stream, &s->launches, pdl));
+  s->pdl_now = false;
   return ES_OK;
 }
 

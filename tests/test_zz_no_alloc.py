@@ -49,8 +49,8 @@ def test_static_scratch_matches_caller_scratch_on_consecutive_calls():
 def test_static_scratch_rejects_oversized_calls():
     from paper_2405_14371_b200 import binding as B
     q, k, v, table, ctx, max_ctx = _case(1, 8, 8, 128, 16, [16], seed=4)
-    # 64 sequences x 64 heads over 40 single-page splits would need far more than 8 MiB of partials
-    Bn, Hq, Hkv, hd, P, pps = 64, 64, 1, 128, 16, 40
+    # 64 sequences x 64 heads over a 6400-token context cut into 10 splits would need 21 MB of partials
+    Bn, Hq, Hkv, hd, P, pps = 64, 64, 1, 128, 16, 400
     with pytest.raises(B.EsError) as e:
         B._check(B.lib.es_op_decode_attention_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), table.data_ptr(),
                                                      ctx.data_ptr(), q.data_ptr(), Bn, Hq, Hkv, hd, P, pps, P * pps, None))
