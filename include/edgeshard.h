@@ -171,10 +171,18 @@ ES_API es_status_t es_shard_device_status(es_shard_t *shard);
 
 /* Launch-by-launch timing of the linear-layer kernels (the weight-streaming and tensor-core
  * products that dominate a pass): while on, every such launch is bracketed by a CUDA event pair on
- * the shard's stream and decode steps are not replayed as graphs.  Switching it on or off clears
+ * the shard's stream (every launch of a pass, by category) and decode steps are not replayed as graphs.  Switching it on or off clears
  * the record.  es_shard_kernel_timing synchronises and reports the summed event time, the weight
  * bytes those launches had to read (N*K*2 each) and their number. */
+typedef enum {
+  ES_KT_EMBED = 0, ES_KT_RMSNORM = 1, ES_KT_QKV = 2, ES_KT_ATTENTION = 3, ES_KT_O = 4, ES_KT_GATE_UP = 5,
+  ES_KT_DOWN = 6, ES_KT_LM_HEAD = 7, ES_KT_ARGMAX = 8, ES_KT_SET_CTX = 9, ES_KT_COUNT = 10
+} es_kernel_category_t;
 ES_API es_status_t es_shard_set_kernel_timing(es_shard_t *shard, int32_t enabled);
+/* The same record split by kernel category: three arrays of ES_KT_COUNT entries (any may be NULL):
+ * summed event milliseconds, algorithmic bytes (weights for the linear kernels, rows for the
+ * element-wise ones, 0 where not modelled) and launches (an attention entry may be two kernels). */
+ES_API es_status_t es_shard_kernel_timing_detail(es_shard_t *shard, double *ms, double *bytes, int64_t *launches);
 ES_API es_status_t es_shard_kernel_timing(es_shard_t *shard, double *total_ms, double *weight_bytes,
                                           int64_t *launches);
 

@@ -22,6 +22,7 @@ STATUS_NAMES = {
     9: "ES_ERR_UNSUPPORTED",
 }
 ES_DTYPE_F16, ES_DTYPE_F32, ES_DTYPE_I32 = 0, 1, 2
+KERNEL_CATEGORIES = ("embed", "rmsnorm", "qkv", "attention", "o", "gate_up", "down", "lm_head", "argmax", "set_ctx")
 LAYER_KEYS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")
 
 
@@ -79,6 +80,7 @@ def _load() -> C.CDLL:
         "es_shard_launch_count": (C.c_int64, [vp]),
         "es_shard_set_kernel_timing": (i32, [vp, i32]),
         "es_shard_kernel_timing": (i32, [vp, P(C.c_double), P(C.c_double), P(C.c_int64)]),
+        "es_shard_kernel_timing_detail": (i32, [vp, P(C.c_double), P(C.c_double), P(C.c_int64)]),
         "es_shard_destroy": (None, [vp]),
         "es_last_error": (C.c_char_p, []),
         "es_version": (C.c_char_p, []),
@@ -100,7 +102,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ("es_shard_workspace_bytes es_shard_create es_shard_prefill es_shard_decode_step es_shard_handoff "
            "es_layer_profile es_shard_set_profiling es_shard_reset_slots es_shard_set_page_table es_shard_set_graphs "
-           "es_shard_device_status es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_destroy es_last_error es_version es_op_rmsnorm "
+           "es_shard_device_status es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_kernel_timing_detail es_shard_destroy es_last_error es_version es_op_rmsnorm "
            "es_op_linear es_op_prefill_attention es_op_decode_attention_scratch_bytes es_op_decode_attention "
            "es_op_decode_attention_static_capacity es_op_decode_attention_static").split()
 
@@ -249,6 +251,12 @@ class Shard:
         ms, by, n = C.c_double(0), C.c_double(0), C.c_int64(0)
         _check(lib.es_shard_kernel_timing(self._handle, C.byref(ms), C.byref(by), C.byref(n)))
         return {"ms": ms.value, "bytes": by.value, "launches": n.value}
+
+    def es_shard_kernel_timing_detail(self) -> dict:
+        n = len(KERNEL_CATEGORIES)
+        ms, by, cnt = (C.c_double * n)(), (C.c_double * n)(), (C.c_int64 * n)()
+        _check(lib.es_shard_kernel_timing_detail(self._handle, ms, by, cnt))
+        return {name: {"ms": ms[i], "bytes": by[i], "launches": cnt[i]} for i, name in enumerate(KERNEL_CATEGORIES)}
 
     @property
     def n_pages(self) -> int:

@@ -37,15 +37,20 @@ __device__ __forceinline__ void prefetch_l2(const void* ptr, uint32_t bytes) {
   asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ptr), "r"(bytes) : "memory");
 }
 
+// acc += w * a over 8 fp16 pairs, each product formed exactly and added in fp32 by the
+// mixed-precision FMA (fp16 x fp16 + fp32), so no conversion instructions are spent.
 __device__ __forceinline__ void fma8(float& acc, const uint4& w, const uint4& a) {
-  const __half2* wh = reinterpret_cast<const __half2*>(&w);
-  const __half2* ah = reinterpret_cast<const __half2*>(&a);
+  const uint32_t* wr = reinterpret_cast<const uint32_t*>(&w);
+  const uint32_t* ar = reinterpret_cast<const uint32_t*>(&a);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const float2 wf = __half22float2(wh[i]);
-    const float2 af = __half22float2(ah[i]);
-    acc = fmaf(wf.x, af.x, acc);
-    acc = fmaf(wf.y, af.y, acc);
+    asm("{\n.reg .b16 wl, wh, al, ah;\n"
+        "mov.b32 {wl, wh}, %1;\n"
+        "mov.b32 {al, ah}, %2;\n"
+        "fma.rn.f32.f16 %0, wl, al, %0;\n"
+        "fma.rn.f32.f16 %0, wh, ah, %0;\n}"
+        : "+f"(acc)
+        : "r"(wr[i]), "r"(ar[i]));
   }
 }
 
@@ -255,7 +260,7 @@ es_status_t launch_mb(const LinearParams& p, cudaStream_t s, bool pdl) {
   const int n_units = (EPI == EPI_SWIGLU) ? p.N : (p.N + 1) / 2;
   if (MB <= 2) {
     if (a_bytes > 200 * 1024) return fail(ES_ERR_SHAPE, "K = %d too large for the weight-streaming kernel", p.K);
-    bool deep = n_units < 24 * 148;             // few units per SM: keep more bytes in flight per warp
+    bool deep = true;                           // measured: 4 KB per warp per buffer beats 2 KB at every layer shape
     if (tunables().stream_deep >= 0) deep = tunables().stream_deep != 0;
     if (p.norm_x) return deep ? launch_inst<MB, EPI, true, 4, true>(p, s, pdl) : launch_inst<MB, EPI, true, 2, true>(p, s, pdl);
     return deep ? launch_inst<MB, EPI, false, 4, true>(p, s, pdl) : launch_inst<MB, EPI, false, 2, true>(p, s, pdl);

@@ -25,7 +25,7 @@ constexpr int A_STAGE_BYTES = BM * BK * 2;
 
 template <int BN> struct TileCfg {
   static constexpr int B_STAGE_BYTES = BN * BK * 2;
-  static constexpr int STAGES = (BN >= 128) ? 6 : 8;
+  static constexpr int STAGES = (BN >= 256) ? 4 : (BN >= 128) ? 6 : 8;
   static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
   static constexpr size_t SMEM = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
 };
@@ -148,12 +148,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 }
 
 // ---- the kernel --------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Persistent: a CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The accumulator is double
+// buffered in TMEM, so the epilogue of one tile runs while the tensor cores work on the next.
 template <int EPI, int BN>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int* status, int m_tiles, int n_tiles) {
   using Cfg = TileCfg<BN>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr int BN_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;   // output columns per tile
+  constexpr int ACC_COLS = Cfg::TMEM_COLS;                    // TMEM columns of one accumulator buffer
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -162,23 +169,24 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
   uint64_t* bars = (uint64_t*)(b_tiles + (size_t)STAGES * Cfg::B_STAGE_BYTES);
   uint64_t* full_bar = bars;
   uint64_t* empty_bar = bars + STAGES;
-  uint64_t* acc_bar = bars + 2 * STAGES;
-  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * STAGES + 1);
+  uint64_t* acc_full = bars + 2 * STAGES;        // [2]
+  uint64_t* acc_empty = bars + 2 * STAGES + 2;   // [2]
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * STAGES + 4);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_tiles = m_tiles * n_tiles;
+  const int num_kb = (p.K + BK - 1) / BK;
 
   // tile order: groups of up to 16 row tiles share each column tile while it is hot in L2
-  constexpr int GM = 16;
-  const int tile = blockIdx.x;
-  const int per_group = GM * n_tiles;
-  const int first_m = (tile / per_group) * GM;
-  const int gsz = min(GM, m_tiles - first_m);
-  const int mt = first_m + (tile % per_group) % gsz;
-  const int nt = (tile % per_group) / gsz;
-  const int m0 = mt * BM;
-  const int n0 = nt * BN_OUT;
-  const int num_kb = (p.K + BK - 1) / BK;
+  auto tile_origin = [&](int tile, int& m0, int& n0) {
+    constexpr int GM = 16;
+    const int per_group = GM * n_tiles;
+    const int first_m = (tile / per_group) * GM;
+    const int gsz = min(GM, m_tiles - first_m);
+    m0 = (first_m + (tile % per_group) % gsz) * BM;
+    n0 = ((tile % per_group) / gsz) * BN_OUT;
+  };
 
   if (threadIdx.x == 0) {
     prefetch_tmap(&maps.a);
@@ -187,11 +195,14 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
-    mbar_init(smem_u32(acc_bar), 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&acc_full[b]), 1);
+      mbar_init(smem_u32(&acc_empty[b]), 4);     // one arrival per epilogue warp
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), Cfg::TMEM_COLS);
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 2 * ACC_COLS);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -203,81 +214,104 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
       // the B stage is BN rows of W, fetched 32 rows per copy; with SwiGLU the first half of the
       // rows comes from the gate matrix and the second half from the up matrix (same row range)
       constexpr int N_LOADS = BN / W_BOX_ROWS;
-      const CUtensorMap* wmap[N_LOADS];
-      int wrow[N_LOADS];
-      if (EPI == EPI_SWIGLU) {
+      int it = 0;                                  // k-block counter across tiles
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        int m0, n0;
+        tile_origin(tile, m0, n0);
+        const CUtensorMap* wmap[N_LOADS];
+        int wrow[N_LOADS];
+        if (EPI == EPI_SWIGLU) {
 #pragma unroll
-        for (int i = 0; i < N_LOADS; ++i) {
-          const bool up = i >= N_LOADS / 2;
-          wmap[i] = up ? &maps.w[1] : &maps.w[0];
-          wrow[i] = n0 + (up ? i - N_LOADS / 2 : i) * W_BOX_ROWS;
+          for (int i = 0; i < N_LOADS; ++i) {
+            const bool up = i >= N_LOADS / 2;
+            wmap[i] = up ? &maps.w[1] : &maps.w[0];
+            wrow[i] = n0 + (up ? i - N_LOADS / 2 : i) * W_BOX_ROWS;
+          }
+        } else {
+          int n = n0, seg = 0;
+          while (seg < 2 && n >= p.seg_rows[seg]) { n -= p.seg_rows[seg]; ++seg; }
+#pragma unroll
+          for (int i = 0; i < N_LOADS; ++i) { wmap[i] = &maps.w[seg]; wrow[i] = n + i * W_BOX_ROWS; }
         }
-      } else {
-        int n = n0, seg = 0;
-        while (seg < 2 && n >= p.seg_rows[seg]) { n -= p.seg_rows[seg]; ++seg; }
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, abort_flag, status, 1)) { ok = false; break; }
+          const uint32_t fb = smem_u32(&full_bar[s]);
+          mbar_expect_tx(fb, A_STAGE_BYTES + Cfg::B_STAGE_BYTES);
+          tma_load_2d(smem_u32(a_tiles + (size_t)s * A_STAGE_BYTES), &maps.a, kb * BK, m0, fb);
+          const uint32_t bdst = smem_u32(b_tiles + (size_t)s * Cfg::B_STAGE_BYTES);
 #pragma unroll
-        for (int i = 0; i < N_LOADS; ++i) { wmap[i] = &maps.w[seg]; wrow[i] = n + i * W_BOX_ROWS; }
-      }
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, abort_flag, status, 1)) break;
-        const uint32_t fb = smem_u32(&full_bar[s]);
-        mbar_expect_tx(fb, A_STAGE_BYTES + Cfg::B_STAGE_BYTES);
-        tma_load_2d(smem_u32(a_tiles + (size_t)s * A_STAGE_BYTES), &maps.a, kb * BK, m0, fb);
-        const uint32_t bdst = smem_u32(b_tiles + (size_t)s * Cfg::B_STAGE_BYTES);
-#pragma unroll
-        for (int i = 0; i < N_LOADS; ++i)
-          tma_load_2d(bdst + i * W_BOX_ROWS * (BK * 2), wmap[i], kb * BK, wrow[i], fb);
+          for (int i = 0; i < N_LOADS; ++i)
+            tma_load_2d(bdst + i * W_BOX_ROWS * (BK * 2), wmap[i], kb * BK, wrow[i], fb);
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       // ---- MMA issuer ----
       constexpr uint32_t idesc = umma_idesc_f16(BM, BN);
+      int it = 0, local = 0;
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        ok = mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag, status, 2);
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++local) {
+        const int buf = local & 1;
+        const uint32_t use = (uint32_t)(local >> 1);
+        ok = mbar_wait(smem_u32(&acc_empty[buf]), (use & 1) ^ 1, abort_flag, status, 5);   // epilogue drained it
         if (!ok) break;
         tc_fence_after();
-        const uint32_t a0 = smem_u32(a_tiles + (size_t)s * A_STAGE_BYTES);
-        const uint32_t b0 = smem_u32(b_tiles + (size_t)s * Cfg::B_STAGE_BYTES);
+        const uint32_t tacc = tmem_base + (uint32_t)(buf * ACC_COLS);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          ok = mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag, status, 2);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a0 = smem_u32(a_tiles + (size_t)s * A_STAGE_BYTES);
+          const uint32_t b0 = smem_u32(b_tiles + (size_t)s * Cfg::B_STAGE_BYTES);
 #pragma unroll
-        for (int k = 0; k < BK / UMMA_K; ++k)
-          umma_f16(tmem_base, umma_desc_sw128(a0 + k * UMMA_K * 2), umma_desc_sw128(b0 + k * UMMA_K * 2), idesc,
-                   (kb > 0 || k > 0) ? 1u : 0u);
-        umma_commit(smem_u32(&empty_bar[s]));      // frees the stage once these MMAs have read it
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            umma_f16(tacc, umma_desc_sw128(a0 + k * UMMA_K * 2), umma_desc_sw128(b0 + k * UMMA_K * 2), idesc,
+                     (kb > 0 || k > 0) ? 1u : 0u);
+          umma_commit(smem_u32(&empty_bar[s]));      // frees the stage once these MMAs have read it
+        }
+        if (ok) umma_commit(smem_u32(&acc_full[buf]));   // accumulator complete
       }
-      if (ok) umma_commit(smem_u32(acc_bar));      // accumulator complete
     }
   } else {
     // ---- epilogue warps: TMEM lane quarter = warp % 4 ----
     const int quarter = warp & 3;
-    const bool ok = mbar_wait(smem_u32(acc_bar), 0, abort_flag, status, 3);
-    tc_fence_after();
-    if (ok) {
+    int local = 0;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++local) {
+      const int buf = local & 1;
+      const uint32_t use = (uint32_t)(local >> 1);
+      if (!mbar_wait(smem_u32(&acc_full[buf]), use & 1, abort_flag, status, 3)) break;
+      tc_fence_after();
+      int m0, n0;
+      tile_origin(tile, m0, n0);
       const int m = m0 + quarter * 32 + lane;
-      const uint32_t trow = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      const uint32_t trow = tmem_base + (uint32_t)(buf * ACC_COLS) + ((uint32_t)(quarter * 32) << 16);
       if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
         for (int c = 0; c < BN_OUT; c += 32) {
           float g[32], u[32];
           tmem_ld32(trow + c, g);
           tmem_ld32(trow + BN_OUT + c, u);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) epi_swiglu(p, m, n0 + c + j, g[j], u[j]);
+          epi_swiglu_chunk32(p, m, n0 + c, g, u);
         }
       } else {
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
           float v[32];
           tmem_ld32(trow + c, v);
-#pragma unroll
-          for (int j = 0; j < 32; j += 2) epi_pair<EPI>(p, m, n0 + c + j, v[j], v[j + 1]);
+          if (EPI == EPI_F32) epi_f32_chunk32(p, m, n0 + c, v);
+          else epi_qkv_chunk32(p, m, n0 + c, v);
         }
       }
+      // this warp has read its quarter of the buffer: hand it back to the MMA issuer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
     }
   }
 
@@ -287,7 +321,7 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
   if (warp == 1) {
     tc_fence_after();
     if (*abort_flag) __nanosleep(100000);     // let copies still in flight land before the CTA's memory is released
-    tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    tmem_dealloc(tmem_base, 2 * ACC_COLS);
   }
 }
 
@@ -326,20 +360,23 @@ es_status_t encode_2d(CUtensorMap* map, const void* base, int64_t rows, int64_t 
 }
 
 int pick_bn(const LinearParams& p, int epi) {
-  // widest tile that still fills the machine; segments must be whole tiles
+  // Every CTA pulls a 128-row slice of A and a bn-row slice of W through L2 for the whole K range,
+  // one CTA per SM at a time, so the time goes as (waves of CTAs) x (128 + bn).  Take the width
+  // that minimises it (the wider one on ties); QKV segments must be whole tiles.
   const int m_tiles = (p.M + BM - 1) / BM;
-  const int cands[3] = {128, 64, 32};
+  const int cands[4] = {256, 128, 64, 32};
   int best = 0;
+  long long best_cost = 0;
   for (int bn : cands) {
     const int out = (epi == EPI_SWIGLU) ? bn / 2 : bn;
     bool fits = !(epi == EPI_SWIGLU && bn < 2 * W_BOX_ROWS);
     if (epi == EPI_QKV)
       for (int s = 0; s < 3; ++s) if (p.seg_rows[s] % out) fits = false;
     if (!fits) continue;
-    if (best == 0) best = bn;
     const long long tiles = (long long)m_tiles * ((p.N + out - 1) / out);
-    if (tiles >= 148) return bn;
-    best = bn;
+    const long long waves = (tiles + 147) / 148;
+    const long long cost = waves * (BM + bn);
+    if (best == 0 || cost < best_cost) { best = bn; best_cost = cost; }
   }
   return best;
 }
@@ -354,7 +391,14 @@ es_status_t launch_bn(const TmapSet& maps, const LinearParams& p, int* status, c
     ES_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TileCfg<BN>::SMEM));
     configured = true;
   }
-  kern<<<m_tiles * n_tiles, TC_THREADS, TileCfg<BN>::SMEM, s>>>(maps, p, status, m_tiles, n_tiles);
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    ES_CUDA_CHECK(cudaGetDevice(&dev));
+    ES_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  }
+  const int tiles = m_tiles * n_tiles;
+  kern<<<tiles < sms ? tiles : sms, TC_THREADS, TileCfg<BN>::SMEM, s>>>(maps, p, status, m_tiles, n_tiles);
   ES_CUDA_CHECK(cudaGetLastError());
   return ES_OK;
 }
@@ -362,6 +406,7 @@ es_status_t launch_bn(const TmapSet& maps, const LinearParams& p, int* status, c
 template <int EPI>
 es_status_t launch_epi(const TmapSet& maps, const LinearParams& p, int bn, int* status, cudaStream_t s) {
   switch (bn) {
+    case 256: return launch_bn<EPI, 256>(maps, p, status, s);
     case 128: return launch_bn<EPI, 128>(maps, p, status, s);
     case 64: return launch_bn<EPI, 64>(maps, p, status, s);
     case 32: return launch_bn<EPI, 32>(maps, p, status, s);

@@ -185,8 +185,10 @@ struct es_shard {
   // launch-by-launch timing of the linear-layer kernels (off by default)
   bool kernel_timing = false;
   std::vector<cudaEvent_t> kt_events;   // pairs
+  std::vector<int> kt_cat;              // category of each pair
+  std::vector<double> kt_pair_bytes;    // algorithmic bytes of each pair
   size_t kt_used = 0;
-  double kt_bytes = 0;
+  int kt_next_cat = 0;
 
   __half* k_pages(int li) const { return kv + (size_t)(2 * li) * lay.n_pages * lay.page_elems; }
   __half* v_pages(int li) const { return kv + (size_t)(2 * li + 1) * lay.n_pages * lay.page_elems; }
@@ -232,8 +234,9 @@ es_status_t dispatch_linear(es_shard* s, const LinearParams& p, int epi) {
   return launch_linear_reference(p, epi, s->stream, &s->launches);
 }
 
-es_status_t run_linear(es_shard* s, const LinearParams& p, int epi) {
-  if (!s->kernel_timing) return dispatch_linear(s, p, epi);
+// Launch-by-launch timing: an event pair around one launch, tagged with a category.
+es_status_t kt_begin(es_shard* s) {
+  if (!s->kernel_timing) return ES_OK;
   if (s->kt_used + 2 > s->kt_events.size()) {
     cudaEvent_t a, b;
     ES_CUDA_CHECK(cudaEventCreate(&a));
@@ -242,11 +245,22 @@ es_status_t run_linear(es_shard* s, const LinearParams& p, int epi) {
     s->kt_events.push_back(b);
   }
   ES_CUDA_CHECK(cudaEventRecord(s->kt_events[s->kt_used], s->stream));
-  ES_TRY(dispatch_linear(s, p, epi));
+  return ES_OK;
+}
+
+es_status_t kt_end(es_shard* s, int cat, double bytes) {
+  if (!s->kernel_timing) return ES_OK;
   ES_CUDA_CHECK(cudaEventRecord(s->kt_events[s->kt_used + 1], s->stream));
   s->kt_used += 2;
-  s->kt_bytes += (double)p.N * p.K * 2.0 * (epi == EPI_SWIGLU ? 2.0 : 1.0);
+  s->kt_cat.push_back(cat);
+  s->kt_pair_bytes.push_back(bytes);
   return ES_OK;
+}
+
+es_status_t run_linear(es_shard* s, const LinearParams& p, int epi) {
+  ES_TRY(kt_begin(s));
+  ES_TRY(dispatch_linear(s, p, epi));
+  return kt_end(s, s->kt_next_cat, (double)p.N * p.K * 2.0 * (epi == EPI_SWIGLU ? 2.0 : 1.0));
 }
 
 LinearParams base_params(const es_shard* s, int M, int T, bool decode) {
@@ -321,7 +335,9 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   const bool fuse_norm = M <= 16 && linear_stream_can_fuse_norm(M);
   if (s->has_emb) {
     prof_mark(s, pi, 0);
+    ES_TRY(kt_begin(s));
     ES_TRY(launch_embed(ids, s->emb, s->x, M, d.d_model, d.vocab, s->stream, &s->launches, pdl));
+    ES_TRY(kt_end(s, ES_KT_EMBED, (double)M * d.d_model * 6.0));
     prof_mark(s, pi, 1);
     ++pi;
   } else {
@@ -330,12 +346,16 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   for (int li = 0; li < s->nl; ++li, ++pi) {
     const es_layer_weights_t& w = s->lw[li];
     prof_mark(s, pi, 0);
-    if (!fuse_norm)
+    if (!fuse_norm) {
+      ES_TRY(kt_begin(s));
       ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl));
+      ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0));
+    }
     int epi = 0;
     {
       LinearParams p = layer_linear(s, li, 0, M, T, decode, xin, &epi);
       if (fuse_norm) { p.norm_x = xin; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.attn_norm; p.norm_eps = d.rms_eps; }
+      s->kt_next_cat = ES_KT_QKV;
       ES_TRY(run_linear(s, p, epi));
     }
     KvView kvv{};
@@ -343,6 +363,7 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     kvv.block_table = s->block_table; kvv.slots = s->slots_dev;
     kvv.page_stride = (int64_t)s->lay.page_elems; kvv.head_stride = (int64_t)d.kv_page_tokens * d.head_dim;
     kvv.tok_stride = d.head_dim; kvv.P = d.kv_page_tokens; kvv.pages_per_slot = s->lay.pages_per_slot;
+    ES_TRY(kt_begin(s));
     if (decode) {
       DecodeAttnParams a{};
       a.q = s->q; a.out = s->ao; a.kv = kvv; a.ctx_len = s->ctx_len; a.ctx_add = 1; a.part = s->part;
@@ -354,20 +375,27 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       a.q = s->q; a.out = s->ao; a.kv = kvv; a.B = B; a.T = T; a.Hq = d.n_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim;
       ES_TRY(launch_prefill_attention(a, s->stream, &s->launches));
     }
+    ES_TRY(kt_end(s, ES_KT_ATTENTION, 0.0));
     {
       LinearParams p = layer_linear(s, li, 1, M, T, decode, xin, &epi);
+      s->kt_next_cat = ES_KT_O;
       ES_TRY(run_linear(s, p, epi));
     }
     xin = s->x;
-    if (!fuse_norm)
+    if (!fuse_norm) {
+      ES_TRY(kt_begin(s));
       ES_TRY(launch_rmsnorm(s->x, (const __half*)w.ffn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl));
+      ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0));
+    }
     {
       LinearParams p = layer_linear(s, li, 2, M, T, decode, xin, &epi);
       if (fuse_norm) { p.norm_x = s->x; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.ffn_norm; p.norm_eps = d.rms_eps; }
+      s->kt_next_cat = ES_KT_GATE_UP;
       ES_TRY(run_linear(s, p, epi));
     }
     {
       LinearParams p = layer_linear(s, li, 3, M, T, decode, xin, &epi);
+      s->kt_next_cat = ES_KT_DOWN;
       ES_TRY(run_linear(s, p, epi));
     }
     prof_mark(s, pi, 1);
@@ -376,8 +404,11 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     prof_mark(s, pi, 0);
     // last position of every sequence only
     const bool fuse_head = linear_stream_can_fuse_norm(B);
-    if (!fuse_head)
+    if (!fuse_head) {
+      ES_TRY(kt_begin(s));
       ES_TRY(launch_rmsnorm(s->x, s->fnorm, s->h_last, B, d.d_model, d.rms_eps, T, T - 1, s->stream, &s->launches, pdl));
+      ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)B * d.d_model * 6.0));
+    }
     for (int b0 = 0; b0 < B; b0 += 16) {
       LinearParams p = base_params(s, (B - b0 < 16 ? B - b0 : 16), 1, decode);
       p.A = s->h_last + (size_t)b0 * d.d_model; p.lda = d.d_model; p.K = d.d_model; p.N = d.vocab;
@@ -387,13 +418,18 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
         p.norm_x = s->x + (size_t)(T - 1) * d.d_model; p.norm_ldx = (int64_t)T * d.d_model;
         p.norm_gain = s->fnorm; p.norm_eps = d.rms_eps;
       }
+      s->kt_next_cat = ES_KT_LM_HEAD;
       ES_TRY(run_linear(s, p, EPI_F32));
     }
+    ES_TRY(kt_begin(s));
     ES_TRY(launch_argmax(s->logits, s->next_ids, B, d.vocab, s->stream, &s->launches, pdl));
+    ES_TRY(kt_end(s, ES_KT_ARGMAX, (double)B * d.vocab * 4.0));
     prof_mark(s, pi, 1);
   }
   // the slots' contexts now hold T (prefill) or one more (decode) position
+  ES_TRY(kt_begin(s));
   ES_TRY(launch_set_ctx(s->ctx_len, s->slots_dev, B, decode ? 1 : T, decode ? 1 : 0, s->stream, &s->launches, pdl));
+  ES_TRY(kt_end(s, ES_KT_SET_CTX, 0.0));
   s->pdl_now = false;
   return ES_OK;
 }
@@ -741,24 +777,49 @@ es_status_t es_shard_set_kernel_timing(es_shard_t* s, int32_t enabled) {
   if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
   s->kernel_timing = enabled != 0;
   s->kt_used = 0;
-  s->kt_bytes = 0;
+  s->kt_cat.clear();
+  s->kt_pair_bytes.clear();
+  return ES_OK;
+}
+
+es_status_t es_shard_kernel_timing_detail(es_shard_t* s, double* ms, double* bytes, int64_t* launches) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  ES_CUDA_CHECK(cudaStreamSynchronize(s->stream));
+  double m[ES_KT_COUNT] = {}, b[ES_KT_COUNT] = {};
+  int64_t n[ES_KT_COUNT] = {};
+  for (size_t i = 0; i + 1 < s->kt_used; i += 2) {
+    float t = 0.f;
+    ES_CUDA_CHECK(cudaEventElapsedTime(&t, s->kt_events[i], s->kt_events[i + 1]));
+    const int c = s->kt_cat[i / 2];
+    m[c] += t;
+    b[c] += s->kt_pair_bytes[i / 2];
+    n[c] += 1;
+  }
+  for (int c = 0; c < ES_KT_COUNT; ++c) {
+    if (ms) ms[c] = m[c];
+    if (bytes) bytes[c] = b[c];
+    if (launches) launches[c] = n[c];
+  }
   return ES_OK;
 }
 
 es_status_t es_shard_kernel_timing(es_shard_t* s, double* total_ms, double* weight_bytes, int64_t* launches) {
-  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
-  ES_CUDA_CHECK(cudaStreamSynchronize(s->stream));
-  double ms = 0;
-  for (size_t i = 0; i + 1 < s->kt_used; i += 2) {
-    float t = 0.f;
-    ES_CUDA_CHECK(cudaEventElapsedTime(&t, s->kt_events[i], s->kt_events[i + 1]));
-    ms += t;
-  }
-  if (total_ms) *total_ms = ms;
-  if (weight_bytes) *weight_bytes = s->kt_bytes;
-  if (launches) *launches = (int64_t)(s->kt_used / 2);
+  double m[ES_KT_COUNT], b[ES_KT_COUNT];
+  int64_t n[ES_KT_COUNT];
+  ES_TRY(es_shard_kernel_timing_detail(s, m, b, n));
+  const int lin[5] = {ES_KT_QKV, ES_KT_O, ES_KT_GATE_UP, ES_KT_DOWN, ES_KT_LM_HEAD};
+  double tm = 0, tb = 0;
+  int64_t tn = 0;
+  for (int c : lin) { tm += m[c]; tb += b[c]; tn += n[c]; }
+  if (total_ms) *total_ms = tm;
+  if (weight_bytes) *weight_bytes = tb;
+  if (launches) *launches = tn;
   return ES_OK;
 }
+
+}  // extern "C"
+
+extern "C" {
 
 // ---- single operations -----------------------------------------------------------------------
 
