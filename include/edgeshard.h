@@ -208,9 +208,10 @@ ES_API es_status_t es_op_linear(const void *A, const void *W, const float *R, fl
                          int32_t K, int32_t path, void *stream);
 
 /* Causal self-attention over a prompt.  q fp16 [B, T, Hq, hd] (already rotated); k, v fp16
- * [B, T, Hkv, hd]; out fp16 [B, T, Hq*hd].  Query t sees keys 0..t; scale 1/sqrt(hd). */
+ * [B, T, Hkv, hd]; out fp16 [B, T, Hq*hd].  Query t sees keys 0..t; scale 1/sqrt(hd).
+ * path: 0 = automatic, 1 = tensor-core (tcgen05) kernel, 2 = CUDA-core kernel. */
 ES_API es_status_t es_op_prefill_attention(const void *q, const void *k, const void *v, void *out, int32_t B,
-                                    int32_t T, int32_t Hq, int32_t Hkv, int32_t hd, void *stream);
+                                    int32_t T, int32_t Hq, int32_t Hkv, int32_t hd, int32_t path, void *stream);
 
 /* Bytes of scratch es_op_decode_attention needs. */
 ES_API size_t es_op_decode_attention_scratch_bytes(int32_t B, int32_t Hq, int32_t hd, int32_t max_ctx,

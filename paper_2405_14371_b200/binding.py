@@ -86,7 +86,7 @@ def _load() -> C.CDLL:
         "es_version": (C.c_char_p, []),
         "es_op_rmsnorm": (i32, [vp, vp, vp, i32, i32, C.c_float, vp]),
         "es_op_linear": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, vp]),
-        "es_op_prefill_attention": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp]),
+        "es_op_prefill_attention": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]),
         "es_op_decode_attention_scratch_bytes": (sz, [i32, i32, i32, i32, i32]),
         "es_op_decode_attention": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp]),
         "es_op_decode_attention_static_capacity": (sz, []),
@@ -307,11 +307,11 @@ def es_op_linear(A: torch.Tensor, W: torch.Tensor, R: Optional[torch.Tensor] = N
     return Cout
 
 
-def es_op_prefill_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, stream=None) -> torch.Tensor:
+def es_op_prefill_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, path: int = 0, stream=None) -> torch.Tensor:
     B, T, Hq, hd = q.shape
     Hkv = k.shape[2]
     out = torch.empty(B, T, Hq * hd, dtype=torch.float16, device=q.device)
-    _check(lib.es_op_prefill_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, T, Hq, Hkv, hd, _stream_ptr(stream)))
+    _check(lib.es_op_prefill_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, T, Hq, Hkv, hd, path, _stream_ptr(stream)))
     return out
 
 

@@ -1,0 +1,346 @@
+// Causal prefill attention on the tensor cores of sm_100a (tcgen05 / TMEM / TMA).
+//
+// One CTA handles 128 query rows of one (sequence, head).  Q stays resident in shared memory; K and
+// V arrive 64 keys at a time through a two-stage TMA ring (a 64-key tile is one KV page, or 64 rows
+// of a contiguous K / V matrix).  Per KV tile:
+//   S = Q K^T      tcgen05.mma, M=128 queries, N=64 keys, K=head_dim, fp32 in TMEM columns [0,64)
+//   softmax        four warps, one query row per thread (the thread holds its whole score row, so
+//                  the row maximum and sum need no cross-lane traffic): running max / sum, P in fp16
+//                  written to shared memory in the 128-byte-swizzled K-major layout
+//   O = O*a + P V  the accumulator lives in TMEM columns [64, 64+head_dim); it is rescaled in place
+//                  (tcgen05.ld / tcgen05.st) by the softmax threads before the P V MMA is issued;
+//                  V is consumed as an MN-major operand straight from its row-major tile
+// Tiles entirely above the diagonal are skipped; the diagonal tile is masked in registers.
+// Every wait is bounded; on a timeout the CTA records a code in the status word and leaves through
+// the normal teardown (TMEM freed).
+#include <string.h>
+
+#include "es_internal.cuh"
+#include "sm100.cuh"
+
+namespace es {
+
+namespace {
+
+constexpr int QT = 128;          // query rows per CTA
+constexpr int KT = 64;           // keys per tile
+constexpr int ATT_THREADS = 192;
+constexpr int TMEM_ALLOC = 256;  // S: 64 columns, O: up to 128
+
+struct AttnMaps {
+  CUtensorMap q, k, v, unused;
+};
+static_assert(sizeof(AttnMaps) == sizeof(TcMaps), "TcMaps must hold the attention maps");
+
+struct AttnArgs {
+  __half* out;               // [B, T, Hq*hd]
+  const int* block_table;    // paged mode
+  const int* slots;          // paged mode: [B] or nullptr
+  int* status;
+  int B, T, Hq, Hkv;
+  int paged, P, pages_per_slot;
+  float scale_log2e;         // log2(e) / sqrt(hd)
+};
+
+template <int HD>
+struct AttnSmem {
+  static constexpr int HALVES = HD / 64;                 // 64-column pieces of a row
+  static constexpr int Q_BYTES = QT * HD * 2;
+  static constexpr int KV_TILE_BYTES = KT * HD * 2;      // one of K / V, one stage
+  static constexpr int P_BYTES = QT * KT * 2;
+  static constexpr size_t TOTAL = 1024 + Q_BYTES + 4 * KV_TILE_BYTES + P_BYTES + 256;
+};
+
+template <int HD>
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) {
+  using L = AttnSmem<HD>;
+  constexpr int HALVES = L::HALVES;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  unsigned char* q_s = smem;                                   // [HALVES][128 rows][128 B]
+  unsigned char* k_s = q_s + L::Q_BYTES;                       // [2 stages][HALVES][64 rows][128 B]
+  unsigned char* v_s = k_s + 2 * L::KV_TILE_BYTES;
+  unsigned char* p_s = v_s + 2 * L::KV_TILE_BYTES;             // [128 rows][128 B]
+  uint64_t* bars = (uint64_t*)(p_s + L::P_BYTES);
+  uint64_t* q_full = bars;           // 1
+  uint64_t* kv_full = bars + 1;      // [2]
+  uint64_t* kv_empty = bars + 3;     // [2]
+  uint64_t* s_full = bars + 5;       // S ready in TMEM
+  uint64_t* p_full = bars + 6;       // P in smem, O rescaled (4 arrivals)
+  uint64_t* pv_done = bars + 7;      // P V accumulated
+  uint32_t* tmem_slot = (uint32_t*)(bars + 8);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q0 = blockIdx.x * QT, h = blockIdx.y, b = blockIdx.z;
+  const int g = h / (a.Hq / a.Hkv);
+  const int q_hi = min(a.T, q0 + QT);                    // one past the last query row of this tile
+  const int n_kv = (q_hi + KT - 1) / KT;                 // causal: keys 0 .. q_hi-1
+
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&maps.q);
+    prefetch_tmap(&maps.k);
+    prefetch_tmap(&maps.v);
+    mbar_init(smem_u32(q_full), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&kv_full[s]), 1);
+      mbar_init(smem_u32(&kv_empty[s]), 1);
+    }
+    mbar_init(smem_u32(s_full), 1);
+    mbar_init(smem_u32(p_full), 4);
+    mbar_init(smem_u32(pv_done), 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_ALLOC);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_s = tmem_base;            // columns [0, 64)
+  const uint32_t tmem_o = tmem_base + 64;       // columns [64, 64 + HD)
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---- TMA producer ----
+      const uint32_t qb = smem_u32(q_full);
+      mbar_expect_tx(qb, L::Q_BYTES);
+#pragma unroll
+      for (int hf = 0; hf < HALVES; ++hf)
+        tma_load_2d(smem_u32(q_s + hf * (QT * 128)), &maps.q, h * HD + hf * 64, b * a.T + q0, qb);
+      const int slot = a.paged ? (a.slots ? a.slots[b] : b) : 0;
+      for (int j = 0; j < n_kv; ++j) {
+        const int s = j & 1;
+        const uint32_t ph = (uint32_t)((j >> 1) & 1);
+        if (!mbar_wait(smem_u32(&kv_empty[s]), ph ^ 1, abort_flag, a.status, 11)) break;
+        int row, col;
+        if (a.paged) {
+          const int t0 = j * KT;
+          const int page = a.block_table[(int64_t)slot * a.pages_per_slot + t0 / a.P];
+          row = (page * a.Hkv + g) * a.P + (t0 % a.P);
+          col = 0;
+        } else {
+          row = b * a.T + j * KT;
+          col = g * HD;
+        }
+        const uint32_t fb = smem_u32(&kv_full[s]);
+        mbar_expect_tx(fb, 2 * L::KV_TILE_BYTES);
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf) {
+          tma_load_2d(smem_u32(k_s + s * L::KV_TILE_BYTES + hf * (KT * 128)), &maps.k, col + hf * 64, row, fb);
+          tma_load_2d(smem_u32(v_s + s * L::KV_TILE_BYTES + hf * (KT * 128)), &maps.v, col + hf * 64, row, fb);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ---- MMA issuer ----
+      constexpr uint32_t idesc_s = umma_idesc_f16(QT, KT);                      // Q, K both K-major
+      constexpr uint32_t idesc_o = umma_idesc_f16(QT, HD) | (1u << 16);          // V is MN-major
+      bool ok = mbar_wait(smem_u32(q_full), 0, abort_flag, a.status, 12);
+      for (int j = 0; j < n_kv && ok; ++j) {
+        const int s = j & 1;
+        ok = mbar_wait(smem_u32(&kv_full[s]), (uint32_t)((j >> 1) & 1), abort_flag, a.status, 13);
+        if (!ok) break;
+        tc_fence_after();
+        // S = Q K^T (the previous tile's softmax has finished with S: its P V MMA was issued after p_full)
+        const uint32_t kb = smem_u32(k_s + s * L::KV_TILE_BYTES);
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) {
+          const int hf = k / 4, kk = k % 4;
+          umma_f16(tmem_s, umma_desc_sw128(smem_u32(q_s + hf * (QT * 128)) + kk * 32),
+                   umma_desc_sw128(kb + hf * (KT * 128) + kk * 32), idesc_s, k > 0 ? 1u : 0u);
+        }
+        umma_commit(smem_u32(s_full));
+        // O += P V once the softmax threads have written P and rescaled O
+        ok = mbar_wait(smem_u32(p_full), (uint32_t)(j & 1), abort_flag, a.status, 14);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t vb = smem_u32(v_s + s * L::KV_TILE_BYTES);
+#pragma unroll
+        for (int k = 0; k < KT / 16; ++k)
+          umma_f16(tmem_o, umma_desc_sw128(smem_u32(p_s) + k * 32),
+                   umma_desc_sw128_mn(vb + k * (16 * 128), KT * 128, 1024), idesc_o, (j > 0 || k > 0) ? 1u : 0u);
+        umma_commit(smem_u32(&kv_empty[s]));
+        umma_commit(smem_u32(pv_done));
+      }
+    }
+  } else {
+    // ---- softmax / epilogue warps: thread = query row, TMEM lane quarter = warp % 4 ----
+    const int quarter = warp & 3;
+    const int r = quarter * 32 + lane;                 // row inside the tile
+    const int qi = q0 + r;                             // absolute query position
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    float m_run = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_kv; ++j) {
+      ok = mbar_wait(smem_u32(s_full), (uint32_t)(j & 1), abort_flag, a.status, 15);
+      if (!ok) break;
+      tc_fence_after();
+      float sc[KT];
+      {
+        float t0[32], t1[32];
+        tmem_ld32(tmem_s + lane_off, t0);
+        tmem_ld32(tmem_s + lane_off + 32, t1);
+#pragma unroll
+        for (int c = 0; c < 32; ++c) { sc[c] = t0[c]; sc[32 + c] = t1[c]; }
+      }
+      const int k0 = j * KT;
+      float mx = -INFINITY;
+      const bool diag = (k0 + KT - 1 > qi);            // some keys of this tile lie after the query
+#pragma unroll
+      for (int c = 0; c < KT; ++c) {
+        float v = sc[c] * a.scale_log2e;
+        if (diag && (k0 + c > qi)) v = -INFINITY;
+        sc[c] = v;
+        mx = fmaxf(mx, v);
+      }
+      const float m_new = fmaxf(m_run, mx);
+      const float m_use = (m_new == -INFINITY) ? 0.f : m_new;      // a fully masked row (only rows past T) stays at 0
+      const float alpha = exp2f(m_run - m_use);                     // m_run = -inf on the first tile -> 0
+      float psum = 0.f;
+      uint32_t packed[KT / 2];
+#pragma unroll
+      for (int c = 0; c < KT; c += 2) {
+        const float p0 = exp2f(sc[c] - m_use), p1 = exp2f(sc[c + 1] - m_use);
+        const __half2 hh = __floats2half2_rn(p0, p1);
+        // the sum uses the rounded probabilities, the same values the tensor cores multiply with V
+        const float2 back = __half22float2(hh);
+        psum += back.x + back.y;
+        packed[c / 2] = *reinterpret_cast<const uint32_t*>(&hh);
+      }
+      l_run = l_run * alpha + psum;
+      m_run = m_new;
+      // P row -> shared memory, 16-byte pieces at their swizzled places
+      unsigned char* prow = p_s + r * 128;
+#pragma unroll
+      for (int c8 = 0; c8 < 8; ++c8) {
+        const uint4 val = make_uint4(packed[4 * c8], packed[4 * c8 + 1], packed[4 * c8 + 2], packed[4 * c8 + 3]);
+        *reinterpret_cast<uint4*>(prow + ((c8 ^ (r & 7)) << 4)) = val;
+      }
+      // rescale the accumulator row (not before the previous P V has landed)
+      if (j > 0) {
+        ok = mbar_wait(smem_u32(pv_done), (uint32_t)((j - 1) & 1), abort_flag, a.status, 16);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll 1
+        for (int c = 0; c < HD; c += 32) {
+          float o[32];
+          tmem_ld32(tmem_o + lane_off + c, o);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] *= alpha;
+          tmem_st32(tmem_o + lane_off + c, o);
+        }
+      }
+      fence_proxy_async_smem();      // P (generic stores) must be visible to the tensor cores' reads
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(p_full));
+    }
+    if (ok) ok = mbar_wait(smem_u32(pv_done), (uint32_t)((n_kv - 1) & 1), abort_flag, a.status, 17);
+    if (ok) {
+      tc_fence_after();
+      const float inv = (l_run > 0.f) ? 1.0f / l_run : 0.f;
+      __half* orow = a.out + ((int64_t)b * a.T + qi) * ((int64_t)a.Hq * HD) + (int64_t)h * HD;
+#pragma unroll 1
+      for (int c = 0; c < HD; c += 32) {
+        float o[32];
+        tmem_ld32(tmem_o + lane_off + c, o);
+        if (qi < a.T) {
+#pragma unroll
+          for (int q8 = 0; q8 < 4; ++q8) {
+            uint4 val;
+            __half2 h0 = __floats2half2_rn(o[8 * q8] * inv, o[8 * q8 + 1] * inv);
+            __half2 h1 = __floats2half2_rn(o[8 * q8 + 2] * inv, o[8 * q8 + 3] * inv);
+            __half2 h2 = __floats2half2_rn(o[8 * q8 + 4] * inv, o[8 * q8 + 5] * inv);
+            __half2 h3 = __floats2half2_rn(o[8 * q8 + 6] * inv, o[8 * q8 + 7] * inv);
+            val.x = *reinterpret_cast<uint32_t*>(&h0); val.y = *reinterpret_cast<uint32_t*>(&h1);
+            val.z = *reinterpret_cast<uint32_t*>(&h2); val.w = *reinterpret_cast<uint32_t*>(&h3);
+            *reinterpret_cast<uint4*>(orow + c + 8 * q8) = val;
+          }
+        }
+      }
+    }
+  }
+
+  // ---- teardown ----
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    if (*abort_flag) __nanosleep(100000);
+    tmem_dealloc(tmem_base, TMEM_ALLOC);
+  }
+}
+
+bool is_paged(const PrefillAttnParams& p) { return p.kv.block_table != nullptr; }
+
+template <int HD>
+es_status_t launch_hd(const AttnMaps& maps, const PrefillAttnParams& p, cudaStream_t s) {
+  auto kern = prefill_attn_tc_kernel<HD>;
+  static bool configured = false;
+  if (!configured) {
+    ES_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttnSmem<HD>::TOTAL));
+    configured = true;
+  }
+  AttnArgs a{};
+  a.out = p.out;
+  a.block_table = p.kv.block_table;
+  a.slots = p.kv.slots;
+  a.status = p.status;
+  a.B = p.B; a.T = p.T; a.Hq = p.Hq; a.Hkv = p.Hkv;
+  a.paged = is_paged(p) ? 1 : 0;
+  a.P = p.kv.P;
+  a.pages_per_slot = p.kv.pages_per_slot;
+  a.scale_log2e = 1.4426950408889634f / sqrtf((float)HD);
+  const dim3 grid((p.T + QT - 1) / QT, p.Hq, p.B);
+  kern<<<grid, ATT_THREADS, AttnSmem<HD>::TOTAL, s>>>(maps, a);
+  ES_CUDA_CHECK(cudaGetLastError());
+  return ES_OK;
+}
+
+}  // namespace
+
+bool prefill_attention_tc_supported(const PrefillAttnParams& p) {
+  if (!tma_available()) return false;
+  if (p.hd != 64 && p.hd != 128) return false;
+  if (p.Hq % p.Hkv) return false;
+  if (((uintptr_t)p.q | (uintptr_t)p.kv.k | (uintptr_t)p.kv.v | (uintptr_t)p.out) % 16) return false;
+  if (is_paged(p)) {
+    // a 64-key tile must be one run of rows of the [pages * heads * page_tokens, head_dim] matrix
+    if (p.kv.P % KT != 0) return false;
+    if (p.kv.tok_stride != p.hd || p.kv.head_stride != (int64_t)p.kv.P * p.hd) return false;
+  } else {
+    if (p.kv.tok_stride != (int64_t)p.Hkv * p.hd || p.kv.head_stride != p.hd) return false;
+  }
+  return true;
+}
+
+es_status_t prefill_attention_tc_build_maps(const PrefillAttnParams& p, int64_t q_rows, TcMaps* out) {
+  AttnMaps* m = reinterpret_cast<AttnMaps*>(out);
+  memset(m, 0, sizeof(*m));
+  const int64_t qw = (int64_t)p.Hq * p.hd;
+  ES_TRY(tma_encode_2d_f16(&m->q, p.q, q_rows, qw, qw, QT));
+  const int64_t kw = is_paged(p) ? p.hd : (int64_t)p.Hkv * p.hd;
+  ES_TRY(tma_encode_2d_f16(&m->k, p.kv.k, p.kv_rows, kw, kw, KT));
+  ES_TRY(tma_encode_2d_f16(&m->v, p.kv.v, p.kv_rows, kw, kw, KT));
+  return ES_OK;
+}
+
+es_status_t launch_prefill_attention_tc(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches) {
+  if (p.B <= 0 || p.T <= 0) return ES_OK;
+  if (!prefill_attention_tc_supported(p)) return fail(ES_ERR_UNSUPPORTED, "tensor-core attention does not take this layout");
+  TcMaps local;
+  const TcMaps* maps = p.tc_maps;
+  if (!maps) {
+    ES_TRY(prefill_attention_tc_build_maps(p, (int64_t)p.B * p.T, &local));
+    maps = &local;
+  }
+  const AttnMaps& m = *reinterpret_cast<const AttnMaps*>(maps);
+  es_status_t st = (p.hd == 128) ? launch_hd<128>(m, p, s) : launch_hd<64>(m, p, s);
+  if (st == ES_OK && launches) ++*launches;
+  return st;
+}
+
+}  // namespace es

@@ -92,6 +92,11 @@ bool linear_tc_supported(const LinearParams& p, int epi);
 // Encodes the tensor maps for p's operands; the A map covers a_rows rows (the buffer's capacity).
 es_status_t tc_build_maps(const LinearParams& p, int epi, int64_t a_rows, TcMaps* out);
 
+// TMA tensor map (128 bytes, 64-byte aligned) of an fp16 row-major matrix [rows, cols] with row stride
+// ld elements: boxes of 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
+es_status_t tma_encode_2d_f16(void* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows);
+bool tma_available();
+
 // ---- element-wise / reductions ---------------------------------------------------------------
 es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, int d, int vocab,
                          cudaStream_t s, int64_t* launches, bool pdl = false);
@@ -129,8 +134,16 @@ struct PrefillAttnParams {
   __half* out;       // [B, T, Hq*hd]
   KvView kv;
   int B, T, Hq, Hkv, hd;
+  int64_t kv_rows;          // rows of the K / V matrices as 2-D [rows, row width] views (tensor-core kernel)
+  const TcMaps* tc_maps;    // pre-encoded maps {q, k, v} or nullptr: encode per launch
+  int* status;
 };
-es_status_t launch_prefill_attention(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches);
+// path: 0 = automatic, 1 = tensor-core (tcgen05) kernel, 2 = CUDA-core kernel
+es_status_t launch_prefill_attention(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches, int path = 0);
+es_status_t launch_prefill_attention_simt(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches);
+bool prefill_attention_tc_supported(const PrefillAttnParams& p);
+es_status_t prefill_attention_tc_build_maps(const PrefillAttnParams& p, int64_t q_rows, TcMaps* out);
+es_status_t launch_prefill_attention_tc(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches);
 
 struct DecodeAttnParams {
   const __half* q;   // [B, Hq, hd]

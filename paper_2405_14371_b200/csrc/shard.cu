@@ -182,6 +182,8 @@ struct es_shard {
   // tensor maps of the prefill GEMMs, encoded once: [layer][qkv, o, gate/up, down]
   std::vector<TcMaps> tmaps;
   bool tmaps_valid = false;
+  std::vector<TcMaps> attn_maps;        // per layer {q, k pages, v pages}
+  bool attn_maps_valid = false;
   // launch-by-launch timing of the linear-layer kernels (off by default)
   bool kernel_timing = false;
   std::vector<cudaEvent_t> kt_events;   // pairs
@@ -373,6 +375,9 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     } else {
       PrefillAttnParams a{};
       a.q = s->q; a.out = s->ao; a.kv = kvv; a.B = B; a.T = T; a.Hq = d.n_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim;
+      a.kv_rows = (int64_t)s->lay.n_pages * d.n_kv_heads * d.kv_page_tokens;
+      a.status = s->status;
+      a.tc_maps = s->attn_maps_valid ? &s->attn_maps[li] : nullptr;
       ES_TRY(launch_prefill_attention(a, s->stream, &s->launches));
     }
     ES_TRY(kt_end(s, ES_KT_ATTENTION, 0.0));
@@ -568,6 +573,22 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
         ok = linear_tc_supported(p, epi) && tc_build_maps(p, epi, desc->max_tokens, &s->tmaps[(size_t)li * 4 + kind]) == ES_OK;
       }
     s->tmaps_valid = ok;
+  }
+  // tensor maps of the prefill attention (q buffer and this layer's K / V pages)
+  {
+    s->attn_maps.resize(nl);
+    bool ok = true;
+    for (int li = 0; li < nl && ok; ++li) {
+      PrefillAttnParams a{};
+      a.q = s->q; a.out = s->ao; a.B = 1; a.T = 1; a.Hq = desc->n_heads; a.Hkv = desc->n_kv_heads; a.hd = desc->head_dim;
+      a.kv.k = s->k_pages(li); a.kv.v = s->v_pages(li); a.kv.block_table = s->block_table; a.kv.slots = s->slots_dev;
+      a.kv.page_stride = (int64_t)L.page_elems; a.kv.head_stride = (int64_t)desc->kv_page_tokens * desc->head_dim;
+      a.kv.tok_stride = desc->head_dim; a.kv.P = desc->kv_page_tokens; a.kv.pages_per_slot = L.pages_per_slot;
+      a.kv_rows = (int64_t)L.n_pages * desc->n_kv_heads * desc->kv_page_tokens;
+      ok = prefill_attention_tc_supported(a) &&
+           prefill_attention_tc_build_maps(a, desc->max_tokens, &s->attn_maps[li]) == ES_OK;
+    }
+    s->attn_maps_valid = ok;
   }
   // profile entries: [embedding] layers... [head]
   auto add_entry = [&](int layer) {
@@ -850,7 +871,7 @@ es_status_t es_op_linear(const void* A, const void* W, const float* R, float* C,
 }
 
 es_status_t es_op_prefill_attention(const void* q, const void* k, const void* v, void* out, int32_t B, int32_t T,
-                                    int32_t Hq, int32_t Hkv, int32_t hd, void* stream) {
+                                    int32_t Hq, int32_t Hkv, int32_t hd, int32_t path, void* stream) {
   if (!q || !k || !v || !out) return fail(ES_ERR_INVALID_ARG, "null argument");
   if (B < 0 || T < 0 || Hq <= 0 || Hkv <= 0) return fail(ES_ERR_INVALID_ARG, "bad sizes");
   PrefillAttnParams p{};
@@ -858,7 +879,9 @@ es_status_t es_op_prefill_attention(const void* q, const void* k, const void* v,
   p.kv.k = (const __half*)k; p.kv.v = (const __half*)v; p.kv.block_table = nullptr; p.kv.slots = nullptr;
   p.kv.page_stride = (int64_t)T * Hkv * hd; p.kv.head_stride = hd; p.kv.tok_stride = (int64_t)Hkv * hd;
   p.kv.P = T > 0 ? T : 1; p.kv.pages_per_slot = 1;
-  return launch_prefill_attention(p, (cudaStream_t)stream, nullptr);
+  p.kv_rows = (int64_t)B * T;
+  if (path == 1 && !prefill_attention_tc_supported(p)) return fail(ES_ERR_UNSUPPORTED, "tensor-core attention does not take this shape");
+  return launch_prefill_attention(p, (cudaStream_t)stream, nullptr, path);
 }
 
 size_t es_op_decode_attention_scratch_bytes(int32_t B, int32_t Hq, int32_t hd, int32_t max_ctx, int32_t page_tokens) {

@@ -82,13 +82,16 @@ def test_linear_rejects_bad_shapes(B):
     assert e.value.status == 2
 
 
+@pytest.mark.parametrize("path", [1, 2])
 @pytest.mark.parametrize("Bn,T,Hq,Hkv,hd", [(1, 1, 4, 4, 64), (2, 16, 4, 4, 64), (1, 37, 4, 2, 128), (2, 130, 8, 1, 128),
-                                            (1, 200, 2, 2, 64)])
-def test_prefill_attention(B, Bn, T, Hq, Hkv, hd):
+                                            (1, 200, 2, 2, 64), (2, 64, 2, 2, 128), (1, 128, 2, 1, 128), (3, 257, 4, 4, 64),
+                                            (1, 512, 2, 2, 128)])
+def test_prefill_attention(B, path, Bn, T, Hq, Hkv, hd):
+    """path 1 = tcgen05 kernel, 2 = CUDA-core kernel; N(0,1) q, k, v give peaked softmax rows."""
     q = _randn(Bn, T, Hq, hd, seed=8)
     k = _randn(Bn, T, Hkv, hd, seed=9)
     v = _randn(Bn, T, Hkv, hd, seed=10)
-    got = B.es_op_prefill_attention(q.cuda(), k.cuda(), v.cuda())
+    got = B.es_op_prefill_attention(q.cuda(), k.cuda(), v.cuda(), path)
     for b in range(Bn):
         want = O.causal_attention_matrix(q[b].double(), k[b].double(), v[b].double()).reshape(T, Hq * hd)
         assert rel_err(got[b], want) < 2e-3
