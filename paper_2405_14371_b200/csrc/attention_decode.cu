@@ -31,14 +31,44 @@ __global__ void __launch_bounds__(DWARPS * 32) decode_attn_split_kernel(const De
 
   const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  pdl_wait();
+  // Everything up to pdl_wait() reads only state that no kernel of the current pass has written:
+  // the slot list and page map (fixed), the slot's context length (last written when the previous
+  // pass ended; the first kernel of a pass is launched with a full dependency) and the K / V rows of
+  // tokens cached by earlier passes.  The newest token's K / V and the query come from the kernel
+  // just before this one and are read after the wait.
   const int slot = p.kv.slots ? p.kv.slots[b] : b;
-  const int ctx = p.ctx_len[slot] + p.ctx_add;
+  const int ctx_old = p.ctx_len[slot];
+  const int ctx = ctx_old + p.ctx_add;
   const int tokens_per_split = p.pages_per_split * p.kv.P;
   const int t_begin = split * tokens_per_split;
-  if (t_begin >= ctx) return;
+  if (t_begin >= ctx) { pdl_wait(); return; }
   const int t_end = min(ctx, t_begin + tokens_per_split);
   const float scale = rsqrtf((float)HD);
+  constexpr bool PRELOAD = (G <= 2);            // K row of the first block kept in registers across the wait
+
+  const int t_first = t_begin + warp * 32 + lane;
+  const bool first_valid = t_first < t_end;
+  const bool first_old = first_valid && t_first < ctx_old;
+  uint32_t off16_first = 0;
+  uint4 kpre[PRELOAD ? HD / 8 : 1];
+  if (first_valid) {
+    const __half* kr = kv_addr(p.kv, p.kv.k, slot, t_first, g);
+    off16_first = (uint32_t)((kr - p.kv.k) >> 3);
+    if (first_old) {
+      if (PRELOAD) {
+#pragma unroll
+        for (int c = 0; c < (PRELOAD ? HD / 8 : 1); ++c) kpre[c] = reinterpret_cast<const uint4*>(kr)[c];
+      } else {
+#pragma unroll
+        for (int c = 0; c < HD * 2; c += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(kr) + c));
+      }
+      const char* vr = reinterpret_cast<const char*>(p.kv.v + ((int64_t)off16_first << 3));
+#pragma unroll
+      for (int c = 0; c < HD * 2; c += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(vr + c));
+    }
+  }
+
+  pdl_wait();
 
   for (int i = threadIdx.x; i < G * HD; i += DWARPS * 32) {
     const int j = i / HD, c = i - j * HD;
@@ -58,20 +88,23 @@ __global__ void __launch_bounds__(DWARPS * 32) decode_attn_split_kernel(const De
   for (int t0 = t_begin + warp * 32; t0 < t_end; t0 += DWARPS * 32) {
     const int t = t0 + lane;
     const bool valid = t < t_end;
+    const bool first = (t0 == t_begin + warp * 32);
     // offset of this lane's token row (same for K and V), in 16-byte units
     uint32_t off16 = 0;
     float s[G];
 #pragma unroll
     for (int j = 0; j < G; ++j) s[j] = 0.f;
     if (valid) {
-      const __half* kr = kv_addr(p.kv, p.kv.k, slot, t, g);
-      off16 = (uint32_t)((kr - p.kv.k) >> 3);
+      const __half* kr;
+      if (first) { off16 = off16_first; kr = p.kv.k + ((int64_t)off16 << 3); }
+      else { kr = kv_addr(p.kv, p.kv.k, slot, t, g); off16 = (uint32_t)((kr - p.kv.k) >> 3); }
       const uint4* k4 = reinterpret_cast<const uint4*>(kr);
+      const bool use_pre = PRELOAD && first && first_old;
       // all 16-byte pieces of the row are requested up front when registers allow (small groups)
       constexpr int KU = (G <= 2) ? HD / 8 : 4;
 #pragma unroll KU
       for (int c = 0; c < HD / 8; ++c) {
-        const uint4 u = k4[c];
+        const uint4 u = use_pre ? kpre[PRELOAD ? c : 0] : k4[c];
         const __half2* h2 = reinterpret_cast<const __half2*>(&u);
         float kf[8];
 #pragma unroll

@@ -122,6 +122,7 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
       }
     }
     issue(b0w0, b0w1);
+    if (total > 1) issue(b1w0, b1w1);        // both buffers on their way: HBM stays busy while activations are staged
   }
 
   pdl_wait();
@@ -217,12 +218,14 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
     }
   };
 
+  // chunks c and c+1 are in flight in buffers 0 and 1; each buffer is refilled (chunk c+2, c+3) as soon
+  // as it has been consumed
   for (int c = 0; c < total; c += 2) {
-    if (c + 1 < total) issue(b1w0, b1w1);
     consume(b0w0, b0w1);
+    if (c + 2 < total) issue(b0w0, b0w1);
     if (c + 1 < total) {
-      if (c + 2 < total) issue(b0w0, b0w1);
       consume(b1w0, b1w1);
+      if (c + 3 < total) issue(b1w0, b1w1);
     }
   }
 }

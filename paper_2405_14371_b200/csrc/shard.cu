@@ -338,7 +338,9 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   if (s->has_emb) {
     prof_mark(s, pi, 0);
     ES_TRY(kt_begin(s));
-    ES_TRY(launch_embed(ids, s->emb, s->x, M, d.d_model, d.vocab, s->stream, &s->launches, pdl));
+    // the first kernel of a pass is launched with a full dependency: everything from earlier passes
+    // has completed before any kernel of this pass begins
+    ES_TRY(launch_embed(ids, s->emb, s->x, M, d.d_model, d.vocab, s->stream, &s->launches, false));
     ES_TRY(kt_end(s, ES_KT_EMBED, (double)M * d.d_model * 6.0));
     prof_mark(s, pi, 1);
     ++pi;
@@ -348,9 +350,10 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   for (int li = 0; li < s->nl; ++li, ++pi) {
     const es_layer_weights_t& w = s->lw[li];
     prof_mark(s, pi, 0);
+    const bool pdl0 = (li == 0 && !s->has_emb) ? false : pdl;     // first kernel of the pass: full dependency
     if (!fuse_norm) {
       ES_TRY(kt_begin(s));
-      ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl));
+      ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl0));
       ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0));
     }
     int epi = 0;
@@ -358,7 +361,9 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       LinearParams p = layer_linear(s, li, 0, M, T, decode, xin, &epi);
       if (fuse_norm) { p.norm_x = xin; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.attn_norm; p.norm_eps = d.rms_eps; }
       s->kt_next_cat = ES_KT_QKV;
+      s->pdl_now = fuse_norm ? pdl0 : pdl;
       ES_TRY(run_linear(s, p, epi));
+      s->pdl_now = pdl;
     }
     KvView kvv{};
     kvv.k = s->k_pages(li); kvv.v = s->v_pages(li);
