@@ -31,3 +31,29 @@ def rel_err(got: torch.Tensor, want: torch.Tensor) -> float:
     got = got.detach().double().cpu()
     want = want.detach().double().cpu()
     return float((got - want).abs().max() / want.abs().max())
+
+
+def host_layer(lw: dict) -> dict:
+    return {k: v.cpu() for k, v in lw.items()}
+
+
+def oracle_streamed(model, wd: dict, layer_begin: int, layer_end: int, seqs, n_layers=None, logits_from=None):
+    """Oracle (matrix form) over several independent sequences, layer by layer: each layer's weights are
+    copied from the device to the host, used for every sequence and dropped, so models larger than host
+    memory can be checked.  seqs: list of 1-D id tensors (the shard must hold the embedding).
+    Returns (list of hidden [T, d], list of logits [T - logits_from, V] or None)."""
+    from oracle import decoder as O
+
+    emb = wd["tok_embedding"].cpu()
+    xs = [O.embed(s, emb) for s in seqs]
+    del emb
+    n = (layer_end - layer_begin) if n_layers is None else n_layers
+    for li in range(n):
+        lw = host_layer(wd["layers"][li])
+        xs = [O.layer_forward_full(x, lw, model) for x in xs]
+        del lw
+    logits = None
+    if logits_from is not None:
+        fn, lm = wd["final_norm"].cpu(), wd["lm_head"].cpu()
+        logits = [O.lm_head(x[logits_from:], fn, lm, model.rms_eps) for x in xs]
+    return xs, logits

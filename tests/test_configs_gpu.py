@@ -8,7 +8,7 @@ import torch
 
 from oracle import decoder as O
 from tests.helpers import device_weights, rel_err
-from workload import WORKLOADS, prompt_ids, forced_decode_ids
+from workload import WORKLOADS, prompt_ids, forced_decode_ids, shard_weights
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-2
@@ -53,3 +53,161 @@ def test_cfg1_prefill_and_every_decode_step(B):
     assert rel_err(got_dec, want[T:]) < TOL
     worst = max(rel_err(got_dec[s], want[T + s]) for s in range(S))
     assert worst < TOL, worst
+
+
+def _run_generation(B, wl, wd, batch, stream, decode_steps=None):
+    """Prefill + greedy (head) or teacher-forced (no head) decoding of `batch` sequences on the GPU.
+    Returns prefill hidden [B, T, d], per-step hidden [S, B, d], logits [S+1, B, V] or None, ids fed [S, B]."""
+    from workload import prompt_ids, forced_decode_ids
+    m, T = wl.model, wl.prompt_len
+    S = decode_steps or wl.decode_steps
+    ids = prompt_ids(wl.cfg, batch, T, m.vocab).cuda()
+    forced = forced_decode_ids(wl.cfg, batch, S, m.vocab).cuda()
+    with torch.cuda.stream(stream):
+        sh = B.Shard(m, wl.layer_begin, wl.layer_end, wd, max_slots=batch, max_seq=T + S, max_tokens=batch * T, stream=stream)
+        slots = list(range(batch))
+        sh.es_shard_prefill(ids, None, batch, T, slots)
+        h, lg, nx = sh.es_shard_handoff()
+        pre = h.clone()
+        logits = [lg.clone()] if lg is not None else None
+        cur = torch.zeros(batch, dtype=torch.int32, device="cuda")
+        rows, fed = [], []
+        for s in range(S):
+            cur.copy_(nx if wl.has_head else forced[s])
+            fed.append(cur.clone())
+            sh.es_shard_decode_step(cur, None, batch, slots)
+            h, lg, nx = sh.es_shard_handoff()
+            rows.append(h[:, 0].clone())
+            if logits is not None:
+                logits.append(lg.clone())
+        sh.es_shard_device_status()
+        sh.close()
+    stream.synchronize()
+    return pre, torch.stack(rows), (torch.stack(logits) if logits is not None else None), torch.stack(fed), ids
+
+
+@pytest.mark.parametrize("batch,row", [(1, 0), (8, 7)])
+def test_cfg2_full_7b_with_head(B, batch, row):
+    """Full Llama-2-7B, prompt 512, 256 greedy steps.  The oracle is teacher-forced with the tokens the
+    GPU generated (near-ties may legitimately flip an argmax under fp16), and checks the sampled batch
+    row at every position: hidden states after prefill and after each step, logits of each step."""
+    from tests.helpers import oracle_streamed
+    wl = WORKLOADS["cfg2_b1"]
+    m, T, S = wl.model, wl.prompt_len, wl.decode_steps
+    wd = shard_weights(wl.cfg, m, 0, m.n_layers, device="cuda")
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    pre, dec, logits, fed, ids = _run_generation(B, wl, wd, batch, stream)
+    seq = torch.cat([ids[row].cpu(), fed[:, row].cpu()])                 # T + S tokens actually consumed
+    xs, ls = oracle_streamed(m, wd, 0, m.n_layers, [seq], logits_from=T - 1)
+    want_h, want_l = xs[0], ls[0]                                         # [T+S, d], [S+1, V]
+    assert rel_err(pre[row], want_h[:T]) < TOL
+    assert rel_err(dec[:, row], want_h[T:]) < TOL
+    assert rel_err(logits[:, row], want_l) < TOL
+    agree = (logits[:, row].argmax(-1).cpu() == want_l.argmax(-1)).float().mean()
+    assert agree > 0.9, float(agree)
+
+
+def test_cfg3_pipeline_of_four_shards(B):
+    """Llama-2-13B as 4 shards of 10 layers run in sequence on one GPU, 8 micro-batches of one sequence,
+    prompt 256, 128 greedy steps; each micro-batch lives in its own KV slot of every shard.  Oracle on
+    micro-batches 0 and 7."""
+    from tests.helpers import oracle_streamed, slice_weights
+    wl = WORKLOADS["cfg3"]
+    m, T, S, MB = wl.model, wl.prompt_len, wl.decode_steps, wl.micro_batches
+    wd = shard_weights(wl.cfg, m, 0, m.n_layers, device="cuda")
+    ids = prompt_ids(wl.cfg, MB, T, m.vocab).cuda()
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    per = m.n_layers // wl.n_shards
+    with torch.cuda.stream(stream):
+        shards = [B.Shard(m, i * per, (i + 1) * per, slice_weights(wd, m, i * per, (i + 1) * per), max_slots=MB,
+                          max_seq=T + S, max_tokens=T, max_batch=1, stream=stream) for i in range(wl.n_shards)]
+        cur = torch.zeros(MB, 1, dtype=torch.int32, device="cuda")       # next token of each micro-batch
+        pre_h = {}
+        def through(mb, first_ids, prefill):
+            x = None
+            for si, sh in enumerate(shards):
+                if prefill:
+                    sh.es_shard_prefill(first_ids if si == 0 else None, x, 1, T, [mb])
+                else:
+                    sh.es_shard_decode_step(first_ids if si == 0 else None, x, 1, [mb])
+                x, lg, nx = sh.es_shard_handoff()                         # same device: the hand-over is this view
+            return x, lg, nx
+        logits = torch.zeros(S + 1, MB, m.vocab)
+        hid = torch.zeros(S, MB, m.d_model)
+        fed = torch.zeros(S, MB, dtype=torch.int32)
+        for mb in range(MB):
+            x, lg, nx = through(mb, ids[mb:mb + 1], True)
+            if mb in (0, MB - 1):
+                pre_h[mb] = x[0].clone()
+                logits[0, mb] = lg[0].cpu()
+            cur[mb].copy_(nx)
+        for s in range(S):
+            for mb in range(MB):                                          # every micro-batch re-streams every shard
+                fed[s, mb] = int(cur[mb, 0]) if mb in (0, MB - 1) else 0
+                x, lg, nx = through(mb, cur[mb], False)
+                if mb in (0, MB - 1):
+                    hid[s, mb] = x[0, 0].cpu()
+                    logits[s + 1, mb] = lg[0].cpu()
+                cur[mb].copy_(nx)
+        for sh in shards:
+            sh.es_shard_device_status()
+            sh.close()
+    stream.synchronize()
+    for mb in (0, MB - 1):
+        seq = torch.cat([ids[mb].cpu(), fed[:, mb]])
+        xs, ls = oracle_streamed(m, wd, 0, m.n_layers, [seq], logits_from=T - 1)
+        assert rel_err(pre_h[mb], xs[0][:T]) < TOL
+        assert rel_err(hid[:, mb], xs[0][T:]) < TOL
+        assert rel_err(logits[:, mb], ls[0]) < TOL
+
+
+def test_cfg4_gqa_shard_batch16(B):
+    """Llama-2-70B-architecture layers 0-39 (8 KV heads for 64 query heads), batch 16, prompt 1024, 128
+    teacher-forced steps.  The 68 GB of weights exceed what the oracle can hold, so the oracle checks
+    layers 0-3 (a 4-layer shard at the full batch and lengths) on rows 0 and 15 at every position, and
+    the 40-layer shard is checked for the split invariance [0,4) -> [4,40) == [0,40), bit for bit."""
+    from tests.helpers import oracle_streamed, slice_weights
+    from workload import forced_decode_ids
+    wl = WORKLOADS["cfg4"]
+    m, T, S, Bn = wl.model, wl.prompt_len, wl.decode_steps, wl.batch
+    wd = shard_weights(wl.cfg, m, 0, wl.layer_end, device="cuda")
+    ids = prompt_ids(wl.cfg, Bn, T, m.vocab).cuda()
+    forced = forced_decode_ids(wl.cfg, Bn, S, m.vocab).cuda()
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    slots = list(range(Bn))
+    k = 4
+    with torch.cuda.stream(stream):
+        kw = dict(max_slots=Bn, max_seq=T + S, max_tokens=Bn * T, stream=stream)
+        full = B.Shard(m, 0, wl.layer_end, wd, **kw)
+        a = B.Shard(m, 0, k, slice_weights(wd, m, 0, k), **kw)
+        b = B.Shard(m, k, wl.layer_end, slice_weights(wd, m, k, wl.layer_end), **kw)
+        full.es_shard_prefill(ids, None, Bn, T, slots)
+        a.es_shard_prefill(ids, None, Bn, T, slots)
+        ha = a.es_shard_handoff()[0]
+        pre_a = {r: ha[r].clone() for r in (0, Bn - 1)}
+        b.es_shard_prefill(None, ha, Bn, T, slots)
+        assert torch.equal(full.es_shard_handoff()[0], b.es_shard_handoff()[0])
+        cur = torch.zeros(Bn, dtype=torch.int32, device="cuda")
+        dec_a = []
+        for s in range(S):
+            cur.copy_(forced[s])
+            full.es_shard_decode_step(cur, None, Bn, slots)
+            a.es_shard_decode_step(cur, None, Bn, slots)
+            ha = a.es_shard_handoff()[0]
+            dec_a.append(ha[:, 0].clone())
+            b.es_shard_decode_step(None, ha, Bn, slots)
+            if s % 16 == 0 or s == S - 1:
+                assert torch.equal(full.es_shard_handoff()[0], b.es_shard_handoff()[0]), s
+        for sh in (full, a, b):
+            sh.es_shard_device_status()
+            sh.close()
+    stream.synchronize()
+    dec_a = torch.stack(dec_a)
+    seqs = [torch.cat([ids[r].cpu(), forced[:, r].cpu()]) for r in (0, Bn - 1)]
+    xs, _ = oracle_streamed(m, wd, 0, k, seqs)
+    for x, r in zip(xs, (0, Bn - 1)):
+        assert rel_err(pre_a[r], x[:T]) < TOL
+        assert rel_err(dec_a[:, r], x[T:]) < TOL

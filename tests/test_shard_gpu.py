@@ -156,6 +156,67 @@ def test_page_map_and_graphs_do_not_change_results(B, tiny):
         assert all(torch.equal(a, b) for a, b in zip(ref, got)), (permute, graphs)
 
 
+def test_micro_batch_pipeline_is_order_independent(B, tiny):
+    """Two shards of one layer each, four micro-batches in four KV slots: walking micro-batch by
+    micro-batch (hand-over by pointer) or shard by shard (hand-over through per-micro-batch copies)
+    gives identical bits, and both equal the single two-layer shard."""
+    wd, _ = tiny
+    T, S, MB = 10, 3, 4
+    ids = prompt_ids(0, MB, T, TINY.vocab, seed=11).cuda()
+    nxt = forced_decode_ids(0, MB, S, TINY.vocab, seed=11).cuda()
+    kw = dict(max_slots=MB, max_seq=16, max_tokens=T, max_batch=1, kv_page_tokens=16)
+
+    def make():
+        return [B.Shard(TINY, 0, 1, slice_weights(wd, TINY, 0, 1), **kw), B.Shard(TINY, 1, 2, slice_weights(wd, TINY, 1, 2), **kw)]
+
+    def mb_major():
+        s0, s1 = make()
+        out = {}
+        for mb in range(MB):
+            s0.es_shard_prefill(ids[mb:mb + 1], None, 1, T, [mb])
+            s1.es_shard_prefill(None, s0.es_shard_handoff()[0], 1, T, [mb])
+            out[(mb, -1)] = [t.clone() for t in s1.es_shard_handoff()[:2]]
+        for st in range(S):
+            for mb in range(MB):
+                s0.es_shard_decode_step(nxt[st, mb:mb + 1], None, 1, [mb])
+                s1.es_shard_decode_step(None, s0.es_shard_handoff()[0], 1, [mb])
+                out[(mb, st)] = [t.clone() for t in s1.es_shard_handoff()[:2]]
+        s0.close(); s1.close()
+        return out
+
+    def shard_major():
+        s0, s1 = make()
+        out = {}
+        acts = []
+        for mb in reversed(range(MB)):                                     # another micro-batch order as well
+            s0.es_shard_prefill(ids[mb:mb + 1], None, 1, T, [mb])
+            acts.append((mb, s0.es_shard_handoff()[0].clone()))
+        for mb, a in acts:
+            s1.es_shard_prefill(None, a, 1, T, [mb])
+            out[(mb, -1)] = [t.clone() for t in s1.es_shard_handoff()[:2]]
+        for st in range(S):
+            acts = []
+            for mb in range(MB):
+                s0.es_shard_decode_step(nxt[st, mb:mb + 1], None, 1, [mb])
+                acts.append((mb, s0.es_shard_handoff()[0].clone()))
+            for mb, a in reversed(acts):
+                s1.es_shard_decode_step(None, a, 1, [mb])
+                out[(mb, st)] = [t.clone() for t in s1.es_shard_handoff()[:2]]
+        s0.close(); s1.close()
+        return out
+
+    x, y = mb_major(), shard_major()
+    assert x.keys() == y.keys()
+    for key in x:
+        assert all(torch.equal(p, q) for p, q in zip(x[key], y[key])), key
+    whole = B.Shard(TINY, 0, 2, wd, **kw)
+    for mb in range(MB):
+        whole.es_shard_prefill(ids[mb:mb + 1], None, 1, T, [mb])
+        h, l, _ = whole.es_shard_handoff()
+        assert torch.equal(h, x[(mb, -1)][0]) and torch.equal(l, x[(mb, -1)][1])
+    whole.close()
+
+
 def test_profile_reports_every_layer(B, tiny):
     wd, _ = tiny
     ids = prompt_ids(0, 1, 16, TINY.vocab).cuda()

@@ -91,8 +91,9 @@ def standard_normal_f32(seed: int, tensor_id: int, start: int, n: int, device="c
     table = _quantile_table(str(device))
     key = stream_key(seed, tensor_id)
     out = torch.empty(n, dtype=torch.float32, device=device)
-    for o in range(0, n, _CHUNK):
-        m = min(_CHUNK, n - o)
+    chunk = _CHUNK * 8 if device.type == "cuda" else _CHUNK      # fewer, larger launches on a GPU
+    for o in range(0, n, chunk):
+        m = min(chunk, n - o)
         h = _hash_range(key, start + o, m, device)
         i = _srl(h, 48)
         f = (_srl(h, 24) & 0xFFFFFF).to(torch.float32) * (2.0 ** -24)
