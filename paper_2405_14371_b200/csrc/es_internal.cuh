@@ -87,6 +87,9 @@ struct LinearParams {
 es_status_t launch_linear_reference(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches);
 es_status_t launch_linear_stream(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl = false);   // M <= 16
 bool linear_stream_can_fuse_norm(int M);
+// tensor-core (mma.sync) variant of the weight-streaming kernel for 3..16 rows
+bool linear_stream_mma_supported(const LinearParams& p, int epi);
+es_status_t launch_linear_stream_mma(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl = false);
 es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word);
 bool linear_tc_supported(const LinearParams& p, int epi);
 // Encodes the tensor maps for p's operands; the A map covers a_rows rows (the buffer's capacity).

@@ -1,0 +1,249 @@
+// Weight-streaming kernel for decode steps with several sequences (3 <= M <= 16 activation rows).
+// Like the single-row kernel it reads every weight byte once, straight from global memory into
+// registers (16-byte loads, double buffered across work units, first chunks requested before the
+// programmatic-dependency wait), but the arithmetic runs on the tensor cores: at 8 or 16 rows the
+// plain ALUs cannot keep up with HBM.
+//
+//  * a work unit is 16 weight rows (or 8 gate rows + 8 up rows for SwiGLU).  A CTA owns a contiguous,
+//    balanced range of units; its 8 warps all work on the same unit, each on one eighth of K, and
+//    their partial sums are added in warp order through shared memory (deterministic);
+//  * per 32 K-elements a lane loads 16 bytes of row g and of row g+8 (g = lane / 4) and issues two
+//    mma.sync.m16n8k16 per group of 8 sequences.  The 8 consecutive elements a lane holds are fed to
+//    the MMAs under a fixed permutation of the K index; the activation operand is read with the
+//    same permutation (one 16-byte load per lane), so the products pair up correctly;
+//  * activations sit in shared memory when they fit, otherwise they are read through L1 / L2.
+#include "epilogue.cuh"
+#include "launch.cuh"
+
+namespace es {
+
+namespace {
+
+constexpr int MW = 8;                 // warps per CTA
+constexpr int MTHREADS = MW * 32;
+constexpr int KSTEP = 32;             // K elements per lane-load step
+constexpr int UM = 4;                 // steps per chunk
+
+__device__ __forceinline__ uint4 ld_stream16(const void* ptr) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(ptr));
+  return v;
+}
+
+__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// NT: groups of 8 activation rows (1 or 2).
+template <int NT, int EPI, bool A_SMEM>
+__global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const LinearParams p, int a_stride) {
+  pdl_launch_dependents();
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __half* a_s = reinterpret_cast<__half*>(smem_raw);                 // [NT*8][a_stride], padded rows
+  __shared__ float red[2][MW][NT][32][4];
+
+  const int K = p.K;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, q = lane & 3;
+  constexpr int COLS = (EPI == EPI_SWIGLU) ? 8 : 16;                 // output columns per unit
+  const int n_units = (p.N + COLS - 1) / COLS;
+  const int u0 = (int)((int64_t)blockIdx.x * n_units / gridDim.x);
+  const int u1 = (int)((int64_t)(blockIdx.x + 1) * n_units / gridDim.x);
+  const int n_my = u1 - u0;
+  const int kslice = K / MW;                                         // multiple of KSTEP (checked on the host)
+  const int k_lo = warp * kslice, k_hi = k_lo + kslice;
+  constexpr int CHUNK_K = KSTEP * UM;
+  const int chunks_per_unit = (kslice + CHUNK_K - 1) / CHUNK_K;
+  const int total = n_my * chunks_per_unit;
+
+  auto unit_rows = [&](int i, const __half*& r0, const __half*& r1) {
+    const int u = u0 + i;
+    if (EPI == EPI_SWIGLU) {
+      const int n = u * 8 + g;
+      r0 = (n < p.N) ? p.w[0] + (int64_t)n * K : nullptr;
+      r1 = (n < p.N) ? p.w[1] + (int64_t)n * K : nullptr;
+    } else {
+      const int n = u * 16 + g;
+      r0 = (n < p.N) ? weight_row(p, n) : nullptr;
+      r1 = (n + 8 < p.N) ? weight_row(p, n + 8) : nullptr;
+    }
+  };
+
+  int nxt_i = 0, nxt_cc = 0;
+  const __half* nr0 = nullptr;
+  const __half* nr1 = nullptr;
+  if (total > 0) unit_rows(0, nr0, nr1);
+  auto issue = [&](uint4 (&w0)[UM], uint4 (&w1)[UM]) {
+    const int kb = k_lo + nxt_cc * CHUNK_K + q * 8;
+#pragma unroll
+    for (int j = 0; j < UM; ++j) {
+      const int k = kb + j * KSTEP;
+      const bool in = k < k_hi;
+      w0[j] = (in && nr0) ? ld_stream16(nr0 + k) : make_uint4(0, 0, 0, 0);
+      w1[j] = (in && nr1) ? ld_stream16(nr1 + k) : make_uint4(0, 0, 0, 0);
+    }
+    if (++nxt_cc == chunks_per_unit) {
+      nxt_cc = 0;
+      if (++nxt_i < n_my) unit_rows(nxt_i, nr0, nr1);
+    }
+  };
+
+  uint4 b0w0[UM], b0w1[UM], b1w0[UM], b1w1[UM];
+  if (total > 0) {
+    issue(b0w0, b0w1);
+    if (total > 1) issue(b1w0, b1w1);
+  }
+
+  pdl_wait();
+
+  if (A_SMEM) {
+    const int chunks = K / 8;
+    for (int i = threadIdx.x; i < NT * 8 * chunks; i += MTHREADS) {
+      const int m = i / chunks, c = i - m * chunks;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (m < p.M) v = *reinterpret_cast<const uint4*>(p.A + (int64_t)m * p.lda + c * 8);
+      *reinterpret_cast<uint4*>(a_s + (int64_t)m * a_stride + c * 8) = v;
+    }
+    __syncthreads();
+  }
+
+  float acc[NT][4];
+#pragma unroll
+  for (int t = 0; t < NT; ++t)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[t][i] = 0.f;
+  int cur_i = 0, cur_cc = 0;
+
+  auto consume = [&](const uint4 (&w0)[UM], const uint4 (&w1)[UM]) {
+    const int kb = k_lo + cur_cc * CHUNK_K + q * 8;
+#pragma unroll
+    for (int j = 0; j < UM; ++j) {
+      const int k = kb + j * KSTEP;
+      if (k < k_hi) {
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+          const int m = t * 8 + g;
+          uint4 a;
+          if (A_SMEM) a = *reinterpret_cast<const uint4*>(a_s + (int64_t)m * a_stride + k);
+          else a = (m < p.M) ? __ldg(reinterpret_cast<const uint4*>(p.A + (int64_t)m * p.lda + k)) : make_uint4(0, 0, 0, 0);
+          mma16816(acc[t], w0[j].x, w1[j].x, w0[j].y, w1[j].y, a.x, a.y);
+          mma16816(acc[t], w0[j].z, w1[j].z, w0[j].w, w1[j].w, a.z, a.w);
+        }
+      }
+    }
+    if (++cur_cc == chunks_per_unit) {
+      // unit finished in this warp's K slice: add the 8 slices in warp order
+      const int buf = cur_i & 1;
+#pragma unroll
+      for (int t = 0; t < NT; ++t) {
+        *reinterpret_cast<float4*>(&red[buf][warp][t][lane][0]) = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[t][i] = 0.f;
+      }
+      __syncthreads();
+      // thread -> (output pair pr, activation row m).  Accumulator element (row r, column m) of group t
+      // lives in lane (r % 8) * 4 + (m % 8) / 2, register (r / 8) * 2 + (m % 2).
+      if (threadIdx.x < 8 * NT * 8) {
+        const int pr = threadIdx.x & 7, m = threadIdx.x >> 3;
+        const int t = m >> 3, mc = m & 7;
+        int ra, rb;                                  // the two accumulator rows this thread combines
+        if (EPI == EPI_SWIGLU) { ra = pr; rb = pr + 8; }
+        else { ra = 2 * pr; rb = 2 * pr + 1; }
+        const int la = (ra & 7) * 4 + (mc >> 1), ia = (ra >> 3) * 2 + (mc & 1);
+        const int lb = (rb & 7) * 4 + (mc >> 1), ib = (rb >> 3) * 2 + (mc & 1);
+        float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+        for (int w = 0; w < MW; ++w) {
+          v0 += red[buf][w][t][la][ia];
+          v1 += red[buf][w][t][lb][ib];
+        }
+        const int u = u0 + cur_i;
+        const int n = (EPI == EPI_SWIGLU) ? u * 8 + pr : u * 16 + 2 * pr;
+        epi_pair<EPI>(p, m, n, v0, v1);
+      }
+      cur_cc = 0;
+      ++cur_i;
+    }
+  };
+
+  for (int c = 0; c < total; c += 2) {
+    consume(b0w0, b0w1);
+    if (c + 2 < total) issue(b0w0, b0w1);
+    if (c + 1 < total) {
+      consume(b1w0, b1w1);
+      if (c + 3 < total) issue(b1w0, b1w1);
+    }
+  }
+}
+
+template <int NT, int EPI, bool A_SMEM>
+es_status_t launch_inst(const LinearParams& p, cudaStream_t s, bool pdl) {
+  auto kern = linear_stream_mma_kernel<NT, EPI, A_SMEM>;
+  const int a_stride = p.K + 8;                       // 16 bytes of padding: the 8 rows fall into different banks
+  const size_t smem = A_SMEM ? (size_t)NT * 8 * a_stride * sizeof(__half) : 0;
+  static size_t configured = 0;
+  if (smem > 16 * 1024 && smem > configured) {      // static shared memory counts against the 48 KB default too
+    ES_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    configured = smem;
+  }
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    ES_CUDA_CHECK(cudaGetDevice(&dev));
+    ES_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  }
+  int per_sm = 0;
+  ES_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, MTHREADS, smem));
+  if (per_sm < 1) return fail(ES_ERR_SHAPE, "tensor-core streaming kernel does not fit (K = %d)", p.K);
+  constexpr int COLS = (EPI == EPI_SWIGLU) ? 8 : 16;
+  const int n_units = (p.N + COLS - 1) / COLS;
+  int grid = sms * per_sm;
+  if (grid > n_units) grid = n_units;
+  ES_CUDA_CHECK(launch_kernel(kern, dim3(grid), dim3(MTHREADS), smem, s, pdl, p, a_stride));
+  return ES_OK;
+}
+
+template <int NT, int EPI>
+es_status_t launch_nt(const LinearParams& p, cudaStream_t s, bool pdl) {
+  const size_t a_bytes = (size_t)NT * 8 * (p.K + 8) * sizeof(__half);
+  if (a_bytes <= 100 * 1024) return launch_inst<NT, EPI, true>(p, s, pdl);
+  return launch_inst<NT, EPI, false>(p, s, pdl);
+}
+
+template <int EPI>
+es_status_t launch_epi(const LinearParams& p, cudaStream_t s, bool pdl) {
+  if (p.M <= 8) return launch_nt<1, EPI>(p, s, pdl);
+  return launch_nt<2, EPI>(p, s, pdl);
+}
+
+}  // namespace
+
+bool linear_stream_mma_supported(const LinearParams& p, int epi) {
+  if (p.M < 1 || p.M > 16 || p.N <= 0 || p.norm_x != nullptr) return false;
+  if (p.K % (MW * KSTEP) != 0) return false;            // every warp gets a whole number of 32-element steps
+  if (p.lda % 8 != 0 || ((uintptr_t)p.A % 16)) return false;
+  for (int i = 0; i < 3; ++i)
+    if (p.w[i] && ((uintptr_t)p.w[i] % 16)) return false;
+  if (epi == EPI_QKV && (p.N % 2)) return false;
+  return true;
+}
+
+es_status_t launch_linear_stream_mma(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl) {
+  if (!linear_stream_mma_supported(p, epi)) return fail(ES_ERR_UNSUPPORTED, "tensor-core streaming kernel does not take this shape");
+  es_status_t st;
+  switch (epi) {
+    case EPI_F32: st = launch_epi<EPI_F32>(p, s, pdl); break;
+    case EPI_SWIGLU: st = launch_epi<EPI_SWIGLU>(p, s, pdl); break;
+    case EPI_QKV: st = launch_epi<EPI_QKV>(p, s, pdl); break;
+    default: return fail(ES_ERR_INVALID_ARG, "unknown epilogue %d", epi);
+  }
+  if (st == ES_OK && launches) ++*launches;
+  return st;
+}
+
+}  // namespace es

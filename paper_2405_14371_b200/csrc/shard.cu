@@ -231,6 +231,8 @@ es_status_t check_tensor(const es_tensor_t* t, int64_t rows, int64_t d, const ch
 }
 
 es_status_t dispatch_linear(es_shard* s, const LinearParams& p, int epi) {
+  if (p.M > 2 && p.M <= 16 && linear_stream_mma_supported(p, epi))
+    return launch_linear_stream_mma(p, epi, s->stream, &s->launches, s->pdl_now);
   if (p.M <= 16) return launch_linear_stream(p, epi, s->stream, &s->launches, s->pdl_now);
   if (linear_tc_supported(p, epi)) return launch_linear_tc(p, epi, s->stream, &s->launches, s->status);
   return launch_linear_reference(p, epi, s->stream, &s->launches);
@@ -864,13 +866,16 @@ es_status_t es_op_linear(const void* A, const void* W, const float* R, float* C,
   p.A = (const __half*)A; p.lda = K; p.w[0] = (const __half*)W; p.seg_rows[0] = N;
   p.M = M; p.N = N; p.K = K; p.out_f32 = C; p.res = R; p.ldo = N; p.T = 1;
   cudaStream_t st = (cudaStream_t)stream;
-  if (path == 0) path = (M <= 16) ? 2 : (linear_tc_supported(p, EPI_F32) ? 1 : 3);
+  if (path == 0) path = (M > 2 && M <= 16 && linear_stream_mma_supported(p, EPI_F32)) ? 4 : (M <= 16) ? 2 : (linear_tc_supported(p, EPI_F32) ? 1 : 3);
   switch (path) {
     case 1:
       if (!linear_tc_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "tensor-core kernel does not take this shape");
       return launch_linear_tc(p, EPI_F32, st, nullptr, nullptr);
     case 2: return launch_linear_stream(p, EPI_F32, st, nullptr);
     case 3: return launch_linear_reference(p, EPI_F32, st, nullptr);
+    case 4:
+      if (!linear_stream_mma_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "tensor-core streaming kernel does not take this shape");
+      return launch_linear_stream_mma(p, EPI_F32, st, nullptr);
     default: return fail(ES_ERR_INVALID_ARG, "unknown path %d", path);
   }
 }

@@ -71,6 +71,19 @@ def test_linear_tensor_core(B, M, N, K):
     assert rel_err(got_r, ref) < 5e-5   # fp32 tensor-core accumulation over K up to 11008
 
 
+@pytest.mark.parametrize("M,N,K", [(3, 64, 256), (8, 4096, 4096), (8, 1000, 512), (13, 136, 1024), (16, 8192, 8192),
+                                   (16, 24, 28672), (5, 11008, 4096), (16, 4096, 11008)])
+def test_linear_streaming_tensor_core(B, M, N, K):
+    """mma.sync weight-streaming kernel (decode with several sequences): ragged N, long K, 1 and 2 row groups."""
+    A = _randn(M, K, seed=16)
+    W = _randn(N, K, seed=17, scale=0.05)
+    R = _randn(M, N, seed=18, dtype=torch.float32)
+    want = A.double() @ W.double().T
+    got = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), 4)
+    assert rel_err(got, want + R.double()) < 5e-5
+    assert rel_err(B.es_op_linear(A.cuda(), W.cuda(), None, 4), want) < 5e-5
+
+
 def test_linear_rejects_bad_shapes(B):
     A = _randn(17, 64).cuda()
     W = _randn(32, 64).cuda()
