@@ -161,43 +161,76 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     stream = torch.cuda.Stream(device=dev)
     weights = shard_weights(wl.cfg, m, wl.layer_begin, wl.layer_end, device=dev)
-    ids_host = prompt_ids(wl.cfg, Bn, T, m.vocab).pin_memory()
-    forced_host = forced_decode_ids(wl.cfg, Bn, S, m.vocab).pin_memory()
+    # a workload may run its layer range as several shards in sequence, with micro-batches of Bn
+    # sequences each living in their own KV slots of every shard (the pipeline of config 3)
+    n_sh, MB = wl.n_shards, wl.micro_batches
+    per = (wl.layer_end - wl.layer_begin) // n_sh
+    ids_host = prompt_ids(wl.cfg, MB * Bn, T, m.vocab).reshape(MB, Bn, T).pin_memory()
+    forced_host = forced_decode_ids(wl.cfg, MB * Bn, S, m.vocab).reshape(S, MB, Bn).pin_memory()
     ids_dev = ids_host.to(dev)
     forced_dev = forced_host.to(dev)
-    cur_ids = torch.zeros(Bn, dtype=torch.int32, device=dev)
-    slots = list(range(Bn))
+    cur_ids = torch.zeros(MB, Bn, dtype=torch.int32, device=dev)
+    slots = [list(range(mb * Bn, (mb + 1) * Bn)) for mb in range(MB)]
     hid_host = torch.empty(Bn, T, m.d_model, dtype=torch.float32).pin_memory()
     row_host = torch.empty(Bn, 1, m.d_model, dtype=torch.float32).pin_memory()
     tok_host = torch.empty(Bn, dtype=torch.int32).pin_memory()
 
+    def shard_slice(i):
+        b0, b1 = wl.layer_begin + i * per, wl.layer_begin + (i + 1) * per
+        w = {"layers": weights["layers"][i * per:(i + 1) * per]}
+        if b0 == 0:
+            w["tok_embedding"] = weights["tok_embedding"]
+        if b1 == m.n_layers:
+            w["final_norm"], w["lm_head"] = weights["final_norm"], weights["lm_head"]
+        return b0, b1, w
+
     with torch.cuda.stream(stream):
-        sh = B.Shard(m, wl.layer_begin, wl.layer_end, weights, max_slots=Bn, max_seq=T + S, max_tokens=Bn * T,
-                     stream=stream)
+        shards = []
+        for i in range(n_sh):
+            b0, b1, w = shard_slice(i)
+            shards.append(B.Shard(m, b0, b1, w, max_slots=MB * Bn, max_seq=T + S, max_tokens=Bn * T, max_batch=Bn,
+                                  stream=stream))
+        sh = shards[0]
+
+        def through(mb, first_ids, prefill):
+            """one micro-batch through every shard; on one device the hand-over is the handoff view itself"""
+            x = None
+            for si, shd in enumerate(shards):
+                if prefill:
+                    shd.es_shard_prefill(first_ids if si == 0 else None, x, Bn, T, slots[mb])
+                else:
+                    shd.es_shard_decode_step(first_ids if si == 0 else None, x, Bn, slots[mb])
+                x, lg, nx = shd.es_shard_handoff()
+            return x, lg, nx
 
         def one_step(e2e: bool, events=None):
             """prefill + S decode steps.  e2e: inputs come from pinned host memory every call and the
-            result (handoff activation, or the token when the shard holds the head) goes back."""
+            result (handoff activation, or the token when the last shard holds the head) goes back."""
             if events:
                 events[0].record(stream)
-            if e2e:
-                ids_dev.copy_(ids_host, non_blocking=True)
-            sh.es_shard_prefill(ids_dev, None, Bn, T, slots)
-            h, lg, nx = sh.es_shard_handoff()
-            if e2e:
-                (tok_host.copy_(nx, non_blocking=True) if wl.has_head else hid_host.copy_(h, non_blocking=True))
+            nx = None
+            for mb in range(MB):
+                if e2e:
+                    ids_dev[mb].copy_(ids_host[mb], non_blocking=True)
+                h, lg, nx = through(mb, ids_dev[mb], True)
+                if wl.has_head and MB > 1:
+                    cur_ids[mb].copy_(nx)
+                if e2e:
+                    (tok_host.copy_(nx, non_blocking=True) if wl.has_head else hid_host.copy_(h, non_blocking=True))
             if events:
                 events[1].record(stream)
             for s in range(S):
-                if wl.has_head:
-                    src = nx                                    # greedy feedback stays on the device
-                else:
-                    cur_ids.copy_(forced_host[s] if e2e else forced_dev[s], non_blocking=True)
-                    src = cur_ids
-                sh.es_shard_decode_step(src, None, Bn, slots)
-                if e2e:
-                    h, lg, nx2 = sh.es_shard_handoff()
-                    (tok_host.copy_(nx2, non_blocking=True) if wl.has_head else row_host.copy_(h, non_blocking=True))
+                for mb in range(MB):
+                    if wl.has_head:
+                        src = nx if MB == 1 else cur_ids[mb]     # greedy feedback stays on the device
+                    else:
+                        cur_ids[mb].copy_(forced_host[s, mb] if e2e else forced_dev[s, mb], non_blocking=True)
+                        src = cur_ids[mb]
+                    h, lg, nx2 = through(mb, src, False)
+                    if wl.has_head and MB > 1:
+                        cur_ids[mb].copy_(nx2)
+                    if e2e:
+                        (tok_host.copy_(nx2, non_blocking=True) if wl.has_head else row_host.copy_(h, non_blocking=True))
             if events:
                 events[2].record(stream)
 
@@ -210,12 +243,12 @@ def run_ours(args):
         def timed(e2e: bool):
             evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
             _barrier(world)
-            n0 = sh.es_shard_launch_count()
+            n0 = sum(x.es_shard_launch_count() for x in shards)
             for k in range(args.steps):
                 one_step(e2e, evs[k])
             stream.synchronize()
             _barrier(world)
-            n1 = sh.es_shard_launch_count()
+            n1 = sum(x.es_shard_launch_count() for x in shards)
             pre = [e[0].elapsed_time(e[1]) for e in evs]
             dec = [e[1].elapsed_time(e[2]) for e in evs]
             return pre, dec, n1 - n0
@@ -237,17 +270,18 @@ def run_ours(args):
         clocks = sampler.stop() if rank == 0 else None
 
         # dominant kernel: the weight-streaming linear kernel, timed launch by launch with CUDA events
-        sh.es_shard_prefill(ids_dev, None, Bn, T, slots)
-        src = sh.es_shard_handoff()[2] if wl.has_head else cur_ids
+        sh.es_shard_prefill(ids_dev[0], None, Bn, T, slots[0])
+        src = sh.es_shard_handoff()[2] if (wl.has_head and n_sh == 1) else cur_ids[0]
         sh.es_shard_set_kernel_timing(True)
         torch.cuda._sleep(4_000_000)           # let the host run ahead so the event pairs bracket only the kernels
         for _ in range(min(4, S)):
-            sh.es_shard_decode_step(src, None, Bn, slots)
+            sh.es_shard_decode_step(src, None, Bn, slots[0])
         t = sh.es_shard_kernel_timing()
         sh.es_shard_set_kernel_timing(False)
         kt = {"gbs": t["bytes"] / (t["ms"] / 1e3) / 1e9, "launches": t["launches"],
               "avg_us": 1e3 * t["ms"] / t["launches"], "bytes_per_launch": t["bytes"] / t["launches"]}
-        sh.es_shard_device_status()
+        for x in shards:
+            x.es_shard_device_status()
 
     dec_total = _max_over_ranks(sum(dec), world)
     pre_mean = _max_over_ranks(sum(pre) / len(pre), world)
@@ -257,11 +291,11 @@ def run_ours(args):
     if rank != 0:
         return None
 
-    tokens = Bn * S * args.steps * world
+    tokens = MB * Bn * S * args.steps * world
     value = tokens / (dec_total / 1e3)
     value_e = tokens / (dec_total_e / 1e3)
     ctx_avg = T + (S + 1) / 2.0
-    step_bytes = algorithmic_decode_bytes(wl, ctx_avg)
+    step_bytes = MB * algorithmic_decode_bytes(wl, ctx_avg)     # every micro-batch pass re-streams the weights
     peak, peak_kind = _peaks()
     decode_ms = dec_total / (S * args.steps)
     out = {
@@ -270,17 +304,18 @@ def run_ours(args):
         "dtype": "f16", "data": "synthetic",
         "config": {"workload": f"{args.workload}: {m.name} layers {wl.layer_begin}-{wl.layer_end - 1}"
                                f"{' +embedding' if wl.has_embedding else ''}{' +head' if wl.has_head else ''}, "
-                               f"batch {Bn}, prompt {T}, decode {S}",
+                               f"batch {Bn}, prompt {T}, decode {S}"
+                               + (f", {n_sh} shards in sequence, {MB} micro-batches" if n_sh > 1 or MB > 1 else ""),
                    "parallelism": "replicas" if world > 1 else "single",
                    "l2": "no flush: each step streams %.2f GB of weights, far more than the 126 MB L2" % (linear_weight_bytes(wl) / 1e9)},
         "prefill_ms": pre_mean,
         "decode_ms_per_step": decode_ms,
         "decode_hbm_frac_of_step": step_bytes / (decode_ms / 1e3) / 1e9 / peak,
-        "prefill_tflops": prefill_flops(wl) / (pre_mean / 1e3) / 1e12,
+        "prefill_tflops": MB * prefill_flops(wl) / (pre_mean / 1e3) / 1e12,
         "e2e": {"value": value_e, "unit": UNIT, "prefill_ms": pre_mean_e,
                 "h2d_bytes_per_step": int(ids_host.numel() * 4 + (0 if wl.has_head else forced_host.numel() * 4)),
-                "d2h_bytes_per_step": int((tok_host.numel() * 4 * (S + 1)) if wl.has_head
-                                          else (hid_host.numel() + S * row_host.numel()) * 4)},
+                "d2h_bytes_per_step": int(MB * ((tok_host.numel() * 4 * (S + 1)) if wl.has_head
+                                                else (hid_host.numel() + S * row_host.numel()) * 4))},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "linear_stream_kernel", "achieved": kt["gbs"], "peak": peak,
