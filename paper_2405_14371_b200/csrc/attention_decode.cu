@@ -20,8 +20,11 @@ namespace {
 
 constexpr int DWARPS = 8;
 
-template <int HD, int G>
-__global__ void __launch_bounds__(DWARPS * 32) decode_attn_split_kernel(const DecodeAttnParams p) {
+// PRE: keep the first block's K rows in registers across the dependency wait.  That shortens the
+// critical path of small, latency-bound launches but costs registers, so launches with many CTAs
+// (several sequences, long contexts), which live on occupancy, are built without it.
+template <int HD, int G, bool PRE>
+__global__ void __launch_bounds__(DWARPS * 32, PRE ? 1 : 2) decode_attn_split_kernel(const DecodeAttnParams p) {
   pdl_launch_dependents();
   constexpr int E = HD / 32;
   __shared__ __align__(16) float q_s[G][HD];
@@ -44,7 +47,7 @@ __global__ void __launch_bounds__(DWARPS * 32) decode_attn_split_kernel(const De
   if (t_begin >= ctx) { pdl_wait(); return; }
   const int t_end = min(ctx, t_begin + tokens_per_split);
   const float scale = rsqrtf((float)HD);
-  constexpr bool PRELOAD = (G <= 2);            // K row of the first block kept in registers across the wait
+  constexpr bool PRELOAD = PRE && (G <= 2);     // K row of the first block kept in registers across the wait
 
   const int t_first = t_begin + warp * 32 + lane;
   const bool first_valid = t_first < t_end;
@@ -101,7 +104,7 @@ __global__ void __launch_bounds__(DWARPS * 32) decode_attn_split_kernel(const De
       const uint4* k4 = reinterpret_cast<const uint4*>(kr);
       const bool use_pre = PRELOAD && first && first_old;
       // all 16-byte pieces of the row are requested up front when registers allow (small groups)
-      constexpr int KU = (G <= 2) ? HD / 8 : 4;
+      constexpr int KU = PRE ? ((G <= 2) ? HD / 8 : 4) : 8;
 #pragma unroll KU
       for (int c = 0; c < HD / 8; ++c) {
         const uint4 u = use_pre ? kpre[PRELOAD ? c : 0] : k4[c];
@@ -143,7 +146,7 @@ __global__ void __launch_bounds__(DWARPS * 32) decode_attn_split_kernel(const De
     }
     // value rows of the 32 tokens; lanes past the end carry probability 0 and a valid (repeated) offset
     const int cnt = min(32, t_end - t0);
-    constexpr int VU = (G <= 2) ? 16 : 8;
+    constexpr int VU = (PRE && G <= 2) ? 16 : 8;
 #pragma unroll VU
     for (int jj = 0; jj < 32; ++jj) {
       const uint32_t o16 = __shfl_sync(0xffffffffu, off16, jj < cnt ? jj : 0);
@@ -222,7 +225,11 @@ __global__ void __launch_bounds__(HD) decode_attn_merge_kernel(const DecodeAttnP
 
 template <int HD, int G>
 es_status_t launch_g(const DecodeAttnParams& p, cudaStream_t s, bool pdl) {
-  ES_CUDA_CHECK(launch_kernel(decode_attn_split_kernel<HD, G>, dim3(p.n_splits, p.Hkv, p.B), dim3(DWARPS * 32), 0, s, pdl, p));
+  const bool small = (long long)p.n_splits * p.Hkv * p.B <= 2 * 148;
+  if (small)
+    ES_CUDA_CHECK(launch_kernel(decode_attn_split_kernel<HD, G, true>, dim3(p.n_splits, p.Hkv, p.B), dim3(DWARPS * 32), 0, s, pdl, p));
+  else
+    ES_CUDA_CHECK(launch_kernel(decode_attn_split_kernel<HD, G, false>, dim3(p.n_splits, p.Hkv, p.B), dim3(DWARPS * 32), 0, s, pdl, p));
   return ES_OK;
 }
 
