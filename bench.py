@@ -157,7 +157,7 @@ def run_ours(args):
     rank, local, world = _dist_setup(args.gpus)
     wl = WORKLOADS[args.workload]
     m = wl.model
-    Bn, T, S = wl.batch, wl.prompt_len, (args.decode_steps or wl.decode_steps)
+    Bn, T, S = (args.batch or wl.batch), (args.prompt_len or wl.prompt_len), (args.decode_steps or wl.decode_steps)
     dev = torch.device("cuda", local)
     stream = torch.cuda.Stream(device=dev)
     weights = shard_weights(wl.cfg, m, wl.layer_begin, wl.layer_end, device=dev)
@@ -262,7 +262,7 @@ def run_ours(args):
             sampler.stop()
             stream.synchronize()
             if rank == 0:
-                print(json.dumps({"profile_run": True, "workload": args.workload, "decode_steps": S,
+                print(json.dumps({"profile_run": True, "workload": args.workload, "batch": Bn, "prompt_len": T, "decode_steps": S,
                                   "prefill_ms": sum(pre) / len(pre), "decode_ms_per_step": sum(dec) / (S * len(dec)),
                                   "gpu_launches": int(launches)}))
             return None
@@ -411,7 +411,11 @@ def main():
     ap.add_argument("--profile", action="store_true",
                     help="short run for an ncu capture: 1 warm-up pass, 1 timed pass, no e2e / kernel-timing / CPU legs")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (profile runs)")
+    ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length (profile runs only)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profile runs only)")
     args = ap.parse_args()
+    if (args.prompt_len or args.batch) and not args.profile:
+        ap.error("--prompt-len / --batch change the workload and are only accepted together with --profile")
     if args.profile:
         args.warmup, args.steps = 1, 1
     else:
