@@ -54,7 +54,7 @@ es_status_t es_op_decode_attention_static(const void* q, const void* k_pages, co
   p.kv.k = (const __half*)k_pages; p.kv.v = (const __half*)v_pages; p.kv.block_table = block_table; p.kv.slots = nullptr;
   p.kv.page_stride = (int64_t)Hkv * page_tokens * hd; p.kv.head_stride = (int64_t)page_tokens * hd; p.kv.tok_stride = hd;
   p.kv.P = page_tokens; p.kv.pages_per_slot = pages_per_seq;
-  choose_splits(max_ctx, page_tokens, B, Hkv, &p.n_splits, &p.pages_per_split);
+  choose_splits(max_ctx, page_tokens, B, Hkv, Hq / Hkv, &p.n_splits, &p.pages_per_split);
   const size_t need = decode_attention_scratch_bytes(B, Hq, hd, p.n_splits);
   if (need > STATIC_SCRATCH_BYTES)
     return fail(ES_ERR_WORKSPACE, "this call needs %zu bytes of split-KV scratch but the built-in array holds %zu; "

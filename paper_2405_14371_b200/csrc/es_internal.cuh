@@ -159,7 +159,7 @@ struct DecodeAttnParams {
   int n_splits, pages_per_split;
 };
 size_t decode_attention_scratch_bytes(int B, int Hq, int hd, int n_splits);
-void choose_splits(int max_ctx, int P, int B, int Hkv, int* n_splits, int* pages_per_split);
+void choose_splits(int max_ctx, int P, int B, int Hkv, int group, int* n_splits, int* pages_per_split);
 es_status_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t s, int64_t* launches, bool pdl = false);
 
 }  // namespace es

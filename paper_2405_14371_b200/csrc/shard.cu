@@ -47,9 +47,12 @@ const Tunables& tunables() {
 
 // How the context of a decode-attention call is cut into splits: enough CTAs to fill the machine,
 // never less than one KV page per split.
-void choose_splits(int max_ctx, int P, int B, int Hkv, int* n_splits, int* pages_per_split) {
+void choose_splits(int max_ctx, int P, int B, int Hkv, int group, int* n_splits, int* pages_per_split) {
   const int pages = (max_ctx + P - 1) / P;
-  long long pps = (long long)pages * B * Hkv / (4 * 148);
+  // about one CTA per SM when every KV head serves one or two query heads (the kernel then lives on
+  // bytes in flight); four times as many for larger groups, whose CTAs are arithmetic heavy
+  const int ctas = (group >= 4 ? 4 : 1) * 148;
+  long long pps = (long long)pages * B * Hkv / ctas;
   const int min_pps = 256 / P > 1 ? 256 / P : 1;      // at least 256 tokens per split
   if (pps < min_pps) pps = min_pps;
   if (pps > pages) pps = pages;
@@ -100,7 +103,7 @@ Layout make_layout(const es_model_desc_t& d, int begin, int end) {
   L.n_pages = L.pages_per_slot * d.max_slots;
   L.page_elems = (size_t)d.n_kv_heads * P * d.head_dim;
   L.kv_bytes = align_up((size_t)nl * 2 * L.n_pages * L.page_elems * sizeof(__half));
-  choose_splits(d.max_seq, P, d.max_batch, d.n_kv_heads, &L.n_splits, &L.pages_per_split);
+  choose_splits(d.max_seq, P, d.max_batch, d.n_kv_heads, d.n_heads / d.n_kv_heads, &L.n_splits, &L.pages_per_split);
   const size_t M = d.max_tokens, B = d.max_batch, nq = (size_t)d.n_heads * d.head_dim;
   const bool head = end == d.n_layers_total;
   size_t o = 0;
@@ -914,7 +917,7 @@ es_status_t es_op_decode_attention(const void* q, const void* k_pages, const voi
   p.kv.k = (const __half*)k_pages; p.kv.v = (const __half*)v_pages; p.kv.block_table = block_table; p.kv.slots = nullptr;
   p.kv.page_stride = (int64_t)Hkv * page_tokens * hd; p.kv.head_stride = (int64_t)page_tokens * hd; p.kv.tok_stride = hd;
   p.kv.P = page_tokens; p.kv.pages_per_slot = pages_per_seq;
-  choose_splits(max_ctx, page_tokens, B, Hkv, &p.n_splits, &p.pages_per_split);
+  choose_splits(max_ctx, page_tokens, B, Hkv, Hq / Hkv, &p.n_splits, &p.pages_per_split);
   if (scratch_bytes < decode_attention_scratch_bytes(B, Hq, hd, p.n_splits))
     return fail(ES_ERR_WORKSPACE, "scratch: %zu bytes given, %zu needed", scratch_bytes,
                 decode_attention_scratch_bytes(B, Hq, hd, p.n_splits));
