@@ -32,6 +32,7 @@ struct Tunables {
   int stream_prefetch_row_bytes;   // ES_STREAM_PREFETCH: bytes of each first row pair prefetched into L2 before the dependency wait
   int stream_ctas_per_sm;          // ES_STREAM_CTAS: cap on resident CTAs per SM of the weight-streaming kernel (0 = occupancy limit)
   int stream_deep;                 // ES_STREAM_DEEP: -1 auto, 0 never, 1 always use the deeper (U = 4) chunking
+  int tc_pair;                     // ES_TC_PAIR: CTA-pair tensor-core kernel for large prefill products (1) or never (0)
   int pdl;                         // ES_PDL: programmatic dependent launch in decode steps (1) or plain stream order (0)
 };
 const Tunables& tunables();
@@ -92,6 +93,9 @@ bool linear_stream_mma_supported(const LinearParams& p, int epi);
 es_status_t launch_linear_stream_mma(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl = false);
 es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word);
 bool linear_tc_supported(const LinearParams& p, int epi);
+// CTA-pair (cta_group::2) variant for large M; uses the same tensor maps
+bool linear_tc2_supported(const LinearParams& p, int epi);
+es_status_t launch_linear_tc2(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word);
 // Encodes the tensor maps for p's operands; the A map covers a_rows rows (the buffer's capacity).
 es_status_t tc_build_maps(const LinearParams& p, int epi, int64_t a_rows, TcMaps* out);
 

@@ -41,7 +41,7 @@ static int env_int(const char* name, int dflt) {
 
 const Tunables& tunables() {
   static const Tunables t = {env_int("ES_STREAM_PREFETCH", 0), env_int("ES_STREAM_CTAS", 0), env_int("ES_STREAM_DEEP", -1),
-                             env_int("ES_PDL", 1)};
+                             env_int("ES_TC_PAIR", 1), env_int("ES_PDL", 1)};
   return t;
 }
 
@@ -237,6 +237,7 @@ es_status_t dispatch_linear(es_shard* s, const LinearParams& p, int epi) {
   if (p.M > 2 && p.M <= 16 && linear_stream_mma_supported(p, epi))
     return launch_linear_stream_mma(p, epi, s->stream, &s->launches, s->pdl_now);
   if (p.M <= 16) return launch_linear_stream(p, epi, s->stream, &s->launches, s->pdl_now);
+  if (tunables().tc_pair && linear_tc2_supported(p, epi)) return launch_linear_tc2(p, epi, s->stream, &s->launches, s->status);
   if (linear_tc_supported(p, epi)) return launch_linear_tc(p, epi, s->stream, &s->launches, s->status);
   return launch_linear_reference(p, epi, s->stream, &s->launches);
 }
@@ -876,6 +877,9 @@ es_status_t es_op_linear(const void* A, const void* W, const float* R, float* C,
       return launch_linear_tc(p, EPI_F32, st, nullptr, nullptr);
     case 2: return launch_linear_stream(p, EPI_F32, st, nullptr);
     case 3: return launch_linear_reference(p, EPI_F32, st, nullptr);
+    case 5:
+      if (!linear_tc2_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "pair kernel does not take this shape");
+      return launch_linear_tc2(p, EPI_F32, st, nullptr, nullptr);
     case 4:
       if (!linear_stream_mma_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "tensor-core streaming kernel does not take this shape");
       return launch_linear_stream_mma(p, EPI_F32, st, nullptr);

@@ -84,6 +84,19 @@ def test_linear_streaming_tensor_core(B, M, N, K):
     assert rel_err(B.es_op_linear(A.cuda(), W.cuda(), None, 4), want) < 5e-5
 
 
+@pytest.mark.parametrize("M,N,K", [(2048, 4096, 1024), (1100, 5000, 520), (4096, 4096, 4096), (512, 12288, 4096)])
+def test_linear_tensor_core_cta_pairs(B, M, N, K):
+    """cta_group::2 kernel: 256 x 256 tiles on CTA pairs, ragged M / N / K, agreement with the single-CTA kernel."""
+    A = _randn(M, K, seed=19)
+    W = _randn(N, K, seed=20, scale=0.05)
+    R = _randn(M, N, seed=21, dtype=torch.float32)
+    got = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), 5)
+    ref = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), 1)
+    want = A.double() @ W.double().T + R.double()
+    assert rel_err(got, want) < 5e-5
+    assert rel_err(got, ref) < 1e-5
+
+
 def test_linear_rejects_bad_shapes(B):
     A = _randn(17, 64).cuda()
     W = _randn(32, 64).cuda()
