@@ -22,7 +22,7 @@ namespace {
 constexpr int MW = 8;                 // warps per CTA
 constexpr int MTHREADS = MW * 32;
 constexpr int KSTEP = 32;             // K elements per lane-load step
-constexpr int UM = 4;                 // steps per chunk
+constexpr int UM_TOTAL = 4;           // lane-load steps per chunk over all row groups of a warp
 
 __device__ __forceinline__ uint4 ld_stream16(const void* ptr) {
   uint4 v;
@@ -39,53 +39,64 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// NT: groups of 8 activation rows (1 or 2).
-template <int NT, int EPI, bool A_SMEM>
+// NT: groups of 8 activation rows (1 or 2).  RG: 16-row groups of weights a warp carries at once (1 or
+// 2); with two, every activation fragment is used twice, which halves the activation traffic when
+// the activations do not fit in shared memory and come through L1 / L2.
+template <int NT, int EPI, bool A_SMEM, int RG>
 __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const LinearParams p, int a_stride) {
   pdl_launch_dependents();
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __half* a_s = reinterpret_cast<__half*>(smem_raw);                 // [NT*8][a_stride], padded rows
-  __shared__ float red[2][MW][NT][32][4];
+  __shared__ float red[2][MW][RG][NT][32][4];
 
   const int K = p.K;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, q = lane & 3;
-  constexpr int COLS = (EPI == EPI_SWIGLU) ? 8 : 16;                 // output columns per unit
+  constexpr int COLS = RG * ((EPI == EPI_SWIGLU) ? 8 : 16);           // output columns per unit
   const int n_units = (p.N + COLS - 1) / COLS;
   const int u0 = (int)((int64_t)blockIdx.x * n_units / gridDim.x);
   const int u1 = (int)((int64_t)(blockIdx.x + 1) * n_units / gridDim.x);
   const int n_my = u1 - u0;
   const int kslice = K / MW;                                         // multiple of KSTEP (checked on the host)
   const int k_lo = warp * kslice, k_hi = k_lo + kslice;
+  constexpr int UM = UM_TOTAL / RG;                                    // steps per chunk: same registers for either RG
   constexpr int CHUNK_K = KSTEP * UM;
   const int chunks_per_unit = (kslice + CHUNK_K - 1) / CHUNK_K;
   const int total = n_my * chunks_per_unit;
 
-  auto unit_rows = [&](int i, const __half*& r0, const __half*& r1) {
+  auto unit_rows = [&](int i, const __half* (&r0)[RG], const __half* (&r1)[RG]) {
     const int u = u0 + i;
-    if (EPI == EPI_SWIGLU) {
-      const int n = u * 8 + g;
-      r0 = (n < p.N) ? p.w[0] + (int64_t)n * K : nullptr;
-      r1 = (n < p.N) ? p.w[1] + (int64_t)n * K : nullptr;
-    } else {
-      const int n = u * 16 + g;
-      r0 = (n < p.N) ? weight_row(p, n) : nullptr;
-      r1 = (n + 8 < p.N) ? weight_row(p, n + 8) : nullptr;
+#pragma unroll
+    for (int rg = 0; rg < RG; ++rg) {
+      if (EPI == EPI_SWIGLU) {
+        const int n = u * COLS + rg * 8 + g;
+        r0[rg] = (n < p.N) ? p.w[0] + (int64_t)n * K : nullptr;
+        r1[rg] = (n < p.N) ? p.w[1] + (int64_t)n * K : nullptr;
+      } else {
+        const int n = u * COLS + rg * 16 + g;
+        r0[rg] = (n < p.N) ? weight_row(p, n) : nullptr;
+        r1[rg] = (n + 8 < p.N) ? weight_row(p, n + 8) : nullptr;
+      }
     }
   };
 
   int nxt_i = 0, nxt_cc = 0;
-  const __half* nr0 = nullptr;
-  const __half* nr1 = nullptr;
+  const __half* nr0[RG];
+  const __half* nr1[RG];
+#pragma unroll
+  for (int rg = 0; rg < RG; ++rg) nr0[rg] = nr1[rg] = nullptr;
   if (total > 0) unit_rows(0, nr0, nr1);
-  auto issue = [&](uint4 (&w0)[UM], uint4 (&w1)[UM]) {
+  auto issue = [&](uint4 (&w0)[RG][UM], uint4 (&w1)[RG][UM]) {
     const int kb = k_lo + nxt_cc * CHUNK_K + q * 8;
 #pragma unroll
     for (int j = 0; j < UM; ++j) {
       const int k = kb + j * KSTEP;
       const bool in = k < k_hi;
-      w0[j] = (in && nr0) ? ld_stream16(nr0 + k) : make_uint4(0, 0, 0, 0);
-      w1[j] = (in && nr1) ? ld_stream16(nr1 + k) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int rg = 0; rg < RG; ++rg) {
+        w0[rg][j] = (in && nr0[rg]) ? ld_stream16(nr0[rg] + k) : make_uint4(0, 0, 0, 0);
+        w1[rg][j] = (in && nr1[rg]) ? ld_stream16(nr1[rg] + k) : make_uint4(0, 0, 0, 0);
+      }
     }
     if (++nxt_cc == chunks_per_unit) {
       nxt_cc = 0;
@@ -93,7 +104,7 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
     }
   };
 
-  uint4 b0w0[UM], b0w1[UM], b1w0[UM], b1w1[UM];
+  uint4 b0w0[RG][UM], b0w1[RG][UM], b1w0[RG][UM], b1w1[RG][UM];
   if (total > 0) {
     issue(b0w0, b0w1);
     if (total > 1) issue(b1w0, b1w1);
@@ -112,14 +123,16 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
     __syncthreads();
   }
 
-  float acc[NT][4];
+  float acc[RG][NT][4];
 #pragma unroll
-  for (int t = 0; t < NT; ++t)
+  for (int rg = 0; rg < RG; ++rg)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) acc[t][i] = 0.f;
+    for (int t = 0; t < NT; ++t)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) acc[rg][t][i] = 0.f;
   int cur_i = 0, cur_cc = 0;
 
-  auto consume = [&](const uint4 (&w0)[UM], const uint4 (&w1)[UM]) {
+  auto consume = [&](const uint4 (&w0)[RG][UM], const uint4 (&w1)[RG][UM]) {
     const int kb = k_lo + cur_cc * CHUNK_K + q * 8;
 #pragma unroll
     for (int j = 0; j < UM; ++j) {
@@ -131,8 +144,11 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
           uint4 a;
           if (A_SMEM) a = *reinterpret_cast<const uint4*>(a_s + (int64_t)m * a_stride + k);
           else a = (m < p.M) ? __ldg(reinterpret_cast<const uint4*>(p.A + (int64_t)m * p.lda + k)) : make_uint4(0, 0, 0, 0);
-          mma16816(acc[t], w0[j].x, w1[j].x, w0[j].y, w1[j].y, a.x, a.y);
-          mma16816(acc[t], w0[j].z, w1[j].z, w0[j].w, w1[j].w, a.z, a.w);
+#pragma unroll
+          for (int rg = 0; rg < RG; ++rg) {
+            mma16816(acc[rg][t], w0[rg][j].x, w1[rg][j].x, w0[rg][j].y, w1[rg][j].y, a.x, a.y);
+            mma16816(acc[rg][t], w0[rg][j].z, w1[rg][j].z, w0[rg][j].w, w1[rg][j].w, a.z, a.w);
+          }
         }
       }
     }
@@ -140,16 +156,19 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
       // unit finished in this warp's K slice: add the 8 slices in warp order
       const int buf = cur_i & 1;
 #pragma unroll
-      for (int t = 0; t < NT; ++t) {
-        *reinterpret_cast<float4*>(&red[buf][warp][t][lane][0]) = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
+      for (int rg = 0; rg < RG; ++rg)
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc[t][i] = 0.f;
-      }
+        for (int t = 0; t < NT; ++t) {
+          *reinterpret_cast<float4*>(&red[buf][warp][rg][t][lane][0]) =
+              make_float4(acc[rg][t][0], acc[rg][t][1], acc[rg][t][2], acc[rg][t][3]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) acc[rg][t][i] = 0.f;
+        }
       __syncthreads();
-      // thread -> (output pair pr, activation row m).  Accumulator element (row r, column m) of group t
-      // lives in lane (r % 8) * 4 + (m % 8) / 2, register (r / 8) * 2 + (m % 2).
-      if (threadIdx.x < 8 * NT * 8) {
-        const int pr = threadIdx.x & 7, m = threadIdx.x >> 3;
+      // thread -> (row group rg, output pair pr, activation row m).  Accumulator element (row r, column m)
+      // of group t lives in lane (r % 8) * 4 + (m % 8) / 2, register (r / 8) * 2 + (m % 2).
+      for (int idx = threadIdx.x; idx < RG * 8 * NT * 8; idx += MTHREADS) {
+        const int pr = idx & 7, m = (idx >> 3) % (NT * 8), rg = idx / (8 * NT * 8);
         const int t = m >> 3, mc = m & 7;
         int ra, rb;                                  // the two accumulator rows this thread combines
         if (EPI == EPI_SWIGLU) { ra = pr; rb = pr + 8; }
@@ -159,11 +178,11 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
         float v0 = 0.f, v1 = 0.f;
 #pragma unroll
         for (int w = 0; w < MW; ++w) {
-          v0 += red[buf][w][t][la][ia];
-          v1 += red[buf][w][t][lb][ib];
+          v0 += red[buf][w][rg][t][la][ia];
+          v1 += red[buf][w][rg][t][lb][ib];
         }
         const int u = u0 + cur_i;
-        const int n = (EPI == EPI_SWIGLU) ? u * 8 + pr : u * 16 + 2 * pr;
+        const int n = (EPI == EPI_SWIGLU) ? u * COLS + rg * 8 + pr : u * COLS + rg * 16 + 2 * pr;
         epi_pair<EPI>(p, m, n, v0, v1);
       }
       cur_cc = 0;
@@ -181,9 +200,9 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
   }
 }
 
-template <int NT, int EPI, bool A_SMEM>
+template <int NT, int EPI, bool A_SMEM, int RG>
 es_status_t launch_inst(const LinearParams& p, cudaStream_t s, bool pdl) {
-  auto kern = linear_stream_mma_kernel<NT, EPI, A_SMEM>;
+  auto kern = linear_stream_mma_kernel<NT, EPI, A_SMEM, RG>;
   const int a_stride = p.K + 8;                       // 16 bytes of padding: the 8 rows fall into different banks
   const size_t smem = A_SMEM ? (size_t)NT * 8 * a_stride * sizeof(__half) : 0;
   static size_t configured = 0;
@@ -200,7 +219,7 @@ es_status_t launch_inst(const LinearParams& p, cudaStream_t s, bool pdl) {
   int per_sm = 0;
   ES_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, MTHREADS, smem));
   if (per_sm < 1) return fail(ES_ERR_SHAPE, "tensor-core streaming kernel does not fit (K = %d)", p.K);
-  constexpr int COLS = (EPI == EPI_SWIGLU) ? 8 : 16;
+  constexpr int COLS = RG * ((EPI == EPI_SWIGLU) ? 8 : 16);
   const int n_units = (p.N + COLS - 1) / COLS;
   int grid = sms * per_sm;
   if (grid > n_units) grid = n_units;
@@ -211,8 +230,10 @@ es_status_t launch_inst(const LinearParams& p, cudaStream_t s, bool pdl) {
 template <int NT, int EPI>
 es_status_t launch_nt(const LinearParams& p, cudaStream_t s, bool pdl) {
   const size_t a_bytes = (size_t)NT * 8 * (p.K + 8) * sizeof(__half);
-  if (a_bytes <= 100 * 1024) return launch_inst<NT, EPI, true>(p, s, pdl);
-  return launch_inst<NT, EPI, false>(p, s, pdl);
+  if (a_bytes <= 100 * 1024) return launch_inst<NT, EPI, true, 1>(p, s, pdl);
+  // through L1 / L2: with 16 activation rows their traffic equals the weights', so a warp carries two
+  // weight row groups per activation fragment; with 8 rows the longer contiguous runs per row win
+  return launch_inst<NT, EPI, false, (NT == 2 ? 2 : 1)>(p, s, pdl);
 }
 
 template <int EPI>
