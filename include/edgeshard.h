@@ -194,6 +194,31 @@ ES_API void es_shard_destroy(es_shard_t *shard);
 ES_API const char *es_last_error(void);
 ES_API const char *es_version(void);
 
+/* ---- partition planners (host only) ------------------------------------------------------------
+ * The paper's two dynamic programs over the profiled traces.  N layers (layer 0 = embedding, pinned to
+ * device 0 by the privacy constraint), M devices; all arrays host, double:
+ *   t_comp [N, M]  time of layer i on device j          O   [N]  activation size of layer i
+ *   Req    [N]     memory of layer i                     Mem [M]  memory budget of device j
+ *   Bw     [M, M]  bandwidth from device k to device j (same unit as O per unit of time; diagonal unused)
+ *   assign [N]     out: device of every layer
+ * ES_ERR_RANGE if no placement fits the memory budgets.
+ *
+ * es_partition_latency — Algorithm 1 / Eq. 4: DP(i, j) = min_k DP(i-1, k) + t_comp(i, j) + O(i-1)/Bw(k, j),
+ * plus the return of the token O(N-1)/Bw(j, 0) at the last layer; DP(0, 0) = t_comp(0, 0).  Memory is
+ * tracked along each cell's own best path (the algorithm's "update memory" step): the result is always
+ * feasible, and optimal whenever the budgets do not bind on that path.  *latency = total time T_tol (Eq. 2).
+ *
+ * es_partition_throughput — Algorithm 2: every chosen device holds one contiguous range of layers;
+ * g(m, S + {j}, j) = min over (i, k) of max(g(i, S, k), O(i-1)/Bw(k, j), t_comp(i..m-1, j)), memory
+ * Req(i..m-1) <= Mem(j) per device; the source device holds the first range, which contains layer 0 and
+ * may contain more.  *bottleneck = the slowest stage's time (its reciprocal is the pipeline throughput).
+ * Exact; cost O(N^2 2^M M^2), M <= 20. */
+ES_API es_status_t es_partition_latency(int32_t N, int32_t M, const double *t_comp, const double *O, const double *Req,
+                                        const double *Mem, const double *Bw, int32_t *assign, double *latency);
+ES_API es_status_t es_partition_throughput(int32_t N, int32_t M, const double *t_comp, const double *O,
+                                           const double *Req, const double *Mem, const double *Bw, int32_t *assign,
+                                           double *bottleneck);
+
 /* ---- single operations (the steps of the path, exposed for unit parity tests) -----------------
  * All pointers dev unless marked host; `stream` is a cudaStream_t cast to void*.              */
 

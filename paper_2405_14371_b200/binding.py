@@ -84,6 +84,8 @@ def _load() -> C.CDLL:
         "es_shard_destroy": (None, [vp]),
         "es_last_error": (C.c_char_p, []),
         "es_version": (C.c_char_p, []),
+        "es_partition_latency": (i32, [i32, i32] + [P(C.c_double)] * 5 + [P(i32), P(C.c_double)]),
+        "es_partition_throughput": (i32, [i32, i32] + [P(C.c_double)] * 5 + [P(i32), P(C.c_double)]),
         "es_op_rmsnorm": (i32, [vp, vp, vp, i32, i32, C.c_float, vp]),
         "es_op_linear": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, vp]),
         "es_op_prefill_attention": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]),
@@ -102,7 +104,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ("es_shard_workspace_bytes es_shard_create es_shard_prefill es_shard_decode_step es_shard_handoff "
            "es_layer_profile es_shard_set_profiling es_shard_reset_slots es_shard_set_page_table es_shard_set_graphs "
-           "es_shard_device_status es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_kernel_timing_detail es_shard_destroy es_last_error es_version es_op_rmsnorm "
+           "es_partition_latency es_partition_throughput es_shard_device_status es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_kernel_timing_detail es_shard_destroy es_last_error es_version es_op_rmsnorm "
            "es_op_linear es_op_prefill_attention es_op_decode_attention_scratch_bytes es_op_decode_attention "
            "es_op_decode_attention_static_capacity es_op_decode_attention_static").split()
 
@@ -353,3 +355,27 @@ def es_op_decode_attention_static(q: torch.Tensor, k_pages: torch.Tensor, v_page
                                              _ptr(out), B, Hq, Hkv, hd, P, block_table.shape[1], max_ctx,
                                              _stream_ptr(stream)))
     return out
+
+
+def _partition(fn, t_comp, O, Req, Mem, Bw):
+    import numpy as np
+    t_comp = np.ascontiguousarray(t_comp, dtype=np.float64)
+    N, M = t_comp.shape
+    arrs = [t_comp] + [np.ascontiguousarray(a, dtype=np.float64) for a in (O, Req, Mem, Bw)]
+    if arrs[1].shape != (N,) or arrs[2].shape != (N,) or arrs[3].shape != (M,) or arrs[4].shape != (M, M):
+        raise EsError(2, "partition planner: array shapes do not match [N, M] / [N] / [N] / [M] / [M, M]")
+    assign = (C.c_int32 * N)()
+    value = C.c_double(0)
+    ptrs = [a.ctypes.data_as(C.POINTER(C.c_double)) for a in arrs]
+    _check(fn(N, M, *ptrs, assign, C.byref(value)))
+    return list(assign), value.value
+
+
+def es_partition_latency(t_comp, O, Req, Mem, Bw):
+    """(device of every layer, total latency): the paper's Algorithm 1 over profiled traces."""
+    return _partition(lib.es_partition_latency, t_comp, O, Req, Mem, Bw)
+
+
+def es_partition_throughput(t_comp, O, Req, Mem, Bw):
+    """(device of every layer, slowest stage time): the paper's Algorithm 2 over profiled traces."""
+    return _partition(lib.es_partition_throughput, t_comp, O, Req, Mem, Bw)

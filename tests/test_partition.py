@@ -1,0 +1,117 @@
+"""The paper's partition planners (Algorithm 1, Algorithm 2) against brute force on tiny instances, plus the
+special cases the paper describes."""
+import math
+import random
+
+import pytest
+
+from oracle.partition import latency_bruteforce, throughput_bruteforce
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2405_14371_b200 import build
+    build.build()
+    from paper_2405_14371_b200 import binding
+    return binding
+
+
+def _instance(rng, N, M, tight):
+    speed = [rng.uniform(0.5, 4.0) for _ in range(M)]
+    t_comp = [[rng.uniform(0.5, 2.0) * speed[j] for j in range(M)] for _ in range(N)]
+    O = [rng.uniform(0.1, 3.0) for _ in range(N)]
+    Req = [rng.uniform(0.5, 2.0) for _ in range(N)]
+    total = sum(Req)
+    Mem = [total * (rng.uniform(0.35, 0.8) if tight else 10.0) for _ in range(M)]
+    Bw = [[rng.uniform(0.2, 5.0) for _ in range(M)] for _ in range(M)]
+    return t_comp, O, Req, Mem, Bw
+
+
+def _latency_of(a, t_comp, O, Req, Mem, Bw):
+    N = len(a)
+    t = sum(t_comp[i][a[i]] for i in range(N))
+    t += sum(0.0 if a[i - 1] == a[i] else O[i - 1] / Bw[a[i - 1]][a[i]] for i in range(1, N))
+    t += 0.0 if a[-1] == 0 else O[N - 1] / Bw[a[-1]][0]
+    return t
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_latency_planner_is_optimal_when_memory_does_not_bind(B, seed):
+    rng = random.Random(seed)
+    N, M = rng.randint(2, 6), rng.randint(1, 3)
+    inst = _instance(rng, N, M, tight=False)
+    a, t = B.es_partition_latency(*inst)
+    _, want = latency_bruteforce(*inst)
+    assert a[0] == 0 and abs(t - want) < 1e-9 * max(1.0, want)
+    assert abs(_latency_of(a, *inst) - t) < 1e-9 * max(1.0, t)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_latency_planner_is_feasible_under_tight_memory(B, seed):
+    rng = random.Random(100 + seed)
+    N, M = rng.randint(3, 6), rng.randint(2, 3)
+    t_comp, O, Req, Mem, Bw = _instance(rng, N, M, tight=True)
+    ref_a, want = latency_bruteforce(t_comp, O, Req, Mem, Bw)
+    try:
+        a, t = B.es_partition_latency(t_comp, O, Req, Mem, Bw)
+    except B.EsError as e:
+        assert e.status == 3        # the path-tracked budget found nothing (allowed: it is a heuristic there)
+        return
+    use = [sum(Req[i] for i in range(N) if a[i] == j) for j in range(M)]
+    assert all(use[j] <= Mem[j] + 1e-12 for j in range(M)) and a[0] == 0
+    assert ref_a is not None and t >= want - 1e-9
+    assert abs(_latency_of(a, t_comp, O, Req, Mem, Bw) - t) < 1e-9 * max(1.0, t)
+
+
+@pytest.mark.parametrize("tight", [False, True])
+@pytest.mark.parametrize("seed", range(10))
+def test_throughput_planner_matches_bruteforce(B, seed, tight):
+    rng = random.Random(200 + seed)
+    N, M = rng.randint(2, 6), rng.randint(1, 3)
+    inst = _instance(rng, N, M, tight)
+    ref_a, want = throughput_bruteforce(*inst)
+    if ref_a is None:
+        with pytest.raises(B.EsError) as e:
+            B.es_partition_throughput(*inst)
+        assert e.value.status == 3
+        return
+    a, t = B.es_partition_throughput(*inst)
+    assert abs(t - want) < 1e-9 * max(1.0, want)
+    # the returned map is a valid plan with that bottleneck: contiguous ranges, each device once, memory ok
+    t_comp, O, Req, Mem, Bw = inst
+    order = [a[0]] + [a[i] for i in range(1, N) if a[i] != a[i - 1]]
+    assert a[0] == 0 and len(set(order)) == len(order)
+    worst = 0.0
+    for q, j in enumerate(order):
+        layers = [i for i in range(N) if a[i] == j]
+        assert layers == list(range(layers[0], layers[-1] + 1))
+        assert sum(Req[i] for i in layers) <= Mem[j] + 1e-12
+        stage = sum(t_comp[i][j] for i in layers)
+        if q:
+            stage = max(stage, O[layers[0] - 1] / Bw[order[q - 1]][j])
+        worst = max(worst, stage)
+    assert abs(worst - t) < 1e-9 * max(1.0, t)
+
+
+def test_low_bandwidth_keeps_everything_on_the_source(B):
+    # the paper's observation: at 1 Mbps to the cloud the best plan degenerates to local execution
+    N, M = 6, 2
+    t_comp = [[1.0, 0.05] for _ in range(N)]
+    O, Req, Mem = [1.0] * N, [1.0] * N, [100.0, 100.0]
+    slow = [[0, 1e-3], [1e-3, 0]]
+    a, t = B.es_partition_latency(t_comp, O, Req, Mem, slow)
+    assert a == [0] * N and abs(t - N) < 1e-12
+    fast = [[0, 1e3], [1e3, 0]]
+    a, t = B.es_partition_latency(t_comp, O, Req, Mem, fast)
+    assert a == [0] + [1] * (N - 1)
+    a, t = B.es_partition_throughput(t_comp, O, Req, Mem, fast)
+    assert a[0] == 0 and 1 in a and t < N
+
+
+def test_planner_argument_errors(B):
+    with pytest.raises(B.EsError) as e:
+        B.es_partition_latency([[1.0, 1.0]], [1.0], [5.0], [1.0, 1.0], [[0, 1], [1, 0]])     # layer 0 too big for device 0
+    assert e.value.status == 3
+    with pytest.raises(B.EsError) as e:
+        B.es_partition_throughput([[1.0]], [1.0, 2.0], [1.0], [1.0], [[0.0]])
+    assert e.value.status == 2

@@ -241,6 +241,33 @@ def test_profile_reports_every_layer(B, tiny):
     sh.close()
 
 
+def test_profile_feeds_the_partition_planners(B, tiny):
+    """The per-layer profile is the planners' input: measured times for this GPU plus two synthetic slower
+    devices (scaled times), activation and memory sizes from the profile."""
+    wd, _ = tiny
+    ids = prompt_ids(0, 1, 16, TINY.vocab).cuda()
+    sh = B.Shard(TINY, 0, 2, wd, max_slots=1, max_seq=32, max_tokens=16)
+    sh.es_shard_set_profiling(True)
+    sh.es_shard_prefill(ids, None, 1, 16, [0])
+    n = sh.es_shard_handoff()[2]
+    for _ in range(4):
+        sh.es_shard_decode_step(n, None, 1, [0])
+    prof = sh.es_layer_profile()
+    sh.close()
+    scale = [1.0, 5.0, 20.0]                                   # device 0 is the source node (a slow one here)
+    order = [2, 0, 1]                                          # so that the fast GPU is not the source
+    t_comp = [[p["avg_ms_per_token"] * scale[order[j]] for j in range(3)] for p in prof]
+    O = [p["activation_bytes"] for p in prof]
+    Req = [p["weight_bytes"] + p["kv_bytes"] for p in prof]
+    Mem = [sum(Req)] * 3
+    Bw = [[0 if a == b else 1e9 for b in range(3)] for a in range(3)]
+    a, t = B.es_partition_latency(t_comp, O, Req, Mem, Bw)
+    assert a[0] == 0 and len(a) == len(prof) and t > 0
+    assert a[1:] == [1] * (len(prof) - 1)                      # with fast links the work moves to the fast device
+    a2, t2 = B.es_partition_throughput(t_comp, O, Req, Mem, Bw)
+    assert a2[0] == 0 and t2 <= max(sum(r) for r in zip(*t_comp))
+
+
 def test_error_paths_launch_nothing(B, tiny):
     wd, _ = tiny
     ids = prompt_ids(0, 1, 8, TINY.vocab).cuda()
