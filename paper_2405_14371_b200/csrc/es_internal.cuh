@@ -29,11 +29,9 @@ es_status_t fail(es_status_t st, const char* fmt, ...);
 
 // ---- tuning knobs (read once from the environment; defaults are the measured best) -----------
 struct Tunables {
-  int stream_prefetch_row_bytes;   // ES_STREAM_PREFETCH: bytes of each first row pair prefetched into L2 before the dependency wait
-  int stream_ctas_per_sm;          // ES_STREAM_CTAS: cap on resident CTAs per SM of the weight-streaming kernel (0 = occupancy limit)
-  int stream_deep;                 // ES_STREAM_DEEP: -1 auto, 0 never, 1 always use the deeper (U = 4) chunking
-  int tc_pair;                     // ES_TC_PAIR: CTA-pair tensor-core kernel for large prefill products (1) or never (0)
-  int pdl;                         // ES_PDL: programmatic dependent launch in decode steps (1) or plain stream order (0)
+  int stream_deep;   // ES_STREAM_DEEP: weight-streaming kernel chunk depth, 1 = 4 KB per warp per buffer (default), 0 = 2 KB
+  int tc_pair;       // ES_TC_PAIR: CTA-pair tensor-core kernel for large prefill products (1, default) or never (0)
+  int pdl;           // ES_PDL: programmatic dependent launch in decode steps (1, default) or plain stream order (0)
 };
 const Tunables& tunables();
 
@@ -57,7 +55,6 @@ struct LinearParams {
   const __half* A;
   int64_t lda;
   // optional fused RMSNorm (weight-streaming kernel, M <= 2): A = rmsnorm(norm_x rows; norm_gain)
-  int prefetch_row_bytes;  // weight-streaming kernel: L2 prefetch per first row (0 = none)
   const float* norm_x;     // fp32 [M, K], row stride norm_ldx; nullptr = read A
   int64_t norm_ldx;
   const __half* norm_gain;

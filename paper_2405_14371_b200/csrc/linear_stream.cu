@@ -31,12 +31,6 @@ __device__ __forceinline__ uint4 ld_stream(const void* ptr) {
   return v;
 }
 
-// Asks for `bytes` (a multiple of 16) starting at ptr to be brought into L2; no register or
-// shared-memory destination, nothing to wait for.
-__device__ __forceinline__ void prefetch_l2(const void* ptr, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ptr), "r"(bytes) : "memory");
-}
-
 // acc += w * a over 8 fp16 pairs, each product formed exactly and added in fp32 by the
 // mixed-precision FMA (fp16 x fp16 + fp32), so no conversion instructions are spent.
 __device__ __forceinline__ void fma8(float& acc, const uint4& w, const uint4& a) {
@@ -111,16 +105,7 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
 
   uint4 b0w0[U], b0w1[U], b1w0[U], b1w1[U];
   if (total > 0) {
-    // Requested while the previous kernel drains: the first chunk into registers, and the next few
-    // KB of both rows into L2 so that HBM keeps working while this CTA stages its activations.
-    if (lane == 0 && p.prefetch_row_bytes > 0) {
-      const int done = CHUNK_K * 2;                         // bytes of each row covered by the first chunk
-      const int more = min(K * 2 - done, p.prefetch_row_bytes);
-      if (more > 0) {
-        prefetch_l2(reinterpret_cast<const unsigned char*>(nr0) + done, (uint32_t)more);
-        prefetch_l2(reinterpret_cast<const unsigned char*>(nr1) + done, (uint32_t)more);
-      }
-    }
+    // requested while the previous kernel drains
     issue(b0w0, b0w1);
     if (total > 1) issue(b1w0, b1w1);        // both buffers on their way: HBM stays busy while activations are staged
   }
@@ -249,7 +234,6 @@ es_status_t launch_inst(const LinearParams& p, cudaStream_t s, bool pdl) {
   ES_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, THREADS, smem));
   if (per_sm < 1) return fail(ES_ERR_SHAPE, "weight-streaming kernel does not fit (K = %d, %d rows)", p.K, p.M);
   const int n_units = (EPI == EPI_SWIGLU) ? p.N : (p.N + 1) / 2;
-  if (tunables().stream_ctas_per_sm > 0 && per_sm > tunables().stream_ctas_per_sm) per_sm = tunables().stream_ctas_per_sm;
   int grid = sms * per_sm;
   const int max_useful = (n_units + WARPS - 1) / WARPS;
   if (grid > max_useful) grid = max_useful;
@@ -263,8 +247,8 @@ es_status_t launch_mb(const LinearParams& p, cudaStream_t s, bool pdl) {
   const int n_units = (EPI == EPI_SWIGLU) ? p.N : (p.N + 1) / 2;
   if (MB <= 2) {
     if (a_bytes > 200 * 1024) return fail(ES_ERR_SHAPE, "K = %d too large for the weight-streaming kernel", p.K);
-    bool deep = true;                           // measured: 4 KB per warp per buffer beats 2 KB at every layer shape
-    if (tunables().stream_deep >= 0) deep = tunables().stream_deep != 0;
+    // 4 KB per warp per buffer (U = 4) beat 2 KB at every layer shape measured; U = 2 is kept for ES_STREAM_DEEP=0
+    const bool deep = tunables().stream_deep != 0;
     if (p.norm_x) return deep ? launch_inst<MB, EPI, true, 4, true>(p, s, pdl) : launch_inst<MB, EPI, true, 2, true>(p, s, pdl);
     return deep ? launch_inst<MB, EPI, false, 4, true>(p, s, pdl) : launch_inst<MB, EPI, false, 2, true>(p, s, pdl);
   }
@@ -286,9 +270,7 @@ es_status_t launch_epi(const LinearParams& p, cudaStream_t s, bool pdl) {
 
 bool linear_stream_can_fuse_norm(int M) { return M <= 2; }
 
-es_status_t launch_linear_stream(const LinearParams& p_in, int epi, cudaStream_t s, int64_t* launches, bool pdl) {
-  LinearParams p = p_in;
-  p.prefetch_row_bytes = tunables().stream_prefetch_row_bytes & ~15;
+es_status_t launch_linear_stream(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl) {
   if (p.M <= 0 || p.N <= 0) return ES_OK;
   if (p.M > 16) return fail(ES_ERR_UNSUPPORTED, "weight-streaming kernel takes at most 16 rows, got %d", p.M);
   if (p.K % 8 != 0) return fail(ES_ERR_SHAPE, "K = %d is not a multiple of 8", p.K);

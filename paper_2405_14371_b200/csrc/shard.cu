@@ -40,8 +40,7 @@ static int env_int(const char* name, int dflt) {
 }
 
 const Tunables& tunables() {
-  static const Tunables t = {env_int("ES_STREAM_PREFETCH", 0), env_int("ES_STREAM_CTAS", 0), env_int("ES_STREAM_DEEP", -1),
-                             env_int("ES_TC_PAIR", 1), env_int("ES_PDL", 1)};
+  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_PDL", 1)};
   return t;
 }
 
