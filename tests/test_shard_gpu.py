@@ -241,6 +241,38 @@ def test_profile_reports_every_layer(B, tiny):
     sh.close()
 
 
+@pytest.mark.parametrize("Bn,T,P", [(1, 1, 64), (16, 3, 16), (5, 70, 64), (2, 129, 64), (16, 17, 64)])
+def test_edge_shapes_match_oracle(B, tiny, Bn, T, P):
+    """One-token prompts, the largest batch, prompts that straddle KV pages and attention tiles, both page
+    sizes (64: tensor-core attention, 16: CUDA-core attention); decode runs until the slot is exactly full."""
+    wd, wh = tiny
+    S = 3
+    ids = prompt_ids(0, Bn, T, TINY.vocab, seed=21)
+    nxt = forced_decode_ids(0, Bn, S, TINY.vocab, seed=21)
+    sh = B.Shard(TINY, 0, 2, wd, max_slots=Bn, max_seq=T + S, max_tokens=Bn * T, kv_page_tokens=P)
+    slots = list(reversed(range(Bn)))
+    sh.es_shard_prefill(ids.cuda(), None, Bn, T, slots)
+    h, l, _ = sh.es_shard_handoff()
+    hs, ls = [h.clone()], [l.clone()]
+    for s_ in range(S):
+        sh.es_shard_decode_step(nxt[s_].cuda(), None, Bn, slots)
+        h, l, _ = sh.es_shard_handoff()
+        hs.append(h.clone()); ls.append(l.clone())
+    with pytest.raises(B.EsError) as e:
+        sh.es_shard_decode_step(nxt[0].cuda(), None, Bn, slots)          # every slot is at max_seq now
+    assert e.value.status == 5
+    sh.es_shard_device_status()
+    sh.close()
+    for b in sorted({0, Bn // 2, Bn - 1}):
+        seq = torch.cat([ids[b], nxt[:, b]])
+        want_h, _ = O.shard_forward_full(TINY, wh, 0, 2, ids=seq)
+        assert rel_err(hs[0][b], want_h[:T]) < TOL
+        for s_ in range(S):
+            assert rel_err(hs[1 + s_][b, 0], want_h[T + s_]) < TOL
+        _, want_l = O.shard_forward_full(TINY, wh, 0, 2, ids=seq[:T + S])
+        assert rel_err(ls[S][b], want_l) < TOL
+
+
 def test_profile_feeds_the_partition_planners(B, tiny):
     """The per-layer profile is the planners' input: measured times for this GPU plus two synthetic slower
     devices (scaled times), activation and memory sizes from the profile."""
