@@ -233,6 +233,20 @@ ES_API es_status_t es_op_rmsnorm(const float *x, const void *gain, void *y, int3
 ES_API es_status_t es_op_linear(const void *A, const void *W, const float *R, float *C, int32_t M, int32_t N,
                          int32_t K, int32_t path, void *stream);
 
+/* The tensor-core product with its K range cut into k_splits slices (Sec. "Experimental Setup" runs
+ * short prompts, for which a d_model-wide product has too few output tiles to fill the machine):
+ * C[M, N] = A[M, K] * W[N, K]^T (+ R), fp16 in, fp32 out, all device pointers, row-major, dense.
+ * Every (tile, slice) pair is computed by its own CTA into `workspace` ([k_splits, M, N] fp32,
+ * device, 16-byte aligned, at least es_op_linear_splitk_workspace_bytes bytes); a second kernel adds
+ * the slices in ascending order and the residual, so the result does not depend on scheduling.
+ * k_splits = 0 lets the library choose (1 = no split, no workspace needed).  Slices must not be
+ * empty: (k_splits - 1) * ceil(ceil(K / 64) / k_splits) < ceil(K / 64), else ES_ERR_INVALID_ARG.
+ * N must be a multiple of 4, K of 8.  R may be NULL and may alias C. */
+ES_API size_t es_op_linear_splitk_workspace_bytes(int32_t M, int32_t N, int32_t k_splits);
+ES_API es_status_t es_op_linear_splitk(const void *A, const void *W, const float *R, float *C, int32_t M, int32_t N,
+                                       int32_t K, int32_t k_splits, void *workspace, size_t workspace_bytes,
+                                       void *stream);
+
 /* Causal self-attention over a prompt.  q fp16 [B, T, Hq, hd] (already rotated); k, v fp16
  * [B, T, Hkv, hd]; out fp16 [B, T, Hq*hd].  Query t sees keys 0..t; scale 1/sqrt(hd).
  * path: 0 = automatic, 1 = tensor-core (tcgen05) kernel, 2 = CUDA-core kernel. */

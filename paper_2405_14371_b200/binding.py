@@ -88,6 +88,8 @@ def _load() -> C.CDLL:
         "es_partition_throughput": (i32, [i32, i32] + [P(C.c_double)] * 5 + [P(i32), P(C.c_double)]),
         "es_op_rmsnorm": (i32, [vp, vp, vp, i32, i32, C.c_float, vp]),
         "es_op_linear": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, vp]),
+        "es_op_linear_splitk_workspace_bytes": (sz, [i32, i32, i32]),
+        "es_op_linear_splitk": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, vp, sz, vp]),
         "es_op_prefill_attention": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]),
         "es_op_decode_attention_scratch_bytes": (sz, [i32, i32, i32, i32, i32]),
         "es_op_decode_attention": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp]),
@@ -105,7 +107,7 @@ lib = _load()
 EXPORTS = ("es_shard_workspace_bytes es_shard_create es_shard_prefill es_shard_decode_step es_shard_handoff "
            "es_layer_profile es_shard_set_profiling es_shard_reset_slots es_shard_set_page_table es_shard_set_graphs "
            "es_partition_latency es_partition_throughput es_shard_device_status es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_kernel_timing_detail es_shard_destroy es_last_error es_version es_op_rmsnorm "
-           "es_op_linear es_op_prefill_attention es_op_decode_attention_scratch_bytes es_op_decode_attention "
+           "es_op_linear es_op_linear_splitk_workspace_bytes es_op_linear_splitk es_op_prefill_attention es_op_decode_attention_scratch_bytes es_op_decode_attention "
            "es_op_decode_attention_static_capacity es_op_decode_attention_static").split()
 
 
@@ -306,6 +308,23 @@ def es_op_linear(A: torch.Tensor, W: torch.Tensor, R: Optional[torch.Tensor] = N
     N = W.shape[0]
     Cout = torch.empty(M, N, dtype=torch.float32, device=A.device)
     _check(lib.es_op_linear(_ptr(A), _ptr(W), _ptr(R), _ptr(Cout), M, N, K, path, _stream_ptr(stream)))
+    return Cout
+
+
+def es_op_linear_splitk_workspace_bytes(M: int, N: int, k_splits: int) -> int:
+    return int(lib.es_op_linear_splitk_workspace_bytes(M, N, k_splits))
+
+
+def es_op_linear_splitk(A: torch.Tensor, W: torch.Tensor, R: Optional[torch.Tensor] = None, k_splits: int = 0,
+                        workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    M, K = A.shape
+    N = W.shape[0]
+    Cout = torch.empty(M, N, dtype=torch.float32, device=A.device)
+    if workspace is None:
+        workspace = torch.empty(max(1, es_op_linear_splitk_workspace_bytes(M, N, max(k_splits, 8))), dtype=torch.uint8,
+                                device=A.device)
+    _check(lib.es_op_linear_splitk(_ptr(A), _ptr(W), _ptr(R), _ptr(Cout), M, N, K, k_splits, _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _stream_ptr(stream)))
     return Cout
 
 

@@ -92,10 +92,10 @@ __global__ void __launch_bounds__(PWARPS * 32) prefill_attn_simt_kernel(const Pr
 
 }  // namespace
 
-es_status_t launch_prefill_attention(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches, int path) {
+es_status_t launch_prefill_attention(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches, int path, bool pdl) {
   if (p.B <= 0 || p.T <= 0) return ES_OK;
   if (path == 0) path = prefill_attention_tc_supported(p) ? 1 : 2;
-  if (path == 1) return launch_prefill_attention_tc(p, s, launches);
+  if (path == 1) return launch_prefill_attention_tc(p, s, launches, pdl);
   if (path == 2) return launch_prefill_attention_simt(p, s, launches);
   return fail(ES_ERR_INVALID_ARG, "unknown attention path %d", path);
 }

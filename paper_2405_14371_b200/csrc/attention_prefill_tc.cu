@@ -16,6 +16,7 @@
 #include <string.h>
 
 #include "es_internal.cuh"
+#include "launch.cuh"
 #include "sm100.cuh"
 
 namespace es {
@@ -56,6 +57,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 1)
 prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) {
   using L = AttnSmem<HD>;
   constexpr int HALVES = L::HALVES;
+  pdl_launch_dependents();
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* q_s = smem;                                   // [HALVES][128 rows][128 B]
@@ -98,6 +100,7 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                   // set-up above overlaps the previous kernel's tail
   const uint32_t tmem_s = tmem_base;            // columns [0, 64)
   const uint32_t tmem_o = tmem_base + 64;       // columns [64, 64 + HD)
 
@@ -277,7 +280,7 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
 bool is_paged(const PrefillAttnParams& p) { return p.kv.block_table != nullptr; }
 
 template <int HD>
-es_status_t launch_hd(const AttnMaps& maps, const PrefillAttnParams& p, cudaStream_t s) {
+es_status_t launch_hd(const AttnMaps& maps, const PrefillAttnParams& p, cudaStream_t s, bool pdl) {
   auto kern = prefill_attn_tc_kernel<HD>;
   static bool configured = false;
   if (!configured) {
@@ -295,8 +298,7 @@ es_status_t launch_hd(const AttnMaps& maps, const PrefillAttnParams& p, cudaStre
   a.pages_per_slot = p.kv.pages_per_slot;
   a.scale_log2e = 1.4426950408889634f / sqrtf((float)HD);
   const dim3 grid((p.T + QT - 1) / QT, p.Hq, p.B);
-  kern<<<grid, ATT_THREADS, AttnSmem<HD>::TOTAL, s>>>(maps, a);
-  ES_CUDA_CHECK(cudaGetLastError());
+  ES_CUDA_CHECK(launch_kernel(kern, grid, dim3(ATT_THREADS), AttnSmem<HD>::TOTAL, s, pdl, maps, a));
   return ES_OK;
 }
 
@@ -328,7 +330,7 @@ es_status_t prefill_attention_tc_build_maps(const PrefillAttnParams& p, int64_t 
   return ES_OK;
 }
 
-es_status_t launch_prefill_attention_tc(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches) {
+es_status_t launch_prefill_attention_tc(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches, bool pdl) {
   if (p.B <= 0 || p.T <= 0) return ES_OK;
   if (!prefill_attention_tc_supported(p)) return fail(ES_ERR_UNSUPPORTED, "tensor-core attention does not take this layout");
   TcMaps local;
@@ -338,7 +340,7 @@ es_status_t launch_prefill_attention_tc(const PrefillAttnParams& p, cudaStream_t
     maps = &local;
   }
   const AttnMaps& m = *reinterpret_cast<const AttnMaps*>(maps);
-  es_status_t st = (p.hd == 128) ? launch_hd<128>(m, p, s) : launch_hd<64>(m, p, s);
+  es_status_t st = (p.hd == 128) ? launch_hd<128>(m, p, s, pdl) : launch_hd<64>(m, p, s, pdl);
   if (st == ES_OK && launches) ++*launches;
   return st;
 }

@@ -90,6 +90,68 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const float* __res
   }
 }
 
+// Finishes a split-K product: out[r, :] = (res ? res[r, :] : 0) + part[0, r, :] + part[1, r, :] + ...
+// (slices in ascending order, so the sum does not depend on scheduling) and, with a gain vector, the
+// RMSNorm of the finished row in fp16 for the next product — one CTA per row, the row kept in
+// registers between the two passes like rmsnorm_kernel does.
+__global__ void __launch_bounds__(RMS_THREADS) splitk_reduce_kernel(const float* __restrict__ part, int k_splits,
+                                                                    const float* res, float* out, int M, int N,
+                                                                    int64_t ldo, const __half* __restrict__ gain,
+                                                                    __half* __restrict__ y, float eps) {
+  __shared__ float red[32];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r = blockIdx.x;
+  const int n4 = N / 4;
+  const int64_t slice = (int64_t)M * N;
+  const float4* src = reinterpret_cast<const float4*>(part + (int64_t)r * N);
+  const float4* rs = res ? reinterpret_cast<const float4*>(res + (int64_t)r * ldo) : nullptr;
+  float4* dst = reinterpret_cast<float4*>(out + (int64_t)r * ldo);
+  auto finish = [&](int c) {
+    float4 a = rs ? rs[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < k_splits; ++s) {
+      const float4 v = __ldcs(src + (s * slice) / 4 + c);
+      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    }
+    dst[c] = a;
+    return a;
+  };
+  float4 v[RMS_REGS];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < RMS_REGS; ++i) {
+    const int c = threadIdx.x + i * RMS_THREADS;
+    if (c < n4) {
+      v[i] = finish(c);
+      ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+    }
+  }
+  for (int c = threadIdx.x + RMS_REGS * RMS_THREADS; c < n4; c += RMS_THREADS) {
+    const float4 t = finish(c);
+    ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+  }
+  if (gain == nullptr) return;                       // uniform over the CTA
+  const float total = block_sum(ss, red);
+  const float inv = 1.0f / sqrtf(total / (float)N + eps);
+  __half2* yd = reinterpret_cast<__half2*>(y + (int64_t)r * N);
+  const __half2* g2 = reinterpret_cast<const __half2*>(gain);
+#pragma unroll
+  for (int i = 0; i < RMS_REGS; ++i) {
+    const int c = threadIdx.x + i * RMS_THREADS;
+    if (c < n4) {
+      const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
+      yd[2 * c] = __floats2half2_rn(v[i].x * inv * ga.x, v[i].y * inv * ga.y);
+      yd[2 * c + 1] = __floats2half2_rn(v[i].z * inv * gb.x, v[i].w * inv * gb.y);
+    }
+  }
+  for (int c = threadIdx.x + RMS_REGS * RMS_THREADS; c < n4; c += RMS_THREADS) {
+    const float4 t = dst[c];                         // written by this thread above
+    const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
+    yd[2 * c] = __floats2half2_rn(t.x * inv * ga.x, t.y * inv * ga.y);
+    yd[2 * c + 1] = __floats2half2_rn(t.z * inv * gb.x, t.w * inv * gb.y);
+  }
+}
+
 // Greedy token: index of the largest logit, the lowest index on ties.  One CTA per sequence.
 __global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ logits, int* __restrict__ out, int V) {
   __shared__ float bv[8];
@@ -157,6 +219,15 @@ es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M,
 es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches, bool pdl) {
   if (B <= 0) return ES_OK;
   ES_CUDA_CHECK(launch_kernel(argmax_kernel, dim3(B), dim3(256), 0, s, pdl, logits, out, V));
+  if (launches) ++*launches;
+  return ES_OK;
+}
+
+es_status_t launch_splitk_reduce(const float* part, int k_splits, const float* res, float* out, int M, int N, int64_t ldo,
+                                 const __half* gain, __half* y, float eps, cudaStream_t s, int64_t* launches, bool pdl) {
+  if (M <= 0 || N <= 0) return ES_OK;
+  if (N % 4 != 0 || ldo % 4 != 0) return fail(ES_ERR_SHAPE, "split-K reduction needs N and the row stride to be multiples of 4");
+  ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel, dim3(M), dim3(RMS_THREADS), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps));
   if (launches) ++*launches;
   return ES_OK;
 }

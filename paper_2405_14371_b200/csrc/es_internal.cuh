@@ -32,6 +32,7 @@ struct Tunables {
   int stream_deep;   // ES_STREAM_DEEP: weight-streaming kernel chunk depth, 1 = 4 KB per warp per buffer (default), 0 = 2 KB
   int tc_pair;       // ES_TC_PAIR: CTA-pair tensor-core kernel for large prefill products (1, default) or never (0)
   int pdl;           // ES_PDL: programmatic dependent launch in decode steps (1, default) or plain stream order (0)
+  int split_k;       // ES_SPLIT_K: split-K for the O and down projections of short prefills (1, default) or never (0)
 };
 const Tunables& tunables();
 
@@ -79,6 +80,10 @@ struct LinearParams {
   int T;                   // rows per sequence: row m belongs to sequence m / T at prompt offset m % T
   int is_decode;           // position = ctx_len[slot] instead of m % T
   int Hq, Hkv, hd, P, pages_per_slot, max_seq;
+  // split-K (tensor-core kernel, EPI_F32 only): > 1 = raw partial sums go to part[k_splits, M, N] instead
+  // of out_f32; launch_splitk_reduce finishes the product
+  int k_splits;
+  float* part;
 };
 
 // Kernel families.  Each returns after enqueuing; `launches` is incremented per kernel launched.
@@ -88,11 +93,19 @@ bool linear_stream_can_fuse_norm(int M);
 // tensor-core (mma.sync) variant of the weight-streaming kernel for 3..16 rows
 bool linear_stream_mma_supported(const LinearParams& p, int epi);
 es_status_t launch_linear_stream_mma(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl = false);
-es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word);
+es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word, bool pdl = false);
 bool linear_tc_supported(const LinearParams& p, int epi);
+// number of K slices the tensor-core kernel should use for this product (1 = do not split), and the
+// workspace that covers any product for which the answer is > 1
+int linear_tc_splits(const LinearParams& p, int epi);
+size_t linear_tc_split_workspace_bytes();
+// out[m, :] = (res ? res[m, :] : 0) + sum over slices (ascending) of part[s, m, :]; with gain != nullptr also
+// y[m, :] = rmsnorm(out[m, :]) * gain in fp16.  N % 4 == 0.  res may alias out.
+es_status_t launch_splitk_reduce(const float* part, int k_splits, const float* res, float* out, int M, int N, int64_t ldo,
+                                 const __half* gain, __half* y, float eps, cudaStream_t s, int64_t* launches, bool pdl = false);
 // CTA-pair (cta_group::2) variant for large M; uses the same tensor maps
 bool linear_tc2_supported(const LinearParams& p, int epi);
-es_status_t launch_linear_tc2(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word);
+es_status_t launch_linear_tc2(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word, bool pdl = false);
 // Encodes the tensor maps for p's operands; the A map covers a_rows rows (the buffer's capacity).
 es_status_t tc_build_maps(const LinearParams& p, int epi, int64_t a_rows, TcMaps* out);
 
@@ -143,11 +156,11 @@ struct PrefillAttnParams {
   int* status;
 };
 // path: 0 = automatic, 1 = tensor-core (tcgen05) kernel, 2 = CUDA-core kernel
-es_status_t launch_prefill_attention(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches, int path = 0);
+es_status_t launch_prefill_attention(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches, int path = 0, bool pdl = false);
 es_status_t launch_prefill_attention_simt(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches);
 bool prefill_attention_tc_supported(const PrefillAttnParams& p);
 es_status_t prefill_attention_tc_build_maps(const PrefillAttnParams& p, int64_t q_rows, TcMaps* out);
-es_status_t launch_prefill_attention_tc(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches);
+es_status_t launch_prefill_attention_tc(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches, bool pdl = false);
 
 struct DecodeAttnParams {
   const __half* q;   // [B, Hq, hd]

@@ -7,12 +7,19 @@
 // accumulator and releases each stage with tcgen05.commit; four epilogue warps read the
 // accumulator back with tcgen05.ld (each warp its own 32-lane quarter) and run the epilogue.
 // Ragged M, N and K are handled by TMA zero fill on the way in and by guards on the way out.
+// Split-K (plain / residual epilogue only): when a product has too few output tiles for the machine
+// (short prompts: M = 128..512 against N = d_model), the K range is cut into k_splits slices, every
+// (tile, slice) pair is a work item, and the raw fp32 accumulators go to a workspace
+// [k_splits, M, N]; a reduction kernel adds the slices in slice order (and the residual) afterwards.
+// That cuts what a CTA must pull through L2 for its tile from 128 + BN rows of K elements to
+// (128 + BN) / k_splits, which is what bounds these launches.
 // Every wait is bounded: if a barrier does not flip within about a second the CTA records an
 // error code in the status word and leaves through the normal teardown (TMEM freed).
 #include <cuda.h>
 #include <string.h>
 
 #include "epilogue.cuh"
+#include "launch.cuh"
 #include "sm100.cuh"
 
 namespace es {
@@ -37,6 +44,20 @@ struct TmapSet {
 };
 static_assert(sizeof(TmapSet) == sizeof(TcMaps), "TcMaps must hold four tensor maps");
 
+// Raw accumulator columns [n, n + 32) of one row into the split-K workspace row `row` (N % 4 == 0).
+__device__ __forceinline__ void partial_chunk32(float* row, bool row_valid, int n, int N, const float (&v)[32]) {
+  if (!row_valid || n >= N) return;
+  if (n + 32 <= N) {
+    float4* dst = reinterpret_cast<float4*>(row + n);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (n + j < N) row[n + j] = v[j];
+  }
+}
+
 // ---- the kernel --------------------------------------------------------------------------------
 // Persistent: a CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The accumulator is double
 // buffered in TMEM, so the epilogue of one tile runs while the tensor cores work on the next.
@@ -48,6 +69,7 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
   constexpr int BN_OUT = (EPI == EPI_SWIGLU) ? BN / 2 : BN;   // output columns per tile
   constexpr int ACC_COLS = Cfg::TMEM_COLS;                    // TMEM columns of one accumulator buffer
 
+  pdl_launch_dependents();
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* a_tiles = smem;
@@ -61,8 +83,11 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int num_tiles = m_tiles * n_tiles;
+  const int k_splits = (EPI == EPI_F32 && p.k_splits > 1) ? p.k_splits : 1;
+  const int mn_tiles = m_tiles * n_tiles;
+  const int num_tiles = mn_tiles * k_splits;        // work items: slice-major, so concurrent CTAs share a K slice of A
   const int num_kb = (p.K + BK - 1) / BK;
+  const int kb_per = (num_kb + k_splits - 1) / k_splits;
 
   // tile order: groups of up to 16 row tiles share each column tile while it is hot in L2
   auto tile_origin = [&](int tile, int& m0, int& n0) {
@@ -93,6 +118,9 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // barriers, tensor-map prefetch and the TMEM allocation above overlap the previous kernel's tail;
+  // nothing below reads or writes global memory before the previous kernel has completed
+  pdl_wait();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -104,7 +132,9 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m0, n0;
-        tile_origin(tile, m0, n0);
+        const int ks = tile / mn_tiles;
+        tile_origin(tile - ks * mn_tiles, m0, n0);
+        const int kb0 = ks * kb_per, kb1 = min(num_kb, kb0 + kb_per);
         const CUtensorMap* wmap[N_LOADS];
         int wrow[N_LOADS];
         if (EPI == EPI_SWIGLU) {
@@ -120,7 +150,7 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
 #pragma unroll
           for (int i = 0; i < N_LOADS; ++i) { wmap[i] = &maps.w[seg]; wrow[i] = n + i * W_BOX_ROWS; }
         }
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, abort_flag, status, 1)) { ok = false; break; }
@@ -147,7 +177,9 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
         if (!ok) break;
         tc_fence_after();
         const uint32_t tacc = tmem_base + (uint32_t)(buf * ACC_COLS);
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        const int ks = tile / mn_tiles;
+        const int kb0 = ks * kb_per, kb1 = min(num_kb, kb0 + kb_per);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           ok = mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag, status, 2);
@@ -158,7 +190,7 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)
             umma_f16(tacc, umma_desc_sw128(a0 + k * UMMA_K * 2), umma_desc_sw128(b0 + k * UMMA_K * 2), idesc,
-                     (kb > 0 || k > 0) ? 1u : 0u);
+                     (kb > kb0 || k > 0) ? 1u : 0u);
           umma_commit(smem_u32(&empty_bar[s]));      // frees the stage once these MMAs have read it
         }
         if (ok) umma_commit(smem_u32(&acc_full[buf]));   // accumulator complete
@@ -174,7 +206,8 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
       if (!mbar_wait(smem_u32(&acc_full[buf]), use & 1, abort_flag, status, 3)) break;
       tc_fence_after();
       int m0, n0;
-      tile_origin(tile, m0, n0);
+      const int ks = tile / mn_tiles;
+      tile_origin(tile - ks * mn_tiles, m0, n0);
       const int m = m0 + quarter * 32 + lane;
       const uint32_t trow = tmem_base + (uint32_t)(buf * ACC_COLS) + ((uint32_t)(quarter * 32) << 16);
       if (EPI == EPI_SWIGLU) {
@@ -190,8 +223,12 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
         for (int c = 0; c < BN; c += 32) {
           float v[32];
           tmem_ld32(trow + c, v);
-          if (EPI == EPI_F32) epi_f32_chunk32(p, m, n0 + c, v);
-          else epi_qkv_chunk32(p, m, n0 + c, v);
+          if (EPI == EPI_F32) {
+            if (k_splits > 1) partial_chunk32(p.part + ((int64_t)ks * p.M + m) * p.N, m < p.M, n0 + c, p.N, v);
+            else epi_f32_chunk32(p, m, n0 + c, v);
+          } else {
+            epi_qkv_chunk32(p, m, n0 + c, v);
+          }
         }
       }
       // this warp has read its quarter of the buffer: hand it back to the MMA issuer
@@ -236,6 +273,7 @@ es_status_t encode_2d(CUtensorMap* map, const void* base, int64_t rows, int64_t 
 }
 
 int pick_bn(const LinearParams& p, int epi) {
+  if (epi == EPI_F32 && p.k_splits > 1) return 256;
   // Every CTA pulls a 128-row slice of A and a bn-row slice of W through L2 for the whole K range,
   // one CTA per SM at a time, so the time goes as (waves of CTAs) x (128 + bn).  Take the width
   // that minimises it (the wider one on ties); QKV segments must be whole tiles.
@@ -258,7 +296,7 @@ int pick_bn(const LinearParams& p, int epi) {
 }
 
 template <int EPI, int BN>
-es_status_t launch_bn(const TmapSet& maps, const LinearParams& p, int* status, cudaStream_t s) {
+es_status_t launch_bn(const TmapSet& maps, const LinearParams& p, int* status, cudaStream_t s, bool pdl) {
   constexpr int out = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
   const int m_tiles = (p.M + BM - 1) / BM, n_tiles = (p.N + out - 1) / out;
   auto kern = linear_tc_kernel<EPI, BN>;
@@ -273,19 +311,19 @@ es_status_t launch_bn(const TmapSet& maps, const LinearParams& p, int* status, c
     ES_CUDA_CHECK(cudaGetDevice(&dev));
     ES_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   }
-  const int tiles = m_tiles * n_tiles;
-  kern<<<tiles < sms ? tiles : sms, TC_THREADS, TileCfg<BN>::SMEM, s>>>(maps, p, status, m_tiles, n_tiles);
-  ES_CUDA_CHECK(cudaGetLastError());
+  const int tiles = m_tiles * n_tiles * ((EPI == EPI_F32 && p.k_splits > 1) ? p.k_splits : 1);
+  ES_CUDA_CHECK(launch_kernel(kern, dim3(tiles < sms ? tiles : sms), dim3(TC_THREADS), TileCfg<BN>::SMEM, s, pdl, maps, p, status,
+                              m_tiles, n_tiles));
   return ES_OK;
 }
 
 template <int EPI>
-es_status_t launch_epi(const TmapSet& maps, const LinearParams& p, int bn, int* status, cudaStream_t s) {
+es_status_t launch_epi(const TmapSet& maps, const LinearParams& p, int bn, int* status, cudaStream_t s, bool pdl) {
   switch (bn) {
-    case 256: return launch_bn<EPI, 256>(maps, p, status, s);
-    case 128: return launch_bn<EPI, 128>(maps, p, status, s);
-    case 64: return launch_bn<EPI, 64>(maps, p, status, s);
-    case 32: return launch_bn<EPI, 32>(maps, p, status, s);
+    case 256: return launch_bn<EPI, 256>(maps, p, status, s, pdl);
+    case 128: return launch_bn<EPI, 128>(maps, p, status, s, pdl);
+    case 64: return launch_bn<EPI, 64>(maps, p, status, s, pdl);
+    case 32: return launch_bn<EPI, 32>(maps, p, status, s, pdl);
   }
   return fail(ES_ERR_UNSUPPORTED, "no tile width for this shape");
 }
@@ -308,6 +346,22 @@ es_status_t tma_encode_2d_f16(void* map, const void* base, int64_t rows, int64_t
   return ES_OK;
 }
 
+int linear_tc_splits(const LinearParams& p, int epi) {
+  // Worth it when 256-wide tiles over the whole K range would leave at least half of the SMs idle;
+  // every slice keeps at least four 64-element K blocks.
+  if (epi != EPI_F32 || p.M <= 16 || p.N % 4 != 0) return 1;
+  const int tiles = ((p.M + BM - 1) / BM) * ((p.N + 255) / 256);
+  const int num_kb = (p.K + BK - 1) / BK;
+  int s = 148 / tiles;
+  if (s > 8) s = 8;
+  if (s > num_kb / 4) s = num_kb / 4;
+  if (s < 2) return 1;
+  const int kb_per = (num_kb + s - 1) / s;
+  return (num_kb + kb_per - 1) / kb_per;       // no empty slice
+}
+
+size_t linear_tc_split_workspace_bytes() { return (size_t)148 * BM * 256 * sizeof(float); }
+
 bool linear_tc_supported(const LinearParams& p, int epi) {
   if (p.M <= 0 || p.N <= 0 || p.K <= 0) return false;
   if (p.K % 8 != 0 || p.lda % 8 != 0) return false;                 // TMA strides are multiples of 16 bytes
@@ -329,8 +383,15 @@ es_status_t tc_build_maps(const LinearParams& p, int epi, int64_t a_rows, TcMaps
   return ES_OK;
 }
 
-es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word) {
+es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word, bool pdl) {
   if (!linear_tc_supported(p, epi)) return fail(ES_ERR_UNSUPPORTED, "tensor-core kernel does not take this shape");
+  if (p.k_splits > 1) {
+    if (epi != EPI_F32 || p.part == nullptr || p.N % 4 != 0)
+      return fail(ES_ERR_INVALID_ARG, "split-K needs the plain epilogue, a workspace and N %% 4 == 0");
+    const int num_kb = (p.K + BK - 1) / BK;
+    const int kb_per = (num_kb + p.k_splits - 1) / p.k_splits;
+    if ((p.k_splits - 1) * kb_per >= num_kb) return fail(ES_ERR_INVALID_ARG, "split-K: %d slices leave one empty (K = %d)", p.k_splits, p.K);
+  }
   TcMaps local;
   const TcMaps* maps = p.tc_maps;
   if (!maps) {
@@ -341,9 +402,9 @@ es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int
   const int bn = pick_bn(p, epi);
   es_status_t st;
   switch (epi) {
-    case EPI_F32: st = launch_epi<EPI_F32>(t, p, bn, status_word, s); break;
-    case EPI_SWIGLU: st = launch_epi<EPI_SWIGLU>(t, p, bn, status_word, s); break;
-    case EPI_QKV: st = launch_epi<EPI_QKV>(t, p, bn, status_word, s); break;
+    case EPI_F32: st = launch_epi<EPI_F32>(t, p, bn, status_word, s, pdl); break;
+    case EPI_SWIGLU: st = launch_epi<EPI_SWIGLU>(t, p, bn, status_word, s, pdl); break;
+    case EPI_QKV: st = launch_epi<EPI_QKV>(t, p, bn, status_word, s, pdl); break;
     default: return fail(ES_ERR_INVALID_ARG, "unknown epilogue %d", epi);
   }
   if (st == ES_OK && launches) ++*launches;

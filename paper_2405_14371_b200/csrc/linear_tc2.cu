@@ -14,6 +14,7 @@
 #include <string.h>
 
 #include "epilogue.cuh"
+#include "launch.cuh"
 #include "sm100.cuh"
 
 namespace es {
@@ -40,6 +41,7 @@ template <int EPI>
 __global__ void __launch_bounds__(T2_THREADS, 1)
 linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, int* status, int m_tiles, int n_tiles) {
   constexpr int BN_OUT = (EPI == EPI_SWIGLU) ? BN2 / 2 : BN2;
+  pdl_launch_dependents();
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -88,6 +90,7 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
   cluster_sync_all();                              // both CTAs' barriers exist before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                      // set-up above overlaps the previous kernel's tail
 
   if (warp == 0) {
     if (lane == 0) {
@@ -201,7 +204,7 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
 }
 
 template <int EPI>
-es_status_t launch_pair(const TmapSet2& maps, const LinearParams& p, int* status, cudaStream_t s) {
+es_status_t launch_pair(const TmapSet2& maps, const LinearParams& p, int* status, cudaStream_t s, bool pdl) {
   constexpr int out = (EPI == EPI_SWIGLU) ? BN2 / 2 : BN2;
   const int m_tiles = (p.M + 2 * BM2 - 1) / (2 * BM2), n_tiles = (p.N + out - 1) / out;
   auto kern = linear_tc2_kernel<EPI>;
@@ -224,13 +227,15 @@ es_status_t launch_pair(const TmapSet2& maps, const LinearParams& p, int* status
   cfg.blockDim = dim3(T2_THREADS);
   cfg.dynamicSmemBytes = SMEM2;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pdl ? 2 : 1;
   ES_CUDA_CHECK(cudaLaunchKernelEx(&cfg, kern, maps, p, status, m_tiles, n_tiles));
   return ES_OK;
 }
@@ -247,7 +252,7 @@ bool linear_tc2_supported(const LinearParams& p, int epi) {
   return p.M >= 2 * BM2 && tiles >= 74;
 }
 
-es_status_t launch_linear_tc2(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word) {
+es_status_t launch_linear_tc2(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word, bool pdl) {
   if (!linear_tc2_supported(p, epi)) return fail(ES_ERR_UNSUPPORTED, "pair kernel does not take this shape");
   TcMaps local;
   const TcMaps* maps = p.tc_maps;
@@ -258,9 +263,9 @@ es_status_t launch_linear_tc2(const LinearParams& p, int epi, cudaStream_t s, in
   const TmapSet2& t = *reinterpret_cast<const TmapSet2*>(maps);
   es_status_t st;
   switch (epi) {
-    case EPI_F32: st = launch_pair<EPI_F32>(t, p, status_word, s); break;
-    case EPI_SWIGLU: st = launch_pair<EPI_SWIGLU>(t, p, status_word, s); break;
-    case EPI_QKV: st = launch_pair<EPI_QKV>(t, p, status_word, s); break;
+    case EPI_F32: st = launch_pair<EPI_F32>(t, p, status_word, s, pdl); break;
+    case EPI_SWIGLU: st = launch_pair<EPI_SWIGLU>(t, p, status_word, s, pdl); break;
+    case EPI_QKV: st = launch_pair<EPI_QKV>(t, p, status_word, s, pdl); break;
     default: return fail(ES_ERR_INVALID_ARG, "unknown epilogue %d", epi);
   }
   if (st == ES_OK && launches) ++*launches;

@@ -40,7 +40,7 @@ static int env_int(const char* name, int dflt) {
 }
 
 const Tunables& tunables() {
-  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_PDL", 1)};
+  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_PDL", 1), env_int("ES_SPLIT_K", 1)};
   return t;
 }
 
@@ -69,7 +69,7 @@ struct Layout {
   size_t page_elems;   // halves in one page of one of K / V
   size_t kv_bytes;
   size_t off_x, off_h, off_q, off_ao, off_act, off_logits, off_next, off_hlast, off_part, off_cos, off_sin,
-      off_table, off_ctx, off_slots, off_status;
+      off_table, off_ctx, off_slots, off_status, off_splitk;
   size_t scratch_bytes;
 };
 
@@ -122,6 +122,7 @@ Layout make_layout(const es_model_desc_t& d, int begin, int end) {
   L.off_ctx = take((size_t)d.max_slots * 4);
   L.off_slots = take(B * 4);
   L.off_status = take(256);
+  L.off_splitk = take(d.max_tokens > 16 ? linear_tc_split_workspace_bytes() : 0);   // split-K partial sums of short prefills
   L.scratch_bytes = o;
   return L;
 }
@@ -170,6 +171,7 @@ struct es_shard {
   __half *h, *q, *ao, *act, *h_last;
   float *logits, *part, *rope_cos, *rope_sin;
   int *next_ids, *block_table, *ctx_len, *slots_dev, *status;
+  float* splitk = nullptr;      // split-K workspace (nullptr when the shard never runs more than 16 rows)
   std::vector<int> ctx;         // host mirror of ctx_len, -1 = never prefilled
   std::vector<int> slots_host;  // slots currently uploaded to slots_dev
   int last_B = 0, last_T = 0;
@@ -236,8 +238,9 @@ es_status_t dispatch_linear(es_shard* s, const LinearParams& p, int epi) {
   if (p.M > 2 && p.M <= 16 && linear_stream_mma_supported(p, epi))
     return launch_linear_stream_mma(p, epi, s->stream, &s->launches, s->pdl_now);
   if (p.M <= 16) return launch_linear_stream(p, epi, s->stream, &s->launches, s->pdl_now);
-  if (tunables().tc_pair && linear_tc2_supported(p, epi)) return launch_linear_tc2(p, epi, s->stream, &s->launches, s->status);
-  if (linear_tc_supported(p, epi)) return launch_linear_tc(p, epi, s->stream, &s->launches, s->status);
+  if (p.k_splits > 1) return launch_linear_tc(p, epi, s->stream, &s->launches, s->status, s->pdl_now);
+  if (tunables().tc_pair && linear_tc2_supported(p, epi)) return launch_linear_tc2(p, epi, s->stream, &s->launches, s->status, s->pdl_now);
+  if (linear_tc_supported(p, epi)) return launch_linear_tc(p, epi, s->stream, &s->launches, s->status, s->pdl_now);
   return launch_linear_reference(p, epi, s->stream, &s->launches);
 }
 
@@ -289,6 +292,13 @@ LinearParams base_params(const es_shard* s, int M, int T, bool decode) {
   return p;
 }
 
+// K slices for a product on the tensor-core path (1 = whole K range per tile).
+int split_k_for(const es_shard* s, const LinearParams& p, int epi) {
+  if (s->splitk == nullptr || p.M <= 16 || tunables().split_k == 0) return 1;
+  if (!linear_tc_supported(p, epi)) return 1;
+  return linear_tc_splits(p, epi);
+}
+
 // Parameters of the four linear layers of decoder layer li (kind: 0 qkv, 1 o, 2 gate/up, 3 down).
 LinearParams layer_linear(const es_shard* s, int li, int kind, int M, int T, bool decode, const float* xin, int* epi) {
   const es_model_desc_t& d = s->d;
@@ -337,9 +347,10 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   const int M = B * T;
   int pi = 0;
   const float* xin = s->x;
-  const bool pdl = decode && tunables().pdl != 0;
+  const bool pdl = tunables().pdl != 0;
   s->pdl_now = pdl;
   const bool fuse_norm = M <= 16 && linear_stream_can_fuse_norm(M);
+  bool h_ready = false;   // s->h already holds the normalised input of the coming layer
   if (s->has_emb) {
     prof_mark(s, pi, 0);
     ES_TRY(kt_begin(s));
@@ -356,11 +367,12 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     const es_layer_weights_t& w = s->lw[li];
     prof_mark(s, pi, 0);
     const bool pdl0 = (li == 0 && !s->has_emb) ? false : pdl;     // first kernel of the pass: full dependency
-    if (!fuse_norm) {
+    if (!fuse_norm && !h_ready) {
       ES_TRY(kt_begin(s));
       ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl0));
       ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0));
     }
+    h_ready = false;
     int epi = 0;
     {
       LinearParams p = layer_linear(s, li, 0, M, T, decode, xin, &epi);
@@ -388,16 +400,29 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       a.kv_rows = (int64_t)s->lay.n_pages * d.n_kv_heads * d.kv_page_tokens;
       a.status = s->status;
       a.tc_maps = s->attn_maps_valid ? &s->attn_maps[li] : nullptr;
-      ES_TRY(launch_prefill_attention(a, s->stream, &s->launches));
+      ES_TRY(launch_prefill_attention(a, s->stream, &s->launches, 0, pdl));
     }
     ES_TRY(kt_end(s, ES_KT_ATTENTION, 0.0));
+    bool o_split = false;
     {
       LinearParams p = layer_linear(s, li, 1, M, T, decode, xin, &epi);
       s->kt_next_cat = ES_KT_O;
-      ES_TRY(run_linear(s, p, epi));
+      const int splits = split_k_for(s, p, epi);
+      if (splits > 1) {
+        // short prompt: K slices into the workspace, then residual + RMSNorm for gate / up in the reduction
+        p.k_splits = splits; p.part = s->splitk;
+        ES_TRY(run_linear(s, p, epi));
+        ES_TRY(kt_begin(s));
+        ES_TRY(launch_splitk_reduce(s->splitk, splits, p.res, p.out_f32, M, p.N, p.ldo, (const __half*)w.ffn_norm, s->h,
+                                    d.rms_eps, s->stream, &s->launches, pdl));
+        ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * (8.0 + 4.0 * splits + 2.0)));
+        o_split = true;
+      } else {
+        ES_TRY(run_linear(s, p, epi));
+      }
     }
     xin = s->x;
-    if (!fuse_norm) {
+    if (!fuse_norm && !o_split) {
       ES_TRY(kt_begin(s));
       ES_TRY(launch_rmsnorm(s->x, (const __half*)w.ffn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl));
       ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0));
@@ -411,7 +436,21 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     {
       LinearParams p = layer_linear(s, li, 3, M, T, decode, xin, &epi);
       s->kt_next_cat = ES_KT_DOWN;
-      ES_TRY(run_linear(s, p, epi));
+      const int splits = split_k_for(s, p, epi);
+      if (splits > 1) {
+        // the reduction also normalises the finished rows for the next layer's QKV projection
+        p.k_splits = splits; p.part = s->splitk;
+        ES_TRY(run_linear(s, p, epi));
+        const bool more = li + 1 < s->nl;
+        ES_TRY(kt_begin(s));
+        ES_TRY(launch_splitk_reduce(s->splitk, splits, p.res, p.out_f32, M, p.N, p.ldo,
+                                    more ? (const __half*)s->lw[li + 1].attn_norm : nullptr, s->h, d.rms_eps, s->stream,
+                                    &s->launches, pdl));
+        ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * (8.0 + 4.0 * splits + (more ? 2.0 : 0.0))));
+        h_ready = more;
+      } else {
+        ES_TRY(run_linear(s, p, epi));
+      }
     }
     prof_mark(s, pi, 1);
   }
@@ -547,6 +586,7 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
   s->ctx_len = (int*)(sb + L.off_ctx);
   s->slots_dev = (int*)(sb + L.off_slots);
   s->status = (int*)(sb + L.off_status);
+  s->splitk = desc->max_tokens > 16 ? (float*)(sb + L.off_splitk) : nullptr;
   s->ctx.assign(desc->max_slots, -1);
 
   auto bail = [&](es_status_t st) { delete s; return st; };
@@ -884,6 +924,32 @@ es_status_t es_op_linear(const void* A, const void* W, const float* R, float* C,
       return launch_linear_stream_mma(p, EPI_F32, st, nullptr);
     default: return fail(ES_ERR_INVALID_ARG, "unknown path %d", path);
   }
+}
+
+size_t es_op_linear_splitk_workspace_bytes(int32_t M, int32_t N, int32_t k_splits) {
+  if (M <= 0 || N <= 0 || k_splits <= 0) return 0;
+  return (size_t)k_splits * M * N * sizeof(float);
+}
+
+es_status_t es_op_linear_splitk(const void* A, const void* W, const float* R, float* C, int32_t M, int32_t N, int32_t K,
+                                int32_t k_splits, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!A || !W || !C) return fail(ES_ERR_INVALID_ARG, "null argument");
+  if (M <= 0 || N <= 0 || K <= 0 || K % 8 || N % 4) return fail(ES_ERR_SHAPE, "M, N, K must be positive, K a multiple of 8 and N of 4");
+  LinearParams p{};
+  p.A = (const __half*)A; p.lda = K; p.w[0] = (const __half*)W; p.seg_rows[0] = N;
+  p.M = M; p.N = N; p.K = K; p.out_f32 = C; p.res = R; p.ldo = N; p.T = 1;
+  if (!linear_tc_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "tensor-core kernel does not take this shape");
+  if (k_splits == 0) k_splits = linear_tc_splits(p, EPI_F32);
+  if (k_splits < 1 || k_splits > 64) return fail(ES_ERR_INVALID_ARG, "k_splits must be 0 (automatic) or 1..64");
+  cudaStream_t st = (cudaStream_t)stream;
+  if (k_splits == 1) return launch_linear_tc(p, EPI_F32, st, nullptr, nullptr);
+  if (!workspace || workspace_bytes < es_op_linear_splitk_workspace_bytes(M, N, k_splits))
+    return fail(ES_ERR_WORKSPACE, "split-K workspace: %zu bytes given, %zu needed", workspace_bytes,
+                es_op_linear_splitk_workspace_bytes(M, N, k_splits));
+  if ((uintptr_t)workspace % 16) return fail(ES_ERR_INVALID_ARG, "workspace must be 16-byte aligned");
+  p.k_splits = k_splits; p.part = (float*)workspace;
+  ES_TRY(launch_linear_tc(p, EPI_F32, st, nullptr, nullptr));
+  return launch_splitk_reduce(p.part, k_splits, R, C, M, N, N, nullptr, nullptr, 0.f, st, nullptr);
 }
 
 es_status_t es_op_prefill_attention(const void* q, const void* k, const void* v, void* out, int32_t B, int32_t T,

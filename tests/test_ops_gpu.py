@@ -97,6 +97,34 @@ def test_linear_tensor_core_cta_pairs(B, M, N, K):
     assert rel_err(got, ref) < 1e-5
 
 
+@pytest.mark.parametrize("M,N,K,S", [(128, 4096, 4096, 0), (128, 4096, 11008, 0), (256, 5120, 5120, 0), (100, 260, 1096, 3),
+                                     (17, 36, 512, 2), (300, 1000, 4096, 5), (128, 512, 256, 4), (512, 4096, 4096, 0),
+                                     (128, 4096, 4096, 1)])
+def test_linear_tensor_core_split_k(B, M, N, K, S):
+    """K range cut into slices (automatic count and fixed counts), ragged M / N / K, residual aliasing the output."""
+    A = _randn(M, K, seed=22)
+    W = _randn(N, K, seed=23, scale=0.05)
+    R = _randn(M, N, seed=24, dtype=torch.float32)
+    want = A.double() @ W.double().T
+    got = B.es_op_linear_splitk(A.cuda(), W.cuda(), None, S)
+    assert rel_err(got, want) < 5e-5
+    got_r = B.es_op_linear_splitk(A.cuda(), W.cuda(), R.cuda(), S)
+    assert rel_err(got_r, want + R.double()) < 5e-5
+    again = B.es_op_linear_splitk(A.cuda(), W.cuda(), R.cuda(), S)
+    assert torch.equal(got_r, again)            # slices are added in a fixed order
+
+
+def test_linear_split_k_rejects(B):
+    A = _randn(128, 256, seed=1).cuda()
+    W = _randn(64, 256, seed=2).cuda()
+    with pytest.raises(B.EsError):               # 4 K blocks cannot make 3 non-empty slices of 2
+        B.es_op_linear_splitk(A, W, None, 3)
+    with pytest.raises(B.EsError):               # workspace too small
+        B.es_op_linear_splitk(A, W, None, 2, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(B.EsError):               # N not a multiple of 4
+        B.es_op_linear_splitk(A, _randn(62, 256, seed=3).cuda(), None, 2)
+
+
 def test_linear_rejects_bad_shapes(B):
     A = _randn(17, 64).cuda()
     W = _randn(32, 64).cuda()
