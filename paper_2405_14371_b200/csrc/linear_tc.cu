@@ -32,9 +32,11 @@ constexpr int TC_THREADS = 192;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 
 template <int BN> struct TileCfg {
+  static_assert(BN % 32 == 0 && BN >= 32 && BN <= 256, "tile width: a multiple of the 32-row weight box, at most one MMA wide");
   static constexpr int B_STAGE_BYTES = BN * BK * 2;
-  static constexpr int STAGES = (BN >= 256) ? 4 : (BN >= 128) ? 6 : 8;
-  static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
+  static constexpr int STAGES = (200 * 1024) / (A_STAGE_BYTES + B_STAGE_BYTES) > 8 ? 8 : (200 * 1024) / (A_STAGE_BYTES + B_STAGE_BYTES);
+  static constexpr int TMEM_COLS = BN;                                       // one accumulator buffer
+  static constexpr int TMEM_ALLOC = 2 * BN <= 64 ? 64 : 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512;   // two buffers, power of two
   static constexpr size_t SMEM = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
 };
 
@@ -113,7 +115,7 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 2 * ACC_COLS);
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), Cfg::TMEM_ALLOC);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -244,7 +246,7 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
   if (warp == 1) {
     tc_fence_after();
     if (*abort_flag) __nanosleep(100000);     // let copies still in flight land before the CTA's memory is released
-    tmem_dealloc(tmem_base, 2 * ACC_COLS);
+    tmem_dealloc(tmem_base, Cfg::TMEM_ALLOC);
   }
 }
 
@@ -278,12 +280,12 @@ int pick_bn(const LinearParams& p, int epi) {
   // one CTA per SM at a time, so the time goes as (waves of CTAs) x (128 + bn).  Take the width
   // that minimises it (the wider one on ties); QKV segments must be whole tiles.
   const int m_tiles = (p.M + BM - 1) / BM;
-  const int cands[4] = {256, 128, 64, 32};
+  const int cands[8] = {256, 224, 192, 160, 128, 96, 64, 32};
   int best = 0;
   long long best_cost = 0;
   for (int bn : cands) {
     const int out = (epi == EPI_SWIGLU) ? bn / 2 : bn;
-    bool fits = !(epi == EPI_SWIGLU && bn < 2 * W_BOX_ROWS);
+    bool fits = !(epi == EPI_SWIGLU && bn % (2 * W_BOX_ROWS) != 0);      // gate half and up half are whole weight boxes
     if (epi == EPI_QKV)
       for (int s = 0; s < 3; ++s) if (p.seg_rows[s] % out) fits = false;
     if (!fits) continue;
@@ -321,9 +323,17 @@ template <int EPI>
 es_status_t launch_epi(const TmapSet& maps, const LinearParams& p, int bn, int* status, cudaStream_t s, bool pdl) {
   switch (bn) {
     case 256: return launch_bn<EPI, 256>(maps, p, status, s, pdl);
+    case 192: return launch_bn<EPI, 192>(maps, p, status, s, pdl);
     case 128: return launch_bn<EPI, 128>(maps, p, status, s, pdl);
     case 64: return launch_bn<EPI, 64>(maps, p, status, s, pdl);
-    case 32: return launch_bn<EPI, 32>(maps, p, status, s, pdl);
+  }
+  if constexpr (EPI != EPI_SWIGLU) {      // widths whose halves are not whole weight boxes
+    switch (bn) {
+      case 224: return launch_bn<EPI, 224>(maps, p, status, s, pdl);
+      case 160: return launch_bn<EPI, 160>(maps, p, status, s, pdl);
+      case 96: return launch_bn<EPI, 96>(maps, p, status, s, pdl);
+      case 32: return launch_bn<EPI, 32>(maps, p, status, s, pdl);
+    }
   }
   return fail(ES_ERR_UNSUPPORTED, "no tile width for this shape");
 }

@@ -56,9 +56,11 @@ def test_linear_reference_large(B, M, N, K):
 
 
 @pytest.mark.parametrize("M,N,K", [(17, 32, 64), (128, 128, 64), (100, 200, 136), (257, 1000, 688), (512, 4096, 4096),
-                                   (300, 96, 4096), (128, 4096, 11008), (1024, 640, 256), (2100, 384, 1024)])
+                                   (300, 96, 4096), (128, 4096, 11008), (1024, 640, 256), (2100, 384, 1024),
+                                   (128, 11008, 512), (128, 20000, 256), (100, 25000, 256), (128, 30000, 320)])
 def test_linear_tensor_core(B, M, N, K):
-    """tcgen05 path: several tile widths, ragged M / N / K, long K, and agreement with the plain kernel."""
+    """tcgen05 path: every tile width (32 .. 256 in steps of 32 — the last four shapes select 96, 160, 192
+    and 224), ragged M / N / K, long K, and agreement with the plain kernel."""
     A = _randn(M, K, seed=13)
     W = _randn(N, K, seed=14, scale=0.05)
     R = _randn(M, N, seed=15, dtype=torch.float32)
