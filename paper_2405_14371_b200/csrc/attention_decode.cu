@@ -236,6 +236,17 @@ es_status_t launch_g(const DecodeAttnParams& p, cudaStream_t s, bool pdl) {
 template <int HD>
 es_status_t launch_hd(const DecodeAttnParams& p, cudaStream_t s, bool pdl, int64_t* launches) {
   es_status_t st;
+  // many items (several sequences, long contexts): the tensor-core kernel, which keeps more bytes in flight
+  const bool many = (long long)p.n_splits * p.Hkv * p.B >= 128;
+  if (many && tunables().attn_mma != 0 && decode_attention_mma_supported(p)) {
+    ES_TRY(launch_decode_attention_mma(p, s, pdl));
+    if (launches) ++*launches;
+    if (p.n_splits > 1) {
+      ES_CUDA_CHECK(launch_kernel(decode_attn_merge_kernel<HD>, dim3(p.Hq, p.B), dim3(HD), 0, s, pdl, p));
+      if (launches) ++*launches;
+    }
+    return ES_OK;
+  }
   switch (p.Hq / p.Hkv) {
     case 1: st = launch_g<HD, 1>(p, s, pdl); break;
     case 2: st = launch_g<HD, 2>(p, s, pdl); break;

@@ -32,6 +32,7 @@ struct Tunables {
   int stream_deep;   // ES_STREAM_DEEP: weight-streaming kernel chunk depth, 1 = 4 KB per warp per buffer (default), 0 = 2 KB
   int tc_pair;       // ES_TC_PAIR: CTA-pair tensor-core kernel for large prefill products (1, default) or never (0)
   int pdl;           // ES_PDL: programmatic dependent launch in decode steps (1, default) or plain stream order (0)
+  int attn_mma;      // ES_ATTN_MMA: tensor-core decode attention for launches with many items (1, default) or never (0)
   int split_k;       // ES_SPLIT_K: split-K for the O and down projections of short prefills (1, default) or never (0)
 };
 const Tunables& tunables();
@@ -175,5 +176,8 @@ struct DecodeAttnParams {
 size_t decode_attention_scratch_bytes(int B, int Hq, int hd, int n_splits);
 void choose_splits(int max_ctx, int P, int B, int Hkv, int group, int* n_splits, int* pages_per_split);
 es_status_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t s, int64_t* launches, bool pdl = false);
+// tensor-core (mma.sync) split kernel for head_dim 128; same partial layout, merged by the same merge kernel
+bool decode_attention_mma_supported(const DecodeAttnParams& p);
+es_status_t launch_decode_attention_mma(const DecodeAttnParams& p, cudaStream_t s, bool pdl = false);
 
 }  // namespace es

@@ -40,7 +40,7 @@ static int env_int(const char* name, int dflt) {
 }
 
 const Tunables& tunables() {
-  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_PDL", 1), env_int("ES_SPLIT_K", 1)};
+  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_PDL", 1), env_int("ES_ATTN_MMA", 1), env_int("ES_SPLIT_K", 1)};
   return t;
 }
 
@@ -52,7 +52,9 @@ void choose_splits(int max_ctx, int P, int B, int Hkv, int group, int* n_splits,
   // bytes in flight); four times as many for larger groups, whose CTAs are arithmetic heavy
   const int ctas = (group >= 4 ? 4 : 1) * 148;
   long long pps = (long long)pages * B * Hkv / ctas;
-  const int min_pps = 256 / P > 1 ? 256 / P : 1;      // at least 256 tokens per split
+  // at least 256 tokens per split (384 for large groups, whose CTAs carry more fixed work per split)
+  const int min_tokens = group >= 4 ? 384 : 256;
+  const int min_pps = min_tokens / P > 1 ? min_tokens / P : 1;
   if (pps < min_pps) pps = min_pps;
   if (pps > pages) pps = pages;
   *pages_per_split = (int)pps;

@@ -156,6 +156,9 @@ def test_prefill_attention(B, path, Bn, T, Hq, Hkv, hd):
 @pytest.mark.parametrize("Bn,Hq,Hkv,hd,P,ctxs", [
     (1, 4, 4, 64, 16, [1]), (2, 4, 4, 64, 16, [16, 17]), (3, 8, 2, 128, 64, [5, 64, 200]),
     (2, 8, 1, 128, 64, [300, 1]), (4, 32, 32, 128, 64, [128, 129, 255, 256]), (16, 64, 8, 128, 64, list(range(1000, 1016))),
+    # many (sequence, head, split) items: the tensor-core kernel, all group sizes, ragged and tiny contexts, small pages
+    (8, 32, 32, 128, 64, [640, 513, 300, 17, 1, 639, 256, 257]), (12, 16, 8, 128, 16, [100 + 27 * i for i in range(12)]),
+    (10, 32, 8, 128, 32, [1, 15, 16, 17, 31, 33, 300, 299, 512, 700]), (40, 8, 8, 128, 64, [3 + 5 * i for i in range(40)]),
 ])
 def test_decode_attention_paged(B, Bn, Hq, Hkv, hd, P, ctxs):
     max_ctx = max(ctxs)
