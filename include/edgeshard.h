@@ -241,7 +241,11 @@ ES_API es_status_t es_op_linear(const void *A, const void *W, const float *R, fl
  * the slices in ascending order and the residual, so the result does not depend on scheduling.
  * k_splits = 0 lets the library choose (1 = no split, no workspace needed).  Slices must not be
  * empty: (k_splits - 1) * ceil(ceil(K / 64) / k_splits) < ceil(K / 64), else ES_ERR_INVALID_ARG.
- * N must be a multiple of 4, K of 8.  R may be NULL and may alias C. */
+ * N must be a multiple of 4, K of 8.  R may be NULL and may alias C.
+ * With 3 <= M <= 16 (a decode step of several sequences) the weight-streaming kernel is used instead:
+ * every CTA keeps one K slice of the activations in shared memory and streams 16-row groups of W over
+ * it; K must be a multiple of 256 and K / 32 divisible by k_splits, a slice of 8 (M <= 8) or 16 rows
+ * must fit 100 KB.  M <= 2 is ES_ERR_UNSUPPORTED (such products never need slicing). */
 ES_API size_t es_op_linear_splitk_workspace_bytes(int32_t M, int32_t N, int32_t k_splits);
 ES_API es_status_t es_op_linear_splitk(const void *A, const void *W, const float *R, float *C, int32_t M, int32_t N,
                                        int32_t K, int32_t k_splits, void *workspace, size_t workspace_bytes,

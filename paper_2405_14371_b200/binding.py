@@ -321,7 +321,7 @@ def es_op_linear_splitk(A: torch.Tensor, W: torch.Tensor, R: Optional[torch.Tens
     N = W.shape[0]
     Cout = torch.empty(M, N, dtype=torch.float32, device=A.device)
     if workspace is None:
-        workspace = torch.empty(max(1, es_op_linear_splitk_workspace_bytes(M, N, max(k_splits, 8))), dtype=torch.uint8,
+        workspace = torch.empty(max(1, es_op_linear_splitk_workspace_bytes(M, N, max(k_splits, 8 if M > 16 else 32))), dtype=torch.uint8,
                                 device=A.device)
     _check(lib.es_op_linear_splitk(_ptr(A), _ptr(W), _ptr(R), _ptr(Cout), M, N, K, k_splits, _ptr(workspace),
                                    workspace.numel() * workspace.element_size(), _stream_ptr(stream)))

@@ -71,7 +71,8 @@ __global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const Decod
   const int g = lane >> 2, t = lane & 3;
   // read-only state of earlier passes (slot list, page map, context length) may be read before the wait
   const int slot = p.kv.slots ? p.kv.slots[b] : b;
-  const int ctx = p.ctx_len[slot] + p.ctx_add;
+  const int ctx_old = p.ctx_len[slot];
+  const int ctx = ctx_old + p.ctx_add;
   const int tokens_per_split = p.pages_per_split * p.kv.P;
   const int t_begin = split * tokens_per_split;
   if (t_begin >= ctx) { pdl_wait(); return; }
@@ -79,16 +80,6 @@ __global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const Decod
   const float scale = rsqrtf((float)HD);
   const int64_t kv_head_off = (int64_t)kvh * p.kv.head_stride;
   const int* table = p.kv.block_table ? p.kv.block_table + (int64_t)slot * p.kv.pages_per_slot : nullptr;
-
-  pdl_wait();
-
-  // query fragments: row g of the A operand = head g of the group (rows >= G and rows 8..15 are zero)
-  uint4 qa[4];
-  {
-    const __half* qrow = p.q + ((int64_t)b * p.Hq + (int64_t)kvh * G + (g < G ? g : 0)) * HD;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) qa[j] = (g < G) ? *reinterpret_cast<const uint4*>(qrow + (4 * j + t) * 8) : make_uint4(0, 0, 0, 0);
-  }
 
   // base address of the 16-token block starting at token T (inside one page: P >= 16, T % 16 == 0)
   auto block_base = [&](int T) -> int64_t {
@@ -125,8 +116,22 @@ __global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const Decod
   for (int i = 0; i < 8; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
   float m_run = -INFINITY, l_run = 0.f;      // head g (replicated in the 4 threads of the group)
 
+  // The first block's K and V rows are requested before the dependency wait when every one of its
+  // tokens was cached by an earlier pass (the newest token's rows come from the kernel just before).
   int T = t_begin + warp * 16;
-  if (T < t_end) { load_k(T); load_v(T); }
+  const bool early = T < t_end && T + 16 <= ctx_old;
+  if (early) { load_k(T); load_v(T); }
+
+  pdl_wait();
+
+  // query fragments: row g of the A operand = head g of the group (rows >= G and rows 8..15 are zero)
+  uint4 qa[4];
+  {
+    const __half* qrow = p.q + ((int64_t)b * p.Hq + (int64_t)kvh * G + (g < G ? g : 0)) * HD;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) qa[j] = (g < G) ? *reinterpret_cast<const uint4*>(qrow + (4 * j + t) * 8) : make_uint4(0, 0, 0, 0);
+  }
+  if (T < t_end && !early) { load_k(T); load_v(T); }
   for (; T < t_end; T += MW * 16) {
     const int Tn = T + MW * 16;
     // ---- scores of 16 tokens ----

@@ -81,8 +81,8 @@ struct LinearParams {
   int T;                   // rows per sequence: row m belongs to sequence m / T at prompt offset m % T
   int is_decode;           // position = ctx_len[slot] instead of m % T
   int Hq, Hkv, hd, P, pages_per_slot, max_seq;
-  // split-K (tensor-core kernel, EPI_F32 only): > 1 = raw partial sums go to part[k_splits, M, N] instead
-  // of out_f32; launch_splitk_reduce finishes the product
+  // split-K (tensor-core kernel with EPI_F32; K-sliced streaming kernel with any epilogue): > 1 = raw partial
+  // sums go to part[k_splits, M, columns] and a second kernel finishes the product
   int k_splits;
   float* part;
 };
@@ -94,6 +94,11 @@ bool linear_stream_can_fuse_norm(int M);
 // tensor-core (mma.sync) variant of the weight-streaming kernel for 3..16 rows
 bool linear_stream_mma_supported(const LinearParams& p, int epi);
 es_status_t launch_linear_stream_mma(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl = false);
+// K slices across CTAs for this product (1 = the activations fit in shared memory whole); with p.k_splits > 1
+// the kernel writes partial sums to p.part ([k_splits, M, N], SwiGLU: [k_splits, M, 2N] gate | up) and the
+// product is finished by launch_splitk_reduce (plain epilogue) or launch_splitk_finish (SwiGLU, QKV)
+int linear_stream_mma_splits(const LinearParams& p, int epi, size_t workspace_bytes);
+es_status_t launch_splitk_finish(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl = false);
 es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word, bool pdl = false);
 bool linear_tc_supported(const LinearParams& p, int epi);
 // number of K slices the tensor-core kernel should use for this product (1 = do not split), and the

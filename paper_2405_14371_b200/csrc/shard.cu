@@ -124,7 +124,7 @@ Layout make_layout(const es_model_desc_t& d, int begin, int end) {
   L.off_ctx = take((size_t)d.max_slots * 4);
   L.off_slots = take(B * 4);
   L.off_status = take(256);
-  L.off_splitk = take(d.max_tokens > 16 ? linear_tc_split_workspace_bytes() : 0);   // split-K partial sums of short prefills
+  L.off_splitk = take(d.max_tokens > 2 ? linear_tc_split_workspace_bytes() : 0);   // split-K partial sums of short prefills
   L.scratch_bytes = o;
   return L;
 }
@@ -173,7 +173,7 @@ struct es_shard {
   __half *h, *q, *ao, *act, *h_last;
   float *logits, *part, *rope_cos, *rope_sin;
   int *next_ids, *block_table, *ctx_len, *slots_dev, *status;
-  float* splitk = nullptr;      // split-K workspace (nullptr when the shard never runs more than 16 rows)
+  float* splitk = nullptr;      // split-K workspace (nullptr when the shard never runs more than 2 rows)
   std::vector<int> ctx;         // host mirror of ctx_len, -1 = never prefilled
   std::vector<int> slots_host;  // slots currently uploaded to slots_dev
   int last_B = 0, last_T = 0;
@@ -296,9 +296,22 @@ LinearParams base_params(const es_shard* s, int M, int T, bool decode) {
 
 // K slices for a product on the tensor-core path (1 = whole K range per tile).
 int split_k_for(const es_shard* s, const LinearParams& p, int epi) {
-  if (s->splitk == nullptr || p.M <= 16 || tunables().split_k == 0) return 1;
+  if (s->splitk == nullptr || p.M <= 2 || tunables().split_k == 0) return 1;
+  if (p.M <= 16) return linear_stream_mma_splits(p, epi, linear_tc_split_workspace_bytes());   // decode with several sequences
   if (!linear_tc_supported(p, epi)) return 1;
   return linear_tc_splits(p, epi);
+}
+
+// A product whose K range may be sliced (QKV and gate / up forms): the kernel, then the finishing kernel.
+es_status_t run_linear_sliced(es_shard* s, LinearParams& p, int epi, bool pdl) {
+  const int splits = split_k_for(s, p, epi);
+  if (splits <= 1 || p.M > 16) return run_linear(s, p, epi);
+  p.k_splits = splits;
+  p.part = s->splitk;
+  ES_TRY(run_linear(s, p, epi));
+  ES_TRY(kt_begin(s));
+  ES_TRY(launch_splitk_finish(p, epi, s->stream, &s->launches, pdl));
+  return kt_end(s, s->kt_next_cat, 0.0);
 }
 
 // Parameters of the four linear layers of decoder layer li (kind: 0 qkv, 1 o, 2 gate/up, 3 down).
@@ -381,7 +394,7 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       if (fuse_norm) { p.norm_x = xin; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.attn_norm; p.norm_eps = d.rms_eps; }
       s->kt_next_cat = ES_KT_QKV;
       s->pdl_now = fuse_norm ? pdl0 : pdl;
-      ES_TRY(run_linear(s, p, epi));
+      ES_TRY(run_linear_sliced(s, p, epi, pdl));
       s->pdl_now = pdl;
     }
     KvView kvv{};
@@ -433,7 +446,7 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       LinearParams p = layer_linear(s, li, 2, M, T, decode, xin, &epi);
       if (fuse_norm) { p.norm_x = s->x; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.ffn_norm; p.norm_eps = d.rms_eps; }
       s->kt_next_cat = ES_KT_GATE_UP;
-      ES_TRY(run_linear(s, p, epi));
+      ES_TRY(run_linear_sliced(s, p, epi, pdl));
     }
     {
       LinearParams p = layer_linear(s, li, 3, M, T, decode, xin, &epi);
@@ -588,7 +601,7 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
   s->ctx_len = (int*)(sb + L.off_ctx);
   s->slots_dev = (int*)(sb + L.off_slots);
   s->status = (int*)(sb + L.off_status);
-  s->splitk = desc->max_tokens > 16 ? (float*)(sb + L.off_splitk) : nullptr;
+  s->splitk = desc->max_tokens > 2 ? (float*)(sb + L.off_splitk) : nullptr;
   s->ctx.assign(desc->max_slots, -1);
 
   auto bail = [&](es_status_t st) { delete s; return st; };
@@ -940,15 +953,28 @@ es_status_t es_op_linear_splitk(const void* A, const void* W, const float* R, fl
   LinearParams p{};
   p.A = (const __half*)A; p.lda = K; p.w[0] = (const __half*)W; p.seg_rows[0] = N;
   p.M = M; p.N = N; p.K = K; p.out_f32 = C; p.res = R; p.ldo = N; p.T = 1;
-  if (!linear_tc_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "tensor-core kernel does not take this shape");
-  if (k_splits == 0) k_splits = linear_tc_splits(p, EPI_F32);
-  if (k_splits < 1 || k_splits > 64) return fail(ES_ERR_INVALID_ARG, "k_splits must be 0 (automatic) or 1..64");
   cudaStream_t st = (cudaStream_t)stream;
-  if (k_splits == 1) return launch_linear_tc(p, EPI_F32, st, nullptr, nullptr);
+  const bool skinny = M <= 16;            // decode-sized: the K-sliced weight-streaming kernel
+  if (skinny) {
+    if (M < 3 || !linear_stream_mma_supported(p, EPI_F32))
+      return fail(ES_ERR_UNSUPPORTED, "K-sliced streaming kernel takes 3..16 rows and K a multiple of 256");
+    if (k_splits == 0) k_splits = linear_stream_mma_splits(p, EPI_F32, workspace ? workspace_bytes : 0);
+  } else {
+    if (!linear_tc_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "tensor-core kernel does not take this shape");
+    if (k_splits == 0) k_splits = linear_tc_splits(p, EPI_F32);
+  }
+  if (k_splits < 1 || k_splits > 64) return fail(ES_ERR_INVALID_ARG, "k_splits must be 0 (automatic) or 1..64");
+  if (k_splits == 1)
+    return skinny ? launch_linear_stream_mma(p, EPI_F32, st, nullptr) : launch_linear_tc(p, EPI_F32, st, nullptr, nullptr);
   if (!workspace || workspace_bytes < es_op_linear_splitk_workspace_bytes(M, N, k_splits))
     return fail(ES_ERR_WORKSPACE, "split-K workspace: %zu bytes given, %zu needed", workspace_bytes,
                 es_op_linear_splitk_workspace_bytes(M, N, k_splits));
   if ((uintptr_t)workspace % 16) return fail(ES_ERR_INVALID_ARG, "workspace must be 16-byte aligned");
+  p.k_splits = k_splits; p.part = (float*)workspace;
+  if (skinny) {
+    ES_TRY(launch_linear_stream_mma(p, EPI_F32, st, nullptr));
+    return launch_splitk_reduce(p.part, k_splits, R, C, M, N, N, nullptr, nullptr, 0.f, st, nullptr);
+  }
   p.k_splits = k_splits; p.part = (float*)workspace;
   ES_TRY(launch_linear_tc(p, EPI_F32, st, nullptr, nullptr));
   return launch_splitk_reduce(p.part, k_splits, R, C, M, N, N, nullptr, nullptr, 0.f, st, nullptr);

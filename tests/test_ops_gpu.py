@@ -116,6 +116,21 @@ def test_linear_tensor_core_split_k(B, M, N, K, S):
     assert torch.equal(got_r, again)            # slices are added in a fixed order
 
 
+@pytest.mark.parametrize("M,N,K,S", [(8, 4096, 11008, 0), (16, 2048, 28672, 0), (16, 1024, 8192, 0), (5, 1000, 2048, 2),
+                                     (3, 36, 1024, 4), (13, 520, 4096, 8), (16, 8192, 8192, 4)])
+def test_linear_streaming_k_sliced(B, M, N, K, S):
+    """Decode-sized products with K sliced across CTAs (activation slice in shared memory), automatic and fixed slice
+    counts, ragged N, 1 and 2 groups of 8 activation rows; must agree with the unsliced streaming kernel."""
+    A = _randn(M, K, seed=25)
+    W = _randn(N, K, seed=26, scale=0.05)
+    R = _randn(M, N, seed=27, dtype=torch.float32)
+    want = A.double() @ W.double().T + R.double()
+    got = B.es_op_linear_splitk(A.cuda(), W.cuda(), R.cuda(), S)
+    assert rel_err(got, want) < 5e-5
+    assert rel_err(got, B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), 4)) < 1e-5
+    assert torch.equal(got, B.es_op_linear_splitk(A.cuda(), W.cuda(), R.cuda(), S))
+
+
 def test_linear_split_k_rejects(B):
     A = _randn(128, 256, seed=1).cuda()
     W = _randn(64, 256, seed=2).cuda()
