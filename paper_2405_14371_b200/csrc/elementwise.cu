@@ -40,12 +40,16 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return t;
 }
 
-// One CTA per row; the row stays in registers between the two passes (up to 8 float4 per thread,
-// i.e. d <= 8192 at 256 threads); longer rows are re-read.
+// One CTA per row; the row stays in registers between the two passes (THREADS x REGS float4, i.e.
+// d <= 8192); longer rows are re-read.  Two shapes: 256 threads x 8 for the many rows of a prefill,
+// 1024 x 2 for the up to 16 rows of a decode step (a row then has four times the threads).  The
+// split-K reduction below uses the same two shapes and the same order of additions, so a row
+// normalised there and a row normalised here agree bit for bit.
 constexpr int RMS_THREADS = 256;
 constexpr int RMS_REGS = 8;
 
-__global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const float* __restrict__ x,
+template <int THREADS, int REGS>
+__global__ void __launch_bounds__(THREADS) rmsnorm_kernel(const float* __restrict__ x,
                                                               const __half* __restrict__ gain,
                                                               __half* __restrict__ y, int d, float eps,
                                                               int64_t row_stride, int64_t row_offset) {
@@ -55,17 +59,17 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const float* __res
   const int r = blockIdx.x;
   const float4* src = reinterpret_cast<const float4*>(x + ((int64_t)r * row_stride + row_offset) * d);
   const int n4 = d / 4;
-  float4 v[RMS_REGS];
+  float4 v[REGS];
   float ss = 0.f;
 #pragma unroll
-  for (int i = 0; i < RMS_REGS; ++i) {
-    const int c = threadIdx.x + i * RMS_THREADS;
+  for (int i = 0; i < REGS; ++i) {
+    const int c = threadIdx.x + i * THREADS;
     if (c < n4) {
       v[i] = src[c];
       ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
     }
   }
-  for (int c = threadIdx.x + RMS_REGS * RMS_THREADS; c < n4; c += RMS_THREADS) {
+  for (int c = threadIdx.x + REGS * THREADS; c < n4; c += THREADS) {
     const float4 t = src[c];
     ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
   }
@@ -74,15 +78,15 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const float* __res
   __half2* dst = reinterpret_cast<__half2*>(y + (int64_t)r * d);
   const __half2* g2 = reinterpret_cast<const __half2*>(gain);
 #pragma unroll
-  for (int i = 0; i < RMS_REGS; ++i) {
-    const int c = threadIdx.x + i * RMS_THREADS;
+  for (int i = 0; i < REGS; ++i) {
+    const int c = threadIdx.x + i * THREADS;
     if (c < n4) {
       const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
       dst[2 * c] = __floats2half2_rn(v[i].x * inv * ga.x, v[i].y * inv * ga.y);
       dst[2 * c + 1] = __floats2half2_rn(v[i].z * inv * gb.x, v[i].w * inv * gb.y);
     }
   }
-  for (int c = threadIdx.x + RMS_REGS * RMS_THREADS; c < n4; c += RMS_THREADS) {
+  for (int c = threadIdx.x + REGS * THREADS; c < n4; c += THREADS) {
     const float4 t = src[c];
     const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
     dst[2 * c] = __floats2half2_rn(t.x * inv * ga.x, t.y * inv * ga.y);
@@ -93,40 +97,48 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(const float* __res
 // Finishes a split-K product: out[r, :] = (res ? res[r, :] : 0) + part[0, r, :] + part[1, r, :] + ...
 // (slices in ascending order, so the sum does not depend on scheduling) and, with a gain vector, the
 // RMSNorm of the finished row in fp16 for the next product — one CTA per row, the row kept in
-// registers between the two passes like rmsnorm_kernel does.
-__global__ void __launch_bounds__(RMS_THREADS) splitk_reduce_kernel(const float* __restrict__ part, int k_splits,
-                                                                    const float* res, float* out, int M, int N,
-                                                                    int64_t ldo, const __half* __restrict__ gain,
-                                                                    __half* __restrict__ y, float eps) {
+// registers between the two passes like rmsnorm_kernel does.  THREADS x REGS float4 columns stay in
+// registers (prefill: many rows, 256 threads; decode: up to 16 rows, 1024 threads each).
+template <int THREADS, int REGS>
+__global__ void __launch_bounds__(THREADS) splitk_reduce_kernel(const float* __restrict__ part, int k_splits,
+                                                                const float* res, float* out, int M, int N,
+                                                                int64_t ldo, const __half* __restrict__ gain,
+                                                                __half* __restrict__ y, float eps) {
   __shared__ float red[32];
   pdl_launch_dependents();
   pdl_wait();
   const int r = blockIdx.x;
   const int n4 = N / 4;
-  const int64_t slice = (int64_t)M * N;
+  const int64_t slice4 = (int64_t)M * N / 4;
   const float4* src = reinterpret_cast<const float4*>(part + (int64_t)r * N);
   const float4* rs = res ? reinterpret_cast<const float4*>(res + (int64_t)r * ldo) : nullptr;
   float4* dst = reinterpret_cast<float4*>(out + (int64_t)r * ldo);
   auto finish = [&](int c) {
     float4 a = rs ? rs[c] : make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < k_splits; ++s) {
-      const float4 v = __ldcs(src + (s * slice) / 4 + c);
-      a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    // eight slices are requested at a time and then added in slice order
+    for (int s0 = 0; s0 < k_splits; s0 += 8) {
+      float4 v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        v[j] = (s0 + j < k_splits) ? __ldcs(src + (s0 + j) * slice4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (s0 + j < k_splits) { a.x += v[j].x; a.y += v[j].y; a.z += v[j].z; a.w += v[j].w; }
     }
     dst[c] = a;
     return a;
   };
-  float4 v[RMS_REGS];
+  float4 v[REGS];
   float ss = 0.f;
 #pragma unroll
-  for (int i = 0; i < RMS_REGS; ++i) {
-    const int c = threadIdx.x + i * RMS_THREADS;
+  for (int i = 0; i < REGS; ++i) {
+    const int c = threadIdx.x + i * THREADS;
     if (c < n4) {
       v[i] = finish(c);
       ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
     }
   }
-  for (int c = threadIdx.x + RMS_REGS * RMS_THREADS; c < n4; c += RMS_THREADS) {
+  for (int c = threadIdx.x + REGS * THREADS; c < n4; c += THREADS) {
     const float4 t = finish(c);
     ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
   }
@@ -136,15 +148,15 @@ __global__ void __launch_bounds__(RMS_THREADS) splitk_reduce_kernel(const float*
   __half2* yd = reinterpret_cast<__half2*>(y + (int64_t)r * N);
   const __half2* g2 = reinterpret_cast<const __half2*>(gain);
 #pragma unroll
-  for (int i = 0; i < RMS_REGS; ++i) {
-    const int c = threadIdx.x + i * RMS_THREADS;
+  for (int i = 0; i < REGS; ++i) {
+    const int c = threadIdx.x + i * THREADS;
     if (c < n4) {
       const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
       yd[2 * c] = __floats2half2_rn(v[i].x * inv * ga.x, v[i].y * inv * ga.y);
       yd[2 * c + 1] = __floats2half2_rn(v[i].z * inv * gb.x, v[i].w * inv * gb.y);
     }
   }
-  for (int c = threadIdx.x + RMS_REGS * RMS_THREADS; c < n4; c += RMS_THREADS) {
+  for (int c = threadIdx.x + REGS * THREADS; c < n4; c += THREADS) {
     const float4 t = dst[c];                         // written by this thread above
     const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
     yd[2 * c] = __floats2half2_rn(t.x * inv * ga.x, t.y * inv * ga.y);
@@ -211,7 +223,10 @@ es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, i
 es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M, int d, float eps,
                            int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches, bool pdl) {
   if (M <= 0) return ES_OK;
-  ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel, dim3(M), dim3(RMS_THREADS), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset));
+  if (M <= 16)
+    ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset));
+  else
+    ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset));
   if (launches) ++*launches;
   return ES_OK;
 }
@@ -227,7 +242,10 @@ es_status_t launch_splitk_reduce(const float* part, int k_splits, const float* r
                                  const __half* gain, __half* y, float eps, cudaStream_t s, int64_t* launches, bool pdl) {
   if (M <= 0 || N <= 0) return ES_OK;
   if (N % 4 != 0 || ldo % 4 != 0) return fail(ES_ERR_SHAPE, "split-K reduction needs N and the row stride to be multiples of 4");
-  ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel, dim3(M), dim3(RMS_THREADS), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps));
+  if (M <= 16)
+    ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps));
+  else
+    ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps));
   if (launches) ++*launches;
   return ES_OK;
 }

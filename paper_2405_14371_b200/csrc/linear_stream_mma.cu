@@ -362,9 +362,18 @@ __global__ void __launch_bounds__(256) splitk_finish_kernel(const LinearParams p
     const bool has1 = (EPI == EPI_SWIGLU) || (n + 1 < p.N);
     const float* src = p.part + (int64_t)m * part_cols;
     float v0 = 0.f, v1 = 0.f;
-    for (int s = 0; s < p.k_splits; ++s) {
-      v0 += __ldcs(src + s * slice + c0);
-      if (has1) v1 += __ldcs(src + s * slice + c1);
+    // eight slices are requested at a time and then added in slice order
+    for (int s0 = 0; s0 < p.k_splits; s0 += 8) {
+      float a[8], b[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const bool in = s0 + j < p.k_splits;
+        a[j] = in ? __ldcs(src + (s0 + j) * slice + c0) : 0.f;
+        b[j] = (in && has1) ? __ldcs(src + (s0 + j) * slice + c1) : 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (s0 + j < p.k_splits) { v0 += a[j]; v1 += b[j]; }
     }
     epi_pair<EPI>(p, m, n, v0, v1);
   }
