@@ -41,12 +41,13 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 // One CTA per row; the row stays in registers between the two passes (THREADS x REGS float4, i.e.
-// d <= 8192); longer rows are re-read.  Two shapes: 256 threads x 8 for the many rows of a prefill,
-// 1024 x 2 for the up to 16 rows of a decode step (a row then has four times the threads).  The
+// d <= 8192); longer rows are re-read.  Two shapes: 256 threads x 8 when there are many rows,
+// 1024 x 2 for decode steps and short prompts (a row then has four times the threads).  The
 // split-K reduction below uses the same two shapes and the same order of additions, so a row
 // normalised there and a row normalised here agree bit for bit.
 constexpr int RMS_THREADS = 256;
 constexpr int RMS_REGS = 8;
+constexpr int WIDE_ROWS_MAX = 256;     // up to this many rows: 1024 threads per row (too few rows to fill the machine otherwise)
 
 template <int THREADS, int REGS>
 __global__ void __launch_bounds__(THREADS) rmsnorm_kernel(const float* __restrict__ x,
@@ -223,7 +224,7 @@ es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, i
 es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M, int d, float eps,
                            int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches, bool pdl) {
   if (M <= 0) return ES_OK;
-  if (M <= 16)
+  if (M <= WIDE_ROWS_MAX)
     ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset));
   else
     ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset));
@@ -242,7 +243,7 @@ es_status_t launch_splitk_reduce(const float* part, int k_splits, const float* r
                                  const __half* gain, __half* y, float eps, cudaStream_t s, int64_t* launches, bool pdl) {
   if (M <= 0 || N <= 0) return ES_OK;
   if (N % 4 != 0 || ldo % 4 != 0) return fail(ES_ERR_SHAPE, "split-K reduction needs N and the row stride to be multiples of 4");
-  if (M <= 16)
+  if (M <= WIDE_ROWS_MAX)
     ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps));
   else
     ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps));
