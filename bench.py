@@ -318,7 +318,7 @@ def run_ours(args):
                                                 else (hid_host.numel() + S * row_host.numel()) * 4))},
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "linear_stream_kernel", "achieved": kt["gbs"], "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": ("linear_stream_kernel" if Bn <= 2 else "linear_stream_mma_kernel / linear_stream_mma_ks_kernel"), "achieved": kt["gbs"], "peak": peak,
                      "unit": "GB/s", "frac": kt["gbs"] / peak, "peak_source": peak_kind + " copy bandwidth",
                      "launches_timed": kt["launches"], "avg_launch_us": kt["avg_us"],
                      "bytes_per_launch": kt["bytes_per_launch"], "traffic": TRAFFIC_PER_LAUNCH.get(args.workload)},
