@@ -184,13 +184,16 @@ def run_ours(args):
             w["final_norm"], w["lm_head"] = weights["final_norm"], weights["lm_head"]
         return b0, b1, w
 
+    pipelined = n_sh > 1 and args.schedule != "sequential"
+    shard_streams = [torch.cuda.Stream(device=dev) if pipelined else stream for _ in range(n_sh)]
     with torch.cuda.stream(stream):
         shards = []
         for i in range(n_sh):
             b0, b1, w = shard_slice(i)
             shards.append(B.Shard(m, b0, b1, w, max_slots=MB * Bn, max_seq=T + S, max_tokens=Bn * T, max_batch=Bn,
-                                  stream=stream))
+                                  stream=shard_streams[i]))
         sh = shards[0]
+        torch.cuda.synchronize(dev)
 
         def through(mb, first_ids, prefill):
             """one micro-batch through every shard; on one device the hand-over is the handoff view itself"""
@@ -234,6 +237,35 @@ def run_ours(args):
             if events:
                 events[2].record(stream)
 
+        def one_step_pipelined(e2e: bool, events=None):
+            """the same work under a pipelined schedule: one stream per shard, dependencies as events"""
+            from paper_2405_14371_b200.pipeline import ShardPipeline
+
+            pipe = ShardPipeline(shards, slots, Bn, args.schedule)
+            if events:
+                events[0].record(stream)
+            if e2e:
+                ids_dev.copy_(ids_host, non_blocking=True)
+
+            def read_back(p, out):
+                if e2e:
+                    (tok_host.copy_(out[2], non_blocking=True) if wl.has_head else
+                     (hid_host if p.iteration == 0 else row_host).copy_(out[0], non_blocking=True))
+
+            pipe.fork(stream)
+            pipe.prefill(ids_dev, T, on_output=read_back)
+            pipe.join(stream)
+            if events:
+                events[1].record(stream)
+            pipe.fork(stream)
+            pipe.decode(S, forced=None if wl.has_head else (forced_host if e2e else forced_dev), on_output=read_back)
+            pipe.join(stream)
+            if events:
+                events[2].record(stream)
+
+        if pipelined:
+            one_step = one_step_pipelined
+
         for _ in range(args.warmup):
             one_step(False)
             if not args.profile:
@@ -270,14 +302,16 @@ def run_ours(args):
         clocks = sampler.stop() if rank == 0 else None
 
         # dominant kernel: the weight-streaming linear kernel, timed launch by launch with CUDA events
-        sh.es_shard_prefill(ids_dev[0], None, Bn, T, slots[0])
-        src = sh.es_shard_handoff()[2] if (wl.has_head and n_sh == 1) else cur_ids[0]
-        sh.es_shard_set_kernel_timing(True)
-        torch.cuda._sleep(4_000_000)           # let the host run ahead so the event pairs bracket only the kernels
-        for _ in range(min(4, S)):
-            sh.es_shard_decode_step(src, None, Bn, slots[0])
-        t = sh.es_shard_kernel_timing()
-        sh.es_shard_set_kernel_timing(False)
+        torch.cuda.synchronize(dev)
+        with torch.cuda.stream(sh.stream):
+            sh.es_shard_prefill(ids_dev[0], None, Bn, T, slots[0])
+            src = sh.es_shard_handoff()[2] if (wl.has_head and n_sh == 1) else cur_ids[0]
+            sh.es_shard_set_kernel_timing(True)
+            torch.cuda._sleep(4_000_000)           # let the host run ahead so the event pairs bracket only the kernels
+            for _ in range(min(4, S)):
+                sh.es_shard_decode_step(src, None, Bn, slots[0])
+            t = sh.es_shard_kernel_timing()
+            sh.es_shard_set_kernel_timing(False)
         kt = {"gbs": t["bytes"] / (t["ms"] / 1e3) / 1e9, "launches": t["launches"],
               "avg_us": 1e3 * t["ms"] / t["launches"], "bytes_per_launch": t["bytes"] / t["launches"]}
         for x in shards:
@@ -305,7 +339,7 @@ def run_ours(args):
         "config": {"workload": f"{args.workload}: {m.name} layers {wl.layer_begin}-{wl.layer_end - 1}"
                                f"{' +embedding' if wl.has_embedding else ''}{' +head' if wl.has_head else ''}, "
                                f"batch {Bn}, prompt {T}, decode {S}"
-                               + (f", {n_sh} shards in sequence, {MB} micro-batches" if n_sh > 1 or MB > 1 else ""),
+                               + (f", {n_sh} shards in sequence, {MB} micro-batches, schedule {args.schedule}" if n_sh > 1 or MB > 1 else ""),
                    "parallelism": "replicas" if world > 1 else "single",
                    "l2": "no flush: each step streams %.2f GB of weights, far more than the 126 MB L2" % (linear_weight_bytes(wl) / 1e9)},
         "prefill_ms": pre_mean,
@@ -408,6 +442,9 @@ def main():
     ap.add_argument("--workload", default="cfg1", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--schedule", default="no_bubbles", choices=["sequential", "bubbles", "no_bubbles"],
+                    help="micro-batch schedule of a multi-shard workload: one pass at a time, or the paper's two "
+                         "pipelined schedules with one stream per shard")
     ap.add_argument("--profile", action="store_true",
                     help="short run for an ncu capture: 1 warm-up pass, 1 timed pass, no e2e / kernel-timing / CPU legs")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (profile runs)")
