@@ -195,6 +195,10 @@ WORKLOADS = {
     "cfg2_b8": Workload(2, LLAMA2_7B, 0, 32, 8, 512, 256),
     "cfg3": Workload(3, LLAMA2_13B, 0, 40, 1, 256, 128, n_shards=4, micro_batches=8),
     "cfg4": Workload(4, LLAMA2_70B, 0, 40, 16, 1024, 128),
+    # the shape the paper measures on (Sec. "Experimental Setup": 32 prompt tokens, 96 generated, batch 8):
+    # a context run next to the paper's own figures, not one of the parity configurations
+    "paper_7b_b8": Workload(2, LLAMA2_7B, 0, 32, 8, 32, 96),
+    "paper_13b_b8": Workload(3, LLAMA2_13B, 0, 40, 8, 32, 96),
 }
 
 _KINDS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")
