@@ -21,7 +21,8 @@ def _randn(*shape, seed=0, scale=1.0, dtype=torch.float16):
     return (torch.randn(*shape, generator=g) * scale).to(dtype)
 
 
-@pytest.mark.parametrize("M,d", [(1, 256), (5, 4096), (3, 8192), (2, 16384), (7, 688), (0, 256)])
+@pytest.mark.parametrize("M,d", [(1, 256), (5, 4096), (3, 8192), (2, 16384), (7, 688), (0, 256), (256, 4096), (257, 688),
+                                 (300, 8192), (260, 16384)])
 def test_rmsnorm(B, M, d):
     x = _randn(M, d, seed=1, scale=3.0, dtype=torch.float32)
     g = (1 + 0.1 * _randn(d, seed=2, dtype=torch.float32)).half()
