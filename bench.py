@@ -94,33 +94,18 @@ class ClockSampler:
 
 
 def _dist_setup(n_gpus: int):
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if world > 1:
-        import torch.distributed as dist
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    else:
-        torch.cuda.set_device(0)
-    return rank, local, world
+    from paper_2405_14371_b200 import replicas
+    return replicas.setup("nccl")
 
 
 def _barrier(world):
-    if world > 1:
-        import torch.distributed as dist
-        dist.barrier()
-    torch.cuda.synchronize()
+    from paper_2405_14371_b200 import replicas
+    replicas.barrier(world)
 
 
 def _max_over_ranks(x: float, world) -> float:
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([x], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t[0])
-    return x
+    from paper_2405_14371_b200 import replicas
+    return replicas.max_over_ranks(x, world)
 
 
 def algorithmic_decode_bytes(wl, ctx_avg: float) -> float:
