@@ -110,6 +110,17 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
     if (total > 1) issue(b1w0, b1w1);        // both buffers on their way: HBM stays busy while activations are staged
   }
 
+  // RMSNorm gains are weights too: the first XV float4-columns of every thread are fetched before the wait
+  constexpr int XV = 4;                            // covers K <= 4096 with 256 threads; further columns are re-read
+  uint2 gpre[XV];
+  if (NORM) {
+#pragma unroll
+    for (int j = 0; j < XV; ++j) {
+      const int i = threadIdx.x + j * THREADS;
+      gpre[j] = (i < K / 4) ? __ldg(reinterpret_cast<const uint2*>(p.norm_gain) + i) : make_uint2(0, 0);
+    }
+  }
+
   pdl_wait();
 
   // ---- activation rows -> shared memory ----
@@ -122,8 +133,19 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
           continue;
         }
         const float4* xr = reinterpret_cast<const float4*>(p.norm_x + (int64_t)m * p.norm_ldx);
+        float4 xv[XV];                             // this thread's first XV float4-columns stay in registers
+#pragma unroll
+        for (int j = 0; j < XV; ++j) {
+          const int i = threadIdx.x + j * THREADS;
+          xv[j] = (i < K / 4) ? xr[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         float ss = 0.f;
-        for (int i = threadIdx.x; i < K / 4; i += THREADS) {
+#pragma unroll
+        for (int j = 0; j < XV; ++j) {
+          const float4 v = xv[j];
+          if (threadIdx.x + j * THREADS < K / 4) ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
+        for (int i = threadIdx.x + XV * THREADS; i < K / 4; i += THREADS) {
           const float4 v = xr[i];
           ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
         }
@@ -138,7 +160,20 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
         const float inv = 1.0f / sqrtf(tot / (float)K + p.norm_eps);
         const __half2* g2 = reinterpret_cast<const __half2*>(p.norm_gain);
         __half2* dst = reinterpret_cast<__half2*>(a_s + (int64_t)m * K);
-        for (int i = threadIdx.x; i < K / 4; i += THREADS) {
+#pragma unroll
+        for (int j = 0; j < XV; ++j) {
+          const int i = threadIdx.x + j * THREADS;
+          if (i < K / 4) {
+            const float4 v = xv[j];
+            const float2 ga = __half22float2(*reinterpret_cast<const __half2*>(&gpre[j].x));
+            const float2 gb = __half22float2(*reinterpret_cast<const __half2*>(&gpre[j].y));
+            uint2 o;
+            *reinterpret_cast<__half2*>(&o.x) = __floats2half2_rn(v.x * inv * ga.x, v.y * inv * ga.y);
+            *reinterpret_cast<__half2*>(&o.y) = __floats2half2_rn(v.z * inv * gb.x, v.w * inv * gb.y);
+            *reinterpret_cast<uint2*>(dst + 2 * i) = o;
+          }
+        }
+        for (int i = threadIdx.x + XV * THREADS; i < K / 4; i += THREADS) {
           const float4 v = xr[i];
           const float2 ga = __half22float2(g2[2 * i]), gb = __half22float2(g2[2 * i + 1]);
           dst[2 * i] = __floats2half2_rn(v.x * inv * ga.x, v.y * inv * ga.y);
