@@ -104,38 +104,48 @@ __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+// SwiGLU of 32 adjacent columns of row m, packed as 32 fp16 values; dst = where they go (nullptr: row past M).
+// False when the chunk is ragged or unaligned and must take the element-wise path (same for every row).
+__device__ __forceinline__ bool swiglu_chunk32_fast(const LinearParams& p, int n) {
+  return (n + 32 <= p.N) && ((p.ldo & 7) == 0) && ((n & 7) == 0) && (((uintptr_t)p.out_f16 & 15) == 0);
+}
+__device__ __forceinline__ void swiglu_pack32(const LinearParams& p, int m, int n, const float (&g)[32], const float (&u)[32],
+                                              uint4 (&o)[4], __half*& dst) {
+  dst = (m < p.M) ? p.out_f16 + (int64_t)m * p.ldo + n : nullptr;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    o[q].x = pack_half2(silu_f(g[8 * q]) * u[8 * q], silu_f(g[8 * q + 1]) * u[8 * q + 1]);
+    o[q].y = pack_half2(silu_f(g[8 * q + 2]) * u[8 * q + 2], silu_f(g[8 * q + 3]) * u[8 * q + 3]);
+    o[q].z = pack_half2(silu_f(g[8 * q + 4]) * u[8 * q + 4], silu_f(g[8 * q + 5]) * u[8 * q + 5]);
+    o[q].w = pack_half2(silu_f(g[8 * q + 6]) * u[8 * q + 6], silu_f(g[8 * q + 7]) * u[8 * q + 7]);
+  }
+}
+
 __device__ __forceinline__ void epi_swiglu_chunk32(const LinearParams& p, int m, int n, const float (&g)[32],
                                                    const float (&u)[32]) {
   if (m >= p.M || n >= p.N) return;
-  const bool fast = (n + 32 <= p.N) && ((p.ldo & 7) == 0) && ((n & 7) == 0) && (((uintptr_t)p.out_f16 & 15) == 0);
-  if (!fast) {
+  if (!swiglu_chunk32_fast(p, n)) {
 #pragma unroll
     for (int j = 0; j < 32; ++j) epi_swiglu(p, m, n + j, g[j], u[j]);
     return;
   }
-  uint4* dst = reinterpret_cast<uint4*>(p.out_f16 + (int64_t)m * p.ldo + n);
+  uint4 o[4];
+  __half* dst;
+  swiglu_pack32(p, m, n, g, u, o, dst);
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    uint4 o;
-    o.x = pack_half2(silu_f(g[8 * q]) * u[8 * q], silu_f(g[8 * q + 1]) * u[8 * q + 1]);
-    o.y = pack_half2(silu_f(g[8 * q + 2]) * u[8 * q + 2], silu_f(g[8 * q + 3]) * u[8 * q + 3]);
-    o.z = pack_half2(silu_f(g[8 * q + 4]) * u[8 * q + 4], silu_f(g[8 * q + 5]) * u[8 * q + 5]);
-    o.w = pack_half2(silu_f(g[8 * q + 6]) * u[8 * q + 6], silu_f(g[8 * q + 7]) * u[8 * q + 7]);
-    dst[q] = o;
-  }
+  for (int q = 0; q < 4; ++q) reinterpret_cast<uint4*>(dst)[q] = o[q];
 }
 
 // 32 columns of the fused [q | k | v] projection; n is a multiple of 32, so the chunk lies inside one
 // head of one segment (head_dim is 64 or 128).
-__device__ __forceinline__ void epi_qkv_chunk32(const LinearParams& p, int m, int n, const float (&v)[32]) {
-  if (m >= p.M || n >= p.N) return;
+__device__ __forceinline__ bool qkv_chunk32_fast(const LinearParams& p, int n) {
+  return (n + 32 <= p.N) && ((n & 31) == 0) && ((p.hd & 31) == 0);
+}
+// Rotated / rounded values of the chunk as 32 fp16 and their destination (nullptr: nothing to store for this row).
+__device__ __forceinline__ void qkv_pack32(const LinearParams& p, int m, int n, const float (&v)[32], uint4 (&o)[4], __half*& dst) {
+  dst = nullptr;
+  if (m >= p.M) return;
   const int nq = p.Hq * p.hd, nkv = p.Hkv * p.hd;
-  const bool fast = (n + 32 <= p.N) && ((n & 31) == 0) && ((p.hd & 31) == 0);
-  if (!fast) {
-#pragma unroll
-    for (int j = 0; j < 32; j += 2) epi_qkv_pair(p, m, n + j, v[j], v[j + 1]);
-    return;
-  }
   const int b = m / p.T;
   const int slot = p.slots[b];
   const int pos = p.is_decode ? p.ctx_len[slot] : (m - b * p.T);
@@ -143,38 +153,150 @@ __device__ __forceinline__ void epi_qkv_chunk32(const LinearParams& p, int m, in
   const bool is_q = n < nq, is_k = !is_q && n < nq + nkv;
   const int local = is_q ? n : (is_k ? n - nq : n - nq - nkv);
   const int head = local / p.hd, c0 = local - head * p.hd;
-  __half* dst;
   if (is_q) {
     dst = p.out_f16 + (int64_t)m * nq + n;
   } else {
     const int page = p.block_table[(int64_t)slot * p.pages_per_slot + pos / p.P];
     dst = (is_k ? p.k_cache : p.v_cache) + (((int64_t)page * p.Hkv + head) * p.P + (pos % p.P)) * p.hd + c0;
   }
-  uint4* d4 = reinterpret_cast<uint4*>(dst);
   if (is_q || is_k) {
     const float4* cs4 = reinterpret_cast<const float4*>(p.rope_cos + (int64_t)pos * (p.hd / 2) + c0 / 2);
     const float4* sn4 = reinterpret_cast<const float4*>(p.rope_sin + (int64_t)pos * (p.hd / 2) + c0 / 2);
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const float4 cs = cs4[q], sn = sn4[q];
-      uint4 o;
-      o.x = pack_half2(v[8 * q] * cs.x - v[8 * q + 1] * sn.x, v[8 * q] * sn.x + v[8 * q + 1] * cs.x);
-      o.y = pack_half2(v[8 * q + 2] * cs.y - v[8 * q + 3] * sn.y, v[8 * q + 2] * sn.y + v[8 * q + 3] * cs.y);
-      o.z = pack_half2(v[8 * q + 4] * cs.z - v[8 * q + 5] * sn.z, v[8 * q + 4] * sn.z + v[8 * q + 5] * cs.z);
-      o.w = pack_half2(v[8 * q + 6] * cs.w - v[8 * q + 7] * sn.w, v[8 * q + 6] * sn.w + v[8 * q + 7] * cs.w);
-      d4[q] = o;
+      o[q].x = pack_half2(v[8 * q] * cs.x - v[8 * q + 1] * sn.x, v[8 * q] * sn.x + v[8 * q + 1] * cs.x);
+      o[q].y = pack_half2(v[8 * q + 2] * cs.y - v[8 * q + 3] * sn.y, v[8 * q + 2] * sn.y + v[8 * q + 3] * cs.y);
+      o[q].z = pack_half2(v[8 * q + 4] * cs.z - v[8 * q + 5] * sn.z, v[8 * q + 4] * sn.z + v[8 * q + 5] * cs.z);
+      o[q].w = pack_half2(v[8 * q + 6] * cs.w - v[8 * q + 7] * sn.w, v[8 * q + 6] * sn.w + v[8 * q + 7] * cs.w);
     }
   } else {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      uint4 o;
-      o.x = pack_half2(v[8 * q], v[8 * q + 1]);
-      o.y = pack_half2(v[8 * q + 2], v[8 * q + 3]);
-      o.z = pack_half2(v[8 * q + 4], v[8 * q + 5]);
-      o.w = pack_half2(v[8 * q + 6], v[8 * q + 7]);
-      d4[q] = o;
+      o[q].x = pack_half2(v[8 * q], v[8 * q + 1]);
+      o[q].y = pack_half2(v[8 * q + 2], v[8 * q + 3]);
+      o[q].z = pack_half2(v[8 * q + 4], v[8 * q + 5]);
+      o[q].w = pack_half2(v[8 * q + 6], v[8 * q + 7]);
     }
   }
+}
+
+__device__ __forceinline__ void epi_qkv_chunk32(const LinearParams& p, int m, int n, const float (&v)[32]) {
+  if (m >= p.M || n >= p.N) return;
+  if (!qkv_chunk32_fast(p, n)) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 2) epi_qkv_pair(p, m, n + j, v[j], v[j + 1]);
+    return;
+  }
+  uint4 o[4];
+  __half* dst;
+  qkv_pack32(p, m, n, v, o, dst);
+  if (dst == nullptr) return;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) reinterpret_cast<uint4*>(dst)[q] = o[q];
+}
+
+// ---- the same chunks stored through a per-warp shared-memory tile -------------------------------
+// A thread that owns 32 adjacent columns of ONE row stores 16 bytes into a row of its own: 32 rows per
+// instruction, half a 32-byte sector each.  The variants below are called by a whole warp whose lane l owns
+// row m0 + l; they pass the chunk through `stage` (EPI_STAGE_BYTES of shared memory private to the warp) so
+// that every store instruction writes whole 64- or 128-byte row segments.  The arithmetic is that of the
+// functions above.
+constexpr int EPI_STAGE_BYTES = 32 * 36 * 4 + 32 * 8;   // a 32 x 32 fp32 tile with 36-word rows, then one pointer per row
+
+// out[m, n .. n+31] = v (+ res[m, n .. n+31]) for the 32 rows m0 + lane; out / res row stride ldo; rows >= M and
+// columns >= N are skipped.  res may alias out.
+__device__ __forceinline__ void f32_chunk32_staged(float* out, const float* res, int64_t ldo, int M, int N, int m0, int n,
+                                                   const float (&v)[32], unsigned char* stage, int lane) {
+  if (n >= N) return;
+  const bool fast = (n + 32 <= N) && ((ldo & 3) == 0) && ((n & 3) == 0) &&
+                    (((uintptr_t)out & 15) == 0) && (res == nullptr || ((uintptr_t)res & 15) == 0);
+  if (!fast) {                                    // same decision in every lane: element-wise, one row per thread
+    const int m = m0 + lane;
+    if (m < M) {
+      const int64_t o = (int64_t)m * ldo + n;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (n + j < N) out[o + j] = (res != nullptr) ? v[j] + res[o + j] : v[j];
+    }
+    return;
+  }
+  // residual first: eight independent 16-byte loads in flight while the tile turns around.  A thread reads and
+  // writes exactly the same elements, so hoisting the loads above the stores is safe when res aliases out.
+  const int cq = (lane & 7) * 4;                  // eight lanes cover the 128 bytes of one row
+  float4 rv[8];
+  if (res != nullptr) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int m = m0 + i * 4 + (lane >> 3);
+      rv[i] = (m < M) ? __ldcs(reinterpret_cast<const float4*>(res + (int64_t)m * ldo + n + cq)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  }
+  float* tile = reinterpret_cast<float*>(stage);
+#pragma unroll
+  for (int q = 0; q < 8; ++q)
+    *reinterpret_cast<float4*>(tile + lane * 36 + 4 * q) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int rr = i * 4 + (lane >> 3);
+    const int m = m0 + rr;
+    if (m < M) {
+      float4 x = *reinterpret_cast<const float4*>(tile + rr * 36 + cq);
+      if (res != nullptr) x = make_float4(x.x + rv[i].x, x.y + rv[i].y, x.z + rv[i].z, x.w + rv[i].w);
+      *reinterpret_cast<float4*>(out + (int64_t)m * ldo + n + cq) = x;
+    }
+  }
+  __syncwarp();
+}
+
+__device__ __forceinline__ void epi_f32_chunk32_staged(const LinearParams& p, int m0, int n, const float (&v)[32],
+                                                       unsigned char* stage, int lane) {
+  f32_chunk32_staged(p.out_f32, p.res, p.ldo, p.M, p.N, m0, n, v, stage, lane);
+}
+
+// 32 fp16 values per row (o) to dst (nullptr = skip the row): four lanes cover the 64 bytes of one row
+__device__ __forceinline__ void rows16_store_staged(__half* dst, const uint4 (&o)[4], unsigned char* stage, int lane) {
+  uint4* tile = reinterpret_cast<uint4*>(stage);                      // rows of 5 x 16 bytes (4 used)
+  unsigned long long* rowptr = reinterpret_cast<unsigned long long*>(stage + 32 * 36 * 4);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) tile[lane * 5 + q] = o[q];
+  rowptr[lane] = reinterpret_cast<unsigned long long>(dst);
+  __syncwarp();
+  const int piece = lane >> 3;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int rr = i * 8 + (lane & 7);
+    __half* d = reinterpret_cast<__half*>(rowptr[rr]);
+    if (d != nullptr) reinterpret_cast<uint4*>(d)[piece] = tile[rr * 5 + piece];
+  }
+  __syncwarp();
+}
+
+__device__ __forceinline__ void epi_swiglu_chunk32_staged(const LinearParams& p, int m0, int n, const float (&g)[32],
+                                                          const float (&u)[32], unsigned char* stage, int lane) {
+  if (n >= p.N) return;
+  if (!swiglu_chunk32_fast(p, n)) {
+    epi_swiglu_chunk32(p, m0 + lane, n, g, u);
+    return;
+  }
+  uint4 o[4];
+  __half* dst;
+  swiglu_pack32(p, m0 + lane, n, g, u, o, dst);
+  rows16_store_staged(dst, o, stage, lane);
+}
+
+__device__ __forceinline__ void epi_qkv_chunk32_staged(const LinearParams& p, int m0, int n, const float (&v)[32],
+                                                       unsigned char* stage, int lane) {
+  if (n >= p.N) return;
+  if (!qkv_chunk32_fast(p, n)) {
+    epi_qkv_chunk32(p, m0 + lane, n, v);
+    return;
+  }
+  uint4 o[4];
+  __half* dst;
+  qkv_pack32(p, m0 + lane, n, v, o, dst);
+  rows16_store_staged(dst, o, stage, lane);
 }
 
 // Pointer to row n (virtual, over the concatenated segments) of the weight; nullptr past N.

@@ -31,6 +31,7 @@ es_status_t fail(es_status_t st, const char* fmt, ...);
 struct Tunables {
   int stream_deep;   // ES_STREAM_DEEP: weight-streaming kernel chunk depth, 1 = 4 KB per warp per buffer (default), 0 = 2 KB
   int tc_pair;       // ES_TC_PAIR: CTA-pair tensor-core kernel for large prefill products (1, default) or never (0)
+  int tc_pair_wide;  // ES_TC_PAIR_WIDE: 256 x 512 pair tiles: chosen per shape (1, default), never (0), always (2)
   int pdl;           // ES_PDL: programmatic dependent launch in decode steps (1, default) or plain stream order (0)
   int attn_mma;      // ES_ATTN_MMA: tensor-core decode attention for launches with many items (1, default) or never (0)
   int split_k;       // ES_SPLIT_K: split-K for the O and down projections of short prefills (1, default) or never (0)
@@ -85,6 +86,8 @@ struct LinearParams {
   // sums go to part[k_splits, M, columns] and a second kernel finishes the product
   int k_splits;
   float* part;
+  // CTA-pair tensor-core kernel: accumulators per tile, 1 = 256 x 256 tiles, 2 = 256 x 512 tiles, 0 = chosen per shape
+  int pair_nacc;
 };
 
 // Kernel families.  Each returns after enqueuing; `launches` is incremented per kernel launched.

@@ -5,7 +5,8 @@
 // stages with TMA (128-byte-swizzled K-major tiles of A and W, 64 K-elements deep); a second
 // elected thread issues tcgen05.mma (M=128, N=BN, K=16, fp16 in, fp32 accumulate) into a TMEM
 // accumulator and releases each stage with tcgen05.commit; four epilogue warps read the
-// accumulator back with tcgen05.ld (each warp its own 32-lane quarter) and run the epilogue.
+// accumulator back with tcgen05.ld (each warp its own 32-lane quarter) and run the epilogue, passing
+// each 32-column chunk through a shared-memory tile so that global accesses cover whole row segments.
 // Ragged M, N and K are handled by TMA zero fill on the way in and by guards on the way out.
 // Split-K (plain / residual epilogue only): when a product has too few output tiles for the machine
 // (short prompts: M = 128..512 against N = d_model), the K range is cut into k_splits slices, every
@@ -37,7 +38,7 @@ template <int BN> struct TileCfg {
   static constexpr int STAGES = (200 * 1024) / (A_STAGE_BYTES + B_STAGE_BYTES) > 8 ? 8 : (200 * 1024) / (A_STAGE_BYTES + B_STAGE_BYTES);
   static constexpr int TMEM_COLS = BN;                                       // one accumulator buffer
   static constexpr int TMEM_ALLOC = 2 * BN <= 64 ? 64 : 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512;   // two buffers, power of two
-  static constexpr size_t SMEM = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 256;
+  static constexpr size_t SMEM = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 4 * EPI_STAGE_BYTES + 256;
 };
 
 struct TmapSet {
@@ -45,20 +46,6 @@ struct TmapSet {
   CUtensorMap w[3];
 };
 static_assert(sizeof(TmapSet) == sizeof(TcMaps), "TcMaps must hold four tensor maps");
-
-// Raw accumulator columns [n, n + 32) of one row into the split-K workspace row `row` (N % 4 == 0).
-__device__ __forceinline__ void partial_chunk32(float* row, bool row_valid, int n, int N, const float (&v)[32]) {
-  if (!row_valid || n >= N) return;
-  if (n + 32 <= N) {
-    float4* dst = reinterpret_cast<float4*>(row + n);
-#pragma unroll
-    for (int q = 0; q < 8; ++q) dst[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
-  } else {
-#pragma unroll
-    for (int j = 0; j < 32; ++j)
-      if (n + j < N) row[n + j] = v[j];
-  }
-}
 
 // ---- the kernel --------------------------------------------------------------------------------
 // Persistent: a CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The accumulator is double
@@ -76,7 +63,8 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* a_tiles = smem;
   unsigned char* b_tiles = smem + (size_t)STAGES * A_STAGE_BYTES;
-  uint64_t* bars = (uint64_t*)(b_tiles + (size_t)STAGES * Cfg::B_STAGE_BYTES);
+  unsigned char* epi_stage = b_tiles + (size_t)STAGES * Cfg::B_STAGE_BYTES;   // one store-staging tile per epilogue warp
+  uint64_t* bars = (uint64_t*)(epi_stage + 4 * EPI_STAGE_BYTES);
   uint64_t* full_bar = bars;
   uint64_t* empty_bar = bars + STAGES;
   uint64_t* acc_full = bars + 2 * STAGES;        // [2]
@@ -210,15 +198,16 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
       int m0, n0;
       const int ks = tile / mn_tiles;
       tile_origin(tile - ks * mn_tiles, m0, n0);
-      const int m = m0 + quarter * 32 + lane;
+      const int mw = m0 + quarter * 32;              // row of lane 0
       const uint32_t trow = tmem_base + (uint32_t)(buf * ACC_COLS) + ((uint32_t)(quarter * 32) << 16);
+      unsigned char* stage = epi_stage + (size_t)(warp - 2) * EPI_STAGE_BYTES;
       if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
         for (int c = 0; c < BN_OUT; c += 32) {
           float g[32], u[32];
           tmem_ld32(trow + c, g);
           tmem_ld32(trow + BN_OUT + c, u);
-          epi_swiglu_chunk32(p, m, n0 + c, g, u);
+          epi_swiglu_chunk32_staged(p, mw, n0 + c, g, u, stage, lane);
         }
       } else {
 #pragma unroll 1
@@ -226,10 +215,11 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
           float v[32];
           tmem_ld32(trow + c, v);
           if (EPI == EPI_F32) {
-            if (k_splits > 1) partial_chunk32(p.part + ((int64_t)ks * p.M + m) * p.N, m < p.M, n0 + c, p.N, v);
-            else epi_f32_chunk32(p, m, n0 + c, v);
+            // split-K: the raw accumulator goes to slice ks of the workspace [k_splits, M, N]
+            if (k_splits > 1) f32_chunk32_staged(p.part + (int64_t)ks * p.M * p.N, nullptr, p.N, p.M, p.N, mw, n0 + c, v, stage, lane);
+            else epi_f32_chunk32_staged(p, mw, n0 + c, v, stage, lane);
           } else {
-            epi_qkv_chunk32(p, m, n0 + c, v);
+            epi_qkv_chunk32_staged(p, mw, n0 + c, v, stage, lane);
           }
         }
       }

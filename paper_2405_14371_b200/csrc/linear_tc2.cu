@@ -7,6 +7,13 @@
 // operand traffic per flop of the single-CTA 128 x 256 tile and a third less staging per K block,
 // so the ring is deeper in time and the tensor pipe stalls less.  Persistent pairs walk the tiles;
 // the accumulator is double buffered in TMEM (2 x 256 columns) so epilogues overlap the next tile.
+// With NACC = 2 a pair computes a 256 x 512 tile instead (two 256-column accumulators that share the A
+// rows; each CTA stages 128 rows of A and 256 rows of W per K block): a quarter fewer operand bytes per
+// flop pulled through L2 — on a power-capped part those transfers cost about as much energy as the MMAs
+// themselves — at the price of an epilogue that no longer overlaps the MMAs (all 512 TMEM columns hold
+// one tile), so the loads of the next tile are all that runs beside it.
+// Epilogue warps pass every 32-column chunk through a small shared-memory tile so that global stores
+// (and residual loads) cover whole row segments instead of 16 bytes in each of 32 rows.
 // Barrier traffic: both CTAs' TMA bytes are counted on the first CTA's "full" barrier; the MMA
 // issuer's commits arrive on the "empty" / "accumulator ready" barriers of both CTAs; both CTAs'
 // epilogue warps arrive on the first CTA's "accumulator free" barrier.  Waits are bounded.
@@ -26,10 +33,11 @@ constexpr int BN2 = 256;
 constexpr int BK2 = 64, UK2 = 16;
 constexpr int W_BOX = 32;
 constexpr int T2_THREADS = 192;
-constexpr int STAGES2 = 6;
 constexpr int A_BYTES2 = BM2 * BK2 * 2;          // 16 KB
-constexpr int B_BYTES2 = (BN2 / 2) * BK2 * 2;    // this CTA's half of the W tile, 16 KB
-constexpr size_t SMEM2 = 1024 + (size_t)STAGES2 * (A_BYTES2 + B_BYTES2) + 256;
+constexpr int B_BYTES2 = (BN2 / 2) * BK2 * 2;    // this CTA's half of one 256-row W tile, 16 KB
+constexpr int RING_BYTES2 = 192 * 1024;          // 6 stages of 32 KB (NACC = 1) or 4 of 48 KB (NACC = 2)
+constexpr int MAX_STAGES2 = 6;
+constexpr size_t SMEM2 = 1024 + (size_t)RING_BYTES2 + 4 * EPI_STAGE_BYTES + 256;
 
 struct TmapSet2 {
   CUtensorMap a;
@@ -37,22 +45,27 @@ struct TmapSet2 {
 };
 static_assert(sizeof(TmapSet2) == sizeof(TcMaps), "TcMaps must hold four tensor maps");
 
-template <int EPI>
+template <int EPI, int NACC>
 __global__ void __launch_bounds__(T2_THREADS, 1)
 linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, int* status, int m_tiles, int n_tiles) {
-  constexpr int BN_OUT = (EPI == EPI_SWIGLU) ? BN2 / 2 : BN2;
+  constexpr int ACC_OUT = (EPI == EPI_SWIGLU) ? BN2 / 2 : BN2;   // output columns of one accumulator
+  constexpr int BN_OUT = NACC * ACC_OUT;                           // output columns of a tile
+  constexpr int STAGE_BYTES = A_BYTES2 + NACC * B_BYTES2;
+  constexpr int STAGES2 = RING_BYTES2 / STAGE_BYTES;
+  constexpr int NBUF = 2 / NACC;                                   // accumulator buffers in the 512 TMEM columns
+  static_assert(STAGES2 <= MAX_STAGES2 && STAGES2 * STAGE_BYTES == RING_BYTES2, "ring layout");
   pdl_launch_dependents();
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  unsigned char* a_tiles = smem;
-  unsigned char* b_tiles = smem + (size_t)STAGES2 * A_BYTES2;
-  uint64_t* bars = (uint64_t*)(b_tiles + (size_t)STAGES2 * B_BYTES2);
-  uint64_t* full_bar = bars;                     // used in rank 0 only
-  uint64_t* empty_bar = bars + STAGES2;          // one copy per CTA
-  uint64_t* acc_full = bars + 2 * STAGES2;       // [2], one copy per CTA
-  uint64_t* acc_empty = bars + 2 * STAGES2 + 2;  // [2], used in rank 0 only (8 arrivals)
-  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * STAGES2 + 4);
+  unsigned char* ring = smem;                    // stage s: A tile, then NACC half W tiles
+  unsigned char* epi_stage = smem + RING_BYTES2;
+  uint64_t* bars = (uint64_t*)(epi_stage + 4 * EPI_STAGE_BYTES);
+  uint64_t* full_bar = bars;                         // used in rank 0 only
+  uint64_t* empty_bar = bars + MAX_STAGES2;          // one copy per CTA
+  uint64_t* acc_full = bars + 2 * MAX_STAGES2;       // [2], one copy per CTA
+  uint64_t* acc_empty = bars + 2 * MAX_STAGES2 + 2;  // [2], used in rank 0 only (8 arrivals)
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * MAX_STAGES2 + 4);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -101,28 +114,37 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
       for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
         int m0, n0;
         tile_origin(tile, m0, n0);
-        const CUtensorMap* wmap;
-        int wrow;
-        if (EPI == EPI_SWIGLU) {
-          wmap = rank ? &maps.w[1] : &maps.w[0];   // rank 0 stages gate rows, rank 1 the up rows of the same columns
-          wrow = n0;
-        } else {
-          int n = n0, seg = 0;
-          while (seg < 2 && n >= p.seg_rows[seg]) { n -= p.seg_rows[seg]; ++seg; }
-          wmap = &maps.w[seg];
-          wrow = n + (int)rank * (BN2 / 2);
+        // W rows this CTA stages for accumulator a: SwiGLU - rank 0 the gate rows, rank 1 the up rows of the same
+        // 128 columns; otherwise rows [r * 128, r * 128 + 128) of the accumulator's 256 columns, inside one segment
+        const CUtensorMap* wmap[NACC];
+        int wrow[NACC];
+#pragma unroll
+        for (int a = 0; a < NACC; ++a) {
+          if (EPI == EPI_SWIGLU) {
+            wmap[a] = rank ? &maps.w[1] : &maps.w[0];
+            wrow[a] = n0 + a * ACC_OUT;
+          } else {
+            int n = n0 + a * ACC_OUT, seg = 0;
+            while (seg < 2 && n >= p.seg_rows[seg]) { n -= p.seg_rows[seg]; ++seg; }
+            wmap[a] = &maps.w[seg];
+            wrow[a] = n + (int)rank * (BN2 / 2);
+          }
         }
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % STAGES2;
           const uint32_t ph = (it / STAGES2) & 1;
           if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, abort_flag, status, 31)) { ok = false; break; }
           const uint32_t fb = smem_u32(&full_bar[s]);
-          if (rank == 0) mbar_expect_tx(fb, 2 * (A_BYTES2 + B_BYTES2));     // both CTAs' bytes land on this barrier
-          tma_load_2d_pair(smem_u32(a_tiles + (size_t)s * A_BYTES2), &maps.a, kb * BK2, m0 + (int)rank * BM2, fb);
-          const uint32_t bdst = smem_u32(b_tiles + (size_t)s * B_BYTES2);
+          if (rank == 0) mbar_expect_tx(fb, 2 * STAGE_BYTES);                 // both CTAs' bytes land on this barrier
+          const uint32_t sdst = smem_u32(ring + (size_t)s * STAGE_BYTES);
+          tma_load_2d_pair(sdst, &maps.a, kb * BK2, m0 + (int)rank * BM2, fb);
 #pragma unroll
-          for (int i = 0; i < N_LOADS; ++i)
-            tma_load_2d_pair(bdst + i * W_BOX * (BK2 * 2), wmap, kb * BK2, wrow + i * W_BOX, fb);
+          for (int a = 0; a < NACC; ++a) {
+            const uint32_t bdst = sdst + A_BYTES2 + a * B_BYTES2;
+#pragma unroll
+            for (int i = 0; i < N_LOADS; ++i)
+              tma_load_2d_pair(bdst + i * W_BOX * (BK2 * 2), wmap[a], kb * BK2, wrow[a] + i * W_BOX, fb);
+          }
         }
       }
     }
@@ -133,8 +155,8 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
       int it = 0, local = 0;
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += n_pairs, ++local) {
-        const int buf = local & 1;
-        const uint32_t use = (uint32_t)(local >> 1);
+        const int buf = local % NBUF;
+        const uint32_t use = (uint32_t)(local / NBUF);
         ok = mbar_wait(smem_u32(&acc_empty[buf]), (use & 1) ^ 1, abort_flag, status, 35);
         if (!ok) break;
         tc_fence_after();
@@ -145,12 +167,16 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
           ok = mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag, status, 32);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t a0 = smem_u32(a_tiles + (size_t)s * A_BYTES2);
-          const uint32_t b0 = smem_u32(b_tiles + (size_t)s * B_BYTES2);
+          const uint32_t a0 = smem_u32(ring + (size_t)s * STAGE_BYTES);
+          const uint32_t b0 = a0 + A_BYTES2;
 #pragma unroll
-          for (int k = 0; k < BK2 / UK2; ++k)
-            umma_f16_pair(tacc, umma_desc_sw128(a0 + k * UK2 * 2), umma_desc_sw128(b0 + k * UK2 * 2), idesc,
-                          (kb > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < BK2 / UK2; ++k) {
+            const uint64_t adesc = umma_desc_sw128(a0 + k * UK2 * 2);
+#pragma unroll
+            for (int a = 0; a < NACC; ++a)
+              umma_f16_pair(tacc + (uint32_t)(a * BN2), adesc, umma_desc_sw128(b0 + a * B_BYTES2 + k * UK2 * 2), idesc,
+                            (kb > 0 || k > 0) ? 1u : 0u);
+          }
           umma_commit_pair(smem_u32(&empty_bar[s]));
         }
         if (ok) umma_commit_pair(smem_u32(&acc_full[buf]));
@@ -159,31 +185,37 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
   } else {
     // ---- epilogue warps (both CTAs): own 128 rows x 256 columns ----
     const int quarter = warp & 3;
+    unsigned char* stage = epi_stage + (size_t)(warp - 2) * EPI_STAGE_BYTES;
     int local = 0;
     for (int tile = pair; tile < num_tiles; tile += n_pairs, ++local) {
-      const int buf = local & 1;
-      const uint32_t use = (uint32_t)(local >> 1);
+      const int buf = local % NBUF;
+      const uint32_t use = (uint32_t)(local / NBUF);
       if (!mbar_wait(smem_u32(&acc_full[buf]), use & 1, abort_flag, status, 33)) break;
       tc_fence_after();
       int m0, n0;
       tile_origin(tile, m0, n0);
-      const int m = m0 + (int)rank * BM2 + quarter * 32 + lane;
+      const int mw = m0 + (int)rank * BM2 + quarter * 32;          // row of lane 0
       const uint32_t trow = tmem_base + (uint32_t)(buf * BN2) + ((uint32_t)(quarter * 32) << 16);
-      if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
-        for (int c = 0; c < BN_OUT; c += 32) {
-          float g[32], u[32];
-          tmem_ld32(trow + c, g);
-          tmem_ld32(trow + BN_OUT + c, u);
-          epi_swiglu_chunk32(p, m, n0 + c, g, u);
-        }
-      } else {
+      for (int a = 0; a < NACC; ++a) {
+        const uint32_t tacc = trow + (uint32_t)(a * BN2);
+        const int na = n0 + a * ACC_OUT;
+        if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
-        for (int c = 0; c < BN2; c += 32) {
-          float v[32];
-          tmem_ld32(trow + c, v);
-          if (EPI == EPI_F32) epi_f32_chunk32(p, m, n0 + c, v);
-          else epi_qkv_chunk32(p, m, n0 + c, v);
+          for (int c = 0; c < ACC_OUT; c += 32) {
+            float g[32], u[32];
+            tmem_ld32(tacc + c, g);
+            tmem_ld32(tacc + ACC_OUT + c, u);
+            epi_swiglu_chunk32_staged(p, mw, na + c, g, u, stage, lane);
+          }
+        } else {
+#pragma unroll 1
+          for (int c = 0; c < BN2; c += 32) {
+            float v[32];
+            tmem_ld32(tacc + c, v);
+            if (EPI == EPI_F32) epi_f32_chunk32_staged(p, mw, na + c, v, stage, lane);
+            else epi_qkv_chunk32_staged(p, mw, na + c, v, stage, lane);
+          }
         }
       }
       tc_fence_before();
@@ -203,11 +235,11 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
   }
 }
 
-template <int EPI>
+template <int EPI, int NACC>
 es_status_t launch_pair(const TmapSet2& maps, const LinearParams& p, int* status, cudaStream_t s, bool pdl) {
-  constexpr int out = (EPI == EPI_SWIGLU) ? BN2 / 2 : BN2;
+  constexpr int out = NACC * ((EPI == EPI_SWIGLU) ? BN2 / 2 : BN2);
   const int m_tiles = (p.M + 2 * BM2 - 1) / (2 * BM2), n_tiles = (p.N + out - 1) / out;
-  auto kern = linear_tc2_kernel<EPI>;
+  auto kern = linear_tc2_kernel<EPI, NACC>;
   static bool configured = false;
   if (!configured) {
     ES_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM2));
@@ -240,6 +272,28 @@ es_status_t launch_pair(const TmapSet2& maps, const LinearParams& p, int* status
   return ES_OK;
 }
 
+// Accumulators per tile: the 256 x 512 tile moves a quarter fewer operand bytes per flop but cannot hide its
+// epilogue and quantises into coarser waves.  Measured against the 256 x 256 tile (same launch, 16384 or 8192
+// rows): K = 4096 +-2 %, K = 8192 +7 % (+1 % with a residual to read), K = 28672 +13 % (+10 %).  It is taken
+// for K >= 8192 when its waves, discounted for the traffic saved, come out shorter.
+int pair_nacc(const LinearParams& p, int epi) {
+  if (p.pair_nacc == 1 || p.pair_nacc == 2) return p.pair_nacc;
+  const int force = tunables().tc_pair_wide;
+  if (force == 0) return 1;
+  if (force == 2) return 2;
+  if (p.K < 8192) return 1;
+  const int out = (epi == EPI_SWIGLU) ? BN2 / 2 : BN2;
+  const long long mt = (p.M + 2 * BM2 - 1) / (2 * BM2);
+  const long long t1 = mt * ((p.N + out - 1) / out), t2 = mt * ((p.N + 2 * out - 1) / (2 * out));
+  const long long w1 = (t1 + 73) / 74, w2 = 2 * ((t2 + 73) / 74);
+  return (w2 * 92 < w1 * 100) ? 2 : 1;
+}
+
+template <int EPI>
+es_status_t launch_pair_epi(const TmapSet2& maps, const LinearParams& p, int* status, cudaStream_t s, bool pdl) {
+  return pair_nacc(p, EPI) == 2 ? launch_pair<EPI, 2>(maps, p, status, s, pdl) : launch_pair<EPI, 1>(maps, p, status, s, pdl);
+}
+
 }  // namespace
 
 // The pair kernel pays off when there are enough 256 x 256 tiles to keep every pair busy.
@@ -263,9 +317,9 @@ es_status_t launch_linear_tc2(const LinearParams& p, int epi, cudaStream_t s, in
   const TmapSet2& t = *reinterpret_cast<const TmapSet2*>(maps);
   es_status_t st;
   switch (epi) {
-    case EPI_F32: st = launch_pair<EPI_F32>(t, p, status_word, s, pdl); break;
-    case EPI_SWIGLU: st = launch_pair<EPI_SWIGLU>(t, p, status_word, s, pdl); break;
-    case EPI_QKV: st = launch_pair<EPI_QKV>(t, p, status_word, s, pdl); break;
+    case EPI_F32: st = launch_pair_epi<EPI_F32>(t, p, status_word, s, pdl); break;
+    case EPI_SWIGLU: st = launch_pair_epi<EPI_SWIGLU>(t, p, status_word, s, pdl); break;
+    case EPI_QKV: st = launch_pair_epi<EPI_QKV>(t, p, status_word, s, pdl); break;
     default: return fail(ES_ERR_INVALID_ARG, "unknown epilogue %d", epi);
   }
   if (st == ES_OK && launches) ++*launches;

@@ -40,7 +40,7 @@ static int env_int(const char* name, int dflt) {
 }
 
 const Tunables& tunables() {
-  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_PDL", 1), env_int("ES_ATTN_MMA", 1), env_int("ES_SPLIT_K", 1)};
+  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_TC_PAIR_WIDE", 1), env_int("ES_PDL", 1), env_int("ES_ATTN_MMA", 1), env_int("ES_SPLIT_K", 1)};
   return t;
 }
 
@@ -932,7 +932,9 @@ es_status_t es_op_linear(const void* A, const void* W, const float* R, float* C,
     case 2: return launch_linear_stream(p, EPI_F32, st, nullptr);
     case 3: return launch_linear_reference(p, EPI_F32, st, nullptr);
     case 5:
+    case 6:
       if (!linear_tc2_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "pair kernel does not take this shape");
+      p.pair_nacc = path == 5 ? 1 : 2;
       return launch_linear_tc2(p, EPI_F32, st, nullptr, nullptr);
     case 4:
       if (!linear_stream_mma_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "tensor-core streaming kernel does not take this shape");

@@ -89,15 +89,17 @@ def test_linear_streaming_tensor_core(B, M, N, K):
 
 @pytest.mark.parametrize("M,N,K", [(2048, 4096, 1024), (1100, 5000, 520), (4096, 4096, 4096), (512, 12288, 4096)])
 def test_linear_tensor_core_cta_pairs(B, M, N, K):
-    """cta_group::2 kernel: 256 x 256 tiles on CTA pairs, ragged M / N / K, agreement with the single-CTA kernel."""
+    """cta_group::2 kernel: 256 x 256 and 256 x 512 tiles on CTA pairs, ragged M / N / K, agreement with the single-CTA kernel."""
     A = _randn(M, K, seed=19)
     W = _randn(N, K, seed=20, scale=0.05)
     R = _randn(M, N, seed=21, dtype=torch.float32)
-    got = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), 5)
     ref = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), 1)
     want = A.double() @ W.double().T + R.double()
-    assert rel_err(got, want) < 5e-5
-    assert rel_err(got, ref) < 1e-5
+    for path in (5, 6):                          # 256 x 256 and 256 x 512 tiles
+        got = B.es_op_linear(A.cuda(), W.cuda(), R.cuda(), path)
+        assert rel_err(got, want) < 5e-5
+        assert rel_err(got, ref) < 1e-5
+    assert rel_err(B.es_op_linear(A.cuda(), W.cuda(), None, 6), A.double() @ W.double().T) < 5e-5
 
 
 @pytest.mark.parametrize("M,N,K,S", [(128, 4096, 4096, 0), (128, 4096, 11008, 0), (256, 5120, 5120, 0), (100, 260, 1096, 3),
