@@ -1,14 +1,23 @@
 // Causal prefill attention on the tensor cores of sm_100a (tcgen05 / TMEM / TMA).
 //
-// One CTA handles 128 query rows of one (sequence, head).  Q stays resident in shared memory; K and
-// V arrive 64 keys at a time through a two-stage TMA ring (a 64-key tile is one KV page, or 64 rows
-// of a contiguous K / V matrix).  Per KV tile:
-//   S = Q K^T      tcgen05.mma, M=128 queries, N=64 keys, K=head_dim, fp32 in TMEM columns [0,64)
+// One CTA handles 128 query rows of one (sequence, head); two CTAs share an SM, so that one's softmax
+// runs beside the other's MMAs.  Q stays resident in shared memory; K and V arrive 64 keys at a time
+// through a two-stage TMA ring (a 64-key tile is one KV page, or 64 rows of a contiguous K / V matrix).
+// Per KV tile j:
+//   S = Q K^T      tcgen05.mma, M=128 queries, N=64 keys, K=head_dim, fp32 in TMEM; S has two buffers
+//                  (columns [0,64) and [64,128)) and S(j+1) is issued before the softmax of tile j has
+//                  finished, so the softmax warps never wait for the tensor cores in steady state
 //   softmax        four warps, one query row per thread (the thread holds its whole score row, so
 //                  the row maximum and sum need no cross-lane traffic): running max / sum, P in fp16
-//                  written to shared memory in the 128-byte-swizzled K-major layout
-//   O = O*a + P V  the accumulator lives in TMEM columns [64, 64+head_dim); it is rescaled in place
-//                  (tcgen05.ld / tcgen05.st) by the softmax threads before the P V MMA is issued;
+//                  written to shared memory in the 128-byte-swizzled K-major layout.  With head_dim 128
+//                  P(j) takes the place of K(j) in its ring stage (same size; K(j) is dead once S(j)
+//                  is complete), which is what lets two CTAs fit in an SM.
+//   O += P V       the accumulator lives in TMEM columns [128, 128+head_dim).  The running maximum is
+//                  moved lazily: a row keeps its old reference maximum until the new one exceeds it by
+//                  more than 8 (in log2 units: probabilities then stay below 256, exact enough in fp16
+//                  and harmless in the fp32 sum), so the in-place rescale of O (tcgen05.ld / tcgen05.st,
+//                  which must wait for the previous P V) is rare; the final division by the row sum makes
+//                  the result independent of the reference used.
 //                  V is consumed as an MN-major operand straight from its row-major tile
 // Tiles entirely above the diagonal are skipped; the diagonal tile is masked in registers.
 // Every wait is bounded; on a timeout the CTA records a code in the status word and leaves through
@@ -26,7 +35,8 @@ namespace {
 constexpr int QT = 128;          // query rows per CTA
 constexpr int KT = 64;           // keys per tile
 constexpr int ATT_THREADS = 192;
-constexpr int TMEM_ALLOC = 256;  // S: 64 columns, O: up to 128
+constexpr int TMEM_ALLOC = 256;  // S: two buffers of 64 columns, O: up to 128
+constexpr float RESCALE_GAP = 8.0f;   // a row's reference maximum moves only when the new maximum exceeds it by this (log2 units)
 
 struct AttnMaps {
   CUtensorMap q, k, v, unused;
@@ -49,11 +59,12 @@ struct AttnSmem {
   static constexpr int Q_BYTES = QT * HD * 2;
   static constexpr int KV_TILE_BYTES = KT * HD * 2;      // one of K / V, one stage
   static constexpr int P_BYTES = QT * KT * 2;
-  static constexpr size_t TOTAL = 1024 + Q_BYTES + 4 * KV_TILE_BYTES + P_BYTES + 256;
+  static constexpr bool P_IN_K = (KV_TILE_BYTES >= P_BYTES);   // P(j) overwrites K(j) in its ring stage
+  static constexpr size_t TOTAL = 1024 + Q_BYTES + 4 * KV_TILE_BYTES + (P_IN_K ? 0 : 2 * P_BYTES) + 128;
 };
 
 template <int HD>
-__global__ void __launch_bounds__(ATT_THREADS, 1)
+__global__ void __launch_bounds__(ATT_THREADS, 2)
 prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) {
   using L = AttnSmem<HD>;
   constexpr int HALVES = L::HALVES;
@@ -63,15 +74,20 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
   unsigned char* q_s = smem;                                   // [HALVES][128 rows][128 B]
   unsigned char* k_s = q_s + L::Q_BYTES;                       // [2 stages][HALVES][64 rows][128 B]
   unsigned char* v_s = k_s + 2 * L::KV_TILE_BYTES;
-  unsigned char* p_s = v_s + 2 * L::KV_TILE_BYTES;             // [128 rows][128 B]
-  uint64_t* bars = (uint64_t*)(p_s + L::P_BYTES);
+  unsigned char* p_own = v_s + 2 * L::KV_TILE_BYTES;           // [2][128 rows][128 B] when P does not fit a K stage
+  uint64_t* bars = (uint64_t*)(p_own + (L::P_IN_K ? 0 : 2 * L::P_BYTES));
   uint64_t* q_full = bars;           // 1
   uint64_t* kv_full = bars + 1;      // [2]
   uint64_t* kv_empty = bars + 3;     // [2]
-  uint64_t* s_full = bars + 5;       // S ready in TMEM
-  uint64_t* p_full = bars + 6;       // P in smem, O rescaled (4 arrivals)
-  uint64_t* pv_done = bars + 7;      // P V accumulated
-  uint32_t* tmem_slot = (uint32_t*)(bars + 8);
+  uint64_t* s_full = bars + 5;       // [2] S buffer ready in TMEM
+  uint64_t* p_full = bars + 7;       // [2] P of tile j in smem, O rescaled if it had to be (4 arrivals); one barrier per
+                                     // tile parity: a warp may be one tile ahead of another, never two
+  uint64_t* pv_done = bars + 9;      // P V accumulated
+  uint32_t* tmem_slot = (uint32_t*)(bars + 10);
+  // P of tile j (ring stage j & 1)
+  auto p_tile = [&](int stage) -> unsigned char* {
+    return L::P_IN_K ? k_s + stage * L::KV_TILE_BYTES : p_own + stage * L::P_BYTES;
+  };
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -89,8 +105,10 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
       mbar_init(smem_u32(&kv_full[s]), 1);
       mbar_init(smem_u32(&kv_empty[s]), 1);
     }
-    mbar_init(smem_u32(s_full), 1);
-    mbar_init(smem_u32(p_full), 4);
+    mbar_init(smem_u32(&s_full[0]), 1);
+    mbar_init(smem_u32(&s_full[1]), 1);
+    mbar_init(smem_u32(&p_full[0]), 4);
+    mbar_init(smem_u32(&p_full[1]), 4);
     mbar_init(smem_u32(pv_done), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -101,8 +119,8 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();                                   // set-up above overlaps the previous kernel's tail
-  const uint32_t tmem_s = tmem_base;            // columns [0, 64)
-  const uint32_t tmem_o = tmem_base + 64;       // columns [64, 64 + HD)
+  const uint32_t tmem_s = tmem_base;            // two S buffers: columns [0, 64) and [64, 128)
+  const uint32_t tmem_o = tmem_base + 128;      // columns [128, 128 + HD)
 
   if (warp == 0) {
     if (lane == 0) {
@@ -142,31 +160,50 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
       constexpr uint32_t idesc_s = umma_idesc_f16(QT, KT);                      // Q, K both K-major
       constexpr uint32_t idesc_o = umma_idesc_f16(QT, HD) | (1u << 16);          // V is MN-major
       bool ok = mbar_wait(smem_u32(q_full), 0, abort_flag, a.status, 12);
-      for (int j = 0; j < n_kv && ok; ++j) {
-        const int s = j & 1;
-        ok = mbar_wait(smem_u32(&kv_full[s]), (uint32_t)((j >> 1) & 1), abort_flag, a.status, 13);
-        if (!ok) break;
-        tc_fence_after();
-        // S = Q K^T (the previous tile's softmax has finished with S: its P V MMA was issued after p_full)
-        const uint32_t kb = smem_u32(k_s + s * L::KV_TILE_BYTES);
+      // S(t) = Q K(t)^T into S buffer t & 1 (its previous reader, the softmax of tile t - 2, has signalled p_full)
+      auto issue_s = [&](int t) {
+        const uint32_t kb = smem_u32(k_s + (t & 1) * L::KV_TILE_BYTES);
 #pragma unroll
         for (int k = 0; k < HD / 16; ++k) {
           const int hf = k / 4, kk = k % 4;
-          umma_f16(tmem_s, umma_desc_sw128(smem_u32(q_s + hf * (QT * 128)) + kk * 32),
+          umma_f16(tmem_s + (uint32_t)((t & 1) * KT), umma_desc_sw128(smem_u32(q_s + hf * (QT * 128)) + kk * 32),
                    umma_desc_sw128(kb + hf * (KT * 128) + kk * 32), idesc_s, k > 0 ? 1u : 0u);
         }
-        umma_commit(smem_u32(s_full));
-        // O += P V once the softmax threads have written P and rescaled O
-        ok = mbar_wait(smem_u32(p_full), (uint32_t)(j & 1), abort_flag, a.status, 14);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t vb = smem_u32(v_s + s * L::KV_TILE_BYTES);
+        umma_commit(smem_u32(&s_full[t & 1]));
+      };
+      int s_next = 0;                              // next S product to issue; runs at most one tile ahead of P V
+      const uint64_t t_start = global_timer_ns();
+      for (int j = 0; j < n_kv && ok;) {
+        bool progressed = false;
+        if (s_next < n_kv && s_next <= j + 1 && mbar_try_wait(smem_u32(&kv_full[s_next & 1]), (uint32_t)((s_next >> 1) & 1))) {
+          tc_fence_after();
+          issue_s(s_next);
+          ++s_next;
+          progressed = true;
+        }
+        // O += P V once the softmax threads have written P (and rescaled O if they had to)
+        if (s_next > j && mbar_try_wait(smem_u32(&p_full[j & 1]), (uint32_t)((j >> 1) & 1))) {
+          tc_fence_after();
+          const int s = j & 1;
+          const uint32_t vb = smem_u32(v_s + s * L::KV_TILE_BYTES);
+          const uint32_t pb = smem_u32(p_tile(s));
 #pragma unroll
-        for (int k = 0; k < KT / 16; ++k)
-          umma_f16(tmem_o, umma_desc_sw128(smem_u32(p_s) + k * 32),
-                   umma_desc_sw128_mn(vb + k * (16 * 128), KT * 128, 1024), idesc_o, (j > 0 || k > 0) ? 1u : 0u);
-        umma_commit(smem_u32(&kv_empty[s]));
-        umma_commit(smem_u32(pv_done));
+          for (int k = 0; k < KT / 16; ++k)
+            umma_f16(tmem_o, umma_desc_sw128(pb + k * 32),
+                     umma_desc_sw128_mn(vb + k * (16 * 128), KT * 128, 1024), idesc_o, (j > 0 || k > 0) ? 1u : 0u);
+          umma_commit(smem_u32(&kv_empty[s]));
+          umma_commit(smem_u32(pv_done));
+          ++j;
+          progressed = true;
+        }
+        if (!progressed) {
+          if (*abort_flag) { ok = false; break; }
+          if (global_timer_ns() - t_start > 2000000000ull) {      // bounded: the whole tile loop gets two seconds
+            *abort_flag = 1;
+            if (a.status) { atomicCAS(a.status, 0, 13); a.status[1] = (int)blockIdx.x; }
+            ok = false;
+          }
+        }
       }
     }
   } else {
@@ -175,17 +212,17 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
     const int r = quarter * 32 + lane;                 // row inside the tile
     const int qi = q0 + r;                             // absolute query position
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    float m_run = -INFINITY, l_run = 0.f;
+    float m_ref = -INFINITY, l_run = 0.f;              // reference maximum of the row (log2 units), running sum
     bool ok = true;
     for (int j = 0; j < n_kv; ++j) {
-      ok = mbar_wait(smem_u32(s_full), (uint32_t)(j & 1), abort_flag, a.status, 15);
+      ok = mbar_wait(smem_u32(&s_full[j & 1]), (uint32_t)((j >> 1) & 1), abort_flag, a.status, 15);
       if (!ok) break;
       tc_fence_after();
       float sc[KT];
       {
         float t0[32], t1[32];
-        tmem_ld32(tmem_s + lane_off, t0);
-        tmem_ld32(tmem_s + lane_off + 32, t1);
+        tmem_ld32(tmem_s + (uint32_t)((j & 1) * KT) + lane_off, t0);
+        tmem_ld32(tmem_s + (uint32_t)((j & 1) * KT) + lane_off + 32, t1);
 #pragma unroll
         for (int c = 0; c < 32; ++c) { sc[c] = t0[c]; sc[32 + c] = t1[c]; }
       }
@@ -199,9 +236,11 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
         sc[c] = v;
         mx = fmaxf(mx, v);
       }
-      const float m_new = fmaxf(m_run, mx);
+      // move the reference only on the first tile or when the new maximum is far above it
+      const bool move = (mx > m_ref + RESCALE_GAP) || (m_ref == -INFINITY && mx > -INFINITY);
+      const float m_new = move ? mx : m_ref;
       const float m_use = (m_new == -INFINITY) ? 0.f : m_new;      // a fully masked row (only rows past T) stays at 0
-      const float alpha = exp2f(m_run - m_use);                     // m_run = -inf on the first tile -> 0
+      const float alpha = move ? exp2f(m_ref - m_use) : 1.0f;       // m_ref = -inf on the first tile -> 0
       float psum = 0.f;
       uint32_t packed[KT / 2];
 #pragma unroll
@@ -214,16 +253,17 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
         packed[c / 2] = *reinterpret_cast<const uint32_t*>(&hh);
       }
       l_run = l_run * alpha + psum;
-      m_run = m_new;
+      m_ref = m_new;
       // P row -> shared memory, 16-byte pieces at their swizzled places
-      unsigned char* prow = p_s + r * 128;
+      unsigned char* prow = p_tile(j & 1) + r * 128;
 #pragma unroll
       for (int c8 = 0; c8 < 8; ++c8) {
         const uint4 val = make_uint4(packed[4 * c8], packed[4 * c8 + 1], packed[4 * c8 + 2], packed[4 * c8 + 3]);
         *reinterpret_cast<uint4*>(prow + ((c8 ^ (r & 7)) << 4)) = val;
       }
-      // rescale the accumulator row (not before the previous P V has landed)
-      if (j > 0) {
+      // rescale the accumulator rows of this warp if any of them moved its reference (not before the previous P V
+      // has landed); on the first tile there is nothing to rescale: P V(0) overwrites O
+      if (j > 0 && __any_sync(0xffffffffu, move)) {
         ok = mbar_wait(smem_u32(pv_done), (uint32_t)((j - 1) & 1), abort_flag, a.status, 16);
         if (!ok) break;
         tc_fence_after();
@@ -239,7 +279,7 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
       fence_proxy_async_smem();      // P (generic stores) must be visible to the tensor cores' reads
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(p_full));
+      if (lane == 0) mbar_arrive(smem_u32(&p_full[j & 1]));
     }
     if (ok) ok = mbar_wait(smem_u32(pv_done), (uint32_t)((n_kv - 1) & 1), abort_flag, a.status, 17);
     if (ok) {
