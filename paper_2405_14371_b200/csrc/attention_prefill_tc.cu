@@ -281,6 +281,10 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&p_full[j & 1]));
     }
+    // The last two P V products may still be in flight: the score product of the last tile was issued before
+    // P V(n_kv - 2), so having seen it complete only proves P V(n_kv - 3).  Phase by phase, so that the parity
+    // test cannot mistake "two behind" for "done".
+    if (ok && n_kv >= 2) ok = mbar_wait(smem_u32(pv_done), (uint32_t)((n_kv - 2) & 1), abort_flag, a.status, 17);
     if (ok) ok = mbar_wait(smem_u32(pv_done), (uint32_t)((n_kv - 1) & 1), abort_flag, a.status, 17);
     if (ok) {
       tc_fence_after();

@@ -159,7 +159,9 @@ def test_linear_rejects_bad_shapes(B):
 @pytest.mark.parametrize("path", [1, 2])
 @pytest.mark.parametrize("Bn,T,Hq,Hkv,hd", [(1, 1, 4, 4, 64), (2, 16, 4, 4, 64), (1, 37, 4, 2, 128), (2, 130, 8, 1, 128),
                                             (1, 200, 2, 2, 64), (2, 64, 2, 2, 128), (1, 128, 2, 1, 128), (3, 257, 4, 4, 64),
-                                            (1, 512, 2, 2, 128)])
+                                            (1, 512, 2, 2, 128),
+                                            # enough CTAs for two to share every SM, many KV tiles per CTA
+                                            (2, 576, 32, 8, 128), (3, 320, 40, 40, 64)])
 def test_prefill_attention(B, path, Bn, T, Hq, Hkv, hd):
     """path 1 = tcgen05 kernel, 2 = CUDA-core kernel; N(0,1) q, k, v give peaked softmax rows."""
     q = _randn(Bn, T, Hq, hd, seed=8)
