@@ -141,6 +141,9 @@ def run_ours(args):
 
     rank, local, world = _dist_setup(args.gpus)
     wl = WORKLOADS[args.workload]
+    if args.layers:
+        import dataclasses
+        wl = dataclasses.replace(wl, layer_end=min(wl.layer_end, wl.layer_begin + args.layers * wl.n_shards))
     m = wl.model
     Bn, T, S = (args.batch or wl.batch), (args.prompt_len or wl.prompt_len), (args.decode_steps or wl.decode_steps)
     dev = torch.device("cuda", local)
@@ -435,9 +438,10 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (profile runs)")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length (profile runs only)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profile runs only)")
+    ap.add_argument("--layers", type=int, default=0, help="keep only the first LAYERS layers of every shard (profile runs only)")
     args = ap.parse_args()
-    if (args.prompt_len or args.batch) and not args.profile:
-        ap.error("--prompt-len / --batch change the workload and are only accepted together with --profile")
+    if (args.prompt_len or args.batch or args.layers) and not args.profile:
+        ap.error("--prompt-len / --batch / --layers change the workload and are only accepted together with --profile")
     if args.profile:
         args.warmup, args.steps = 1, 1
     else:

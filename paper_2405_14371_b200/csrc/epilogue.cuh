@@ -8,7 +8,9 @@
 
 namespace es {
 
-__device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)); }
+// silu(z) = z / (1 + e^-z) with the fast exponential and the fast division (2 ulp; a denominator beyond 2^126, i.e.
+// z below about -87, gives 0 where the exact value is below 1e-36 in magnitude).  Every kernel path uses this one.
+__device__ __forceinline__ float silu_f(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 
 // Residual / plain store of columns n and n+1 of row m.
 __device__ __forceinline__ void epi_f32_pair(const LinearParams& p, int m, int n, float v0, float v1) {
@@ -141,27 +143,44 @@ __device__ __forceinline__ void epi_swiglu_chunk32(const LinearParams& p, int m,
 __device__ __forceinline__ bool qkv_chunk32_fast(const LinearParams& p, int n) {
   return (n + 32 <= p.N) && ((n & 31) == 0) && ((p.hd & 31) == 0);
 }
-// Rotated / rounded values of the chunk as 32 fp16 and their destination (nullptr: nothing to store for this row).
-__device__ __forceinline__ void qkv_pack32(const LinearParams& p, int m, int n, const float (&v)[32], uint4 (&o)[4], __half*& dst) {
-  dst = nullptr;
-  if (m >= p.M) return;
-  const int nq = p.Hq * p.hd, nkv = p.Hkv * p.hd;
+// What a row of the fused QKV product needs from memory, the same for every column chunk of the row: its
+// position (for the rotation table), its row of the q output and its token's place in the KV pages.
+struct QkvRow {
+  bool valid;            // row < M and position inside the tables
+  int rope_off;          // pos * (hd / 2): offset of the row's cos / sin entries
+  int64_t q_off;         // m * Hq * hd
+  int64_t kv_off;        // (page * Hkv * P + pos % P) * hd: head 0, column 0 of the token in a K or V page
+};
+__device__ __forceinline__ QkvRow qkv_row(const LinearParams& p, int m) {
+  QkvRow r;
+  r.valid = false;
+  r.rope_off = 0; r.q_off = 0; r.kv_off = 0;
+  if (m >= p.M) return r;
   const int b = m / p.T;
   const int slot = p.slots[b];
   const int pos = p.is_decode ? p.ctx_len[slot] : (m - b * p.T);
-  if (pos < 0 || pos >= p.max_seq) return;
+  if (pos < 0 || pos >= p.max_seq) return r;
+  const int page = p.block_table[(int64_t)slot * p.pages_per_slot + pos / p.P];
+  r.valid = true;
+  r.rope_off = pos * (p.hd / 2);
+  r.q_off = (int64_t)m * p.Hq * p.hd;
+  r.kv_off = ((int64_t)page * p.Hkv * p.P + (pos % p.P)) * p.hd;
+  return r;
+}
+// Rotated / rounded values of the chunk as 32 fp16 and their destination (nullptr: nothing to store for this row).
+__device__ __forceinline__ void qkv_pack32_row(const LinearParams& p, const QkvRow& row, int n, const float (&v)[32],
+                                               uint4 (&o)[4], __half*& dst) {
+  dst = nullptr;
+  if (!row.valid) return;
+  const int nq = p.Hq * p.hd, nkv = p.Hkv * p.hd;
   const bool is_q = n < nq, is_k = !is_q && n < nq + nkv;
   const int local = is_q ? n : (is_k ? n - nq : n - nq - nkv);
   const int head = local / p.hd, c0 = local - head * p.hd;
-  if (is_q) {
-    dst = p.out_f16 + (int64_t)m * nq + n;
-  } else {
-    const int page = p.block_table[(int64_t)slot * p.pages_per_slot + pos / p.P];
-    dst = (is_k ? p.k_cache : p.v_cache) + (((int64_t)page * p.Hkv + head) * p.P + (pos % p.P)) * p.hd + c0;
-  }
+  if (is_q) dst = p.out_f16 + row.q_off + n;
+  else dst = (is_k ? p.k_cache : p.v_cache) + row.kv_off + (int64_t)head * p.P * p.hd + c0;
   if (is_q || is_k) {
-    const float4* cs4 = reinterpret_cast<const float4*>(p.rope_cos + (int64_t)pos * (p.hd / 2) + c0 / 2);
-    const float4* sn4 = reinterpret_cast<const float4*>(p.rope_sin + (int64_t)pos * (p.hd / 2) + c0 / 2);
+    const float4* cs4 = reinterpret_cast<const float4*>(p.rope_cos + row.rope_off + c0 / 2);
+    const float4* sn4 = reinterpret_cast<const float4*>(p.rope_sin + row.rope_off + c0 / 2);
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const float4 cs = cs4[q], sn = sn4[q];
@@ -180,6 +199,9 @@ __device__ __forceinline__ void qkv_pack32(const LinearParams& p, int m, int n, 
     }
   }
 }
+__device__ __forceinline__ void qkv_pack32(const LinearParams& p, int m, int n, const float (&v)[32], uint4 (&o)[4], __half*& dst) {
+  qkv_pack32_row(p, qkv_row(p, m), n, v, o, dst);
+}
 
 __device__ __forceinline__ void epi_qkv_chunk32(const LinearParams& p, int m, int n, const float (&v)[32]) {
   if (m >= p.M || n >= p.N) return;
@@ -197,21 +219,72 @@ __device__ __forceinline__ void epi_qkv_chunk32(const LinearParams& p, int m, in
 }
 
 // ---- the same chunks stored through a per-warp shared-memory tile -------------------------------
-// A thread that owns 32 adjacent columns of ONE row stores 16 bytes into a row of its own: 32 rows per
+// A thread that owns 32 adjacent columns of ONE row would store 16 bytes into a row of its own: 32 rows per
 // instruction, half a 32-byte sector each.  The variants below are called by a whole warp whose lane l owns
-// row m0 + l; they pass the chunk through `stage` (EPI_STAGE_BYTES of shared memory private to the warp) so
-// that every store instruction writes whole 64- or 128-byte row segments.  The arithmetic is that of the
-// functions above.
-constexpr int EPI_STAGE_BYTES = 32 * 36 * 4 + 32 * 8;   // a 32 x 32 fp32 tile with 36-word rows, then one pointer per row
+// row m0 + l; they pass the chunk through `stage` (shared memory private to the warp) and then store it with
+// several lanes per row, so that every instruction writes (and, for the residual, reads) whole row segments.
+// The arithmetic is that of the functions above.
+constexpr int EPI_STAGE_BYTES = 32 * 80 + 32 * 8;   // fp16 chunks: 32 rows of 64 bytes in 80-byte rows, then one pointer per row
+
+// After the turn-around lane l holds, for i = 0..3, piece (l >> 3) of row i * 8 + (l & 7).
+__device__ __forceinline__ int staged_row(int i, int lane) { return i * 8 + (lane & 7); }
+__device__ __forceinline__ int staged_piece(int lane) { return lane >> 3; }
+
+// in: o = this lane's row, 64 bytes.  out: t[i] = piece staged_piece(lane) of row staged_row(i, lane).
+__device__ __forceinline__ void stage_turn(const uint4 (&o)[4], uint4 (&t)[4], unsigned char* stage, int lane) {
+  uint4* tile = reinterpret_cast<uint4*>(stage);                      // rows of 5 x 16 bytes (4 used): conflict-free both ways
+#pragma unroll
+  for (int q = 0; q < 4; ++q) tile[lane * 5 + q] = o[q];
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) t[i] = tile[staged_row(i, lane) * 5 + staged_piece(lane)];
+  __syncwarp();
+}
+
+// 32 fp16 values per row (o) to dst (nullptr = skip the row)
+__device__ __forceinline__ void rows16_store_staged(__half* dst, const uint4 (&o)[4], unsigned char* stage, int lane) {
+  unsigned long long* rowptr = reinterpret_cast<unsigned long long*>(stage + 32 * 80);
+  rowptr[lane] = reinterpret_cast<unsigned long long>(dst);
+  uint4 t[4];
+  stage_turn(o, t, stage, lane);                 // its first __syncwarp also publishes rowptr
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __half* d = reinterpret_cast<__half*>(rowptr[staged_row(i, lane)]);
+    if (d != nullptr) reinterpret_cast<uint4*>(d)[staged_piece(lane)] = t[i];
+  }
+  __syncwarp();                                  // rowptr is rewritten by the next call
+}
+
+// fp32 chunks turn around as a whole 32 x 32 tile (rows of 36 words: conflict-free both ways), so that eight
+// lanes cover the 128 bytes of a row and every store writes whole lines.
+constexpr int EPI_STAGE_F32_BYTES = 32 * 36 * 4;
+
+__device__ __forceinline__ bool f32_chunk32_fast(const float* out, const float* res, int64_t ldo, int N, int n) {
+  return (n + 32 <= N) && ((ldo & 3) == 0) && ((n & 3) == 0) && (((uintptr_t)out & 15) == 0) &&
+         (res == nullptr || ((uintptr_t)res & 15) == 0);
+}
+// The residual values this lane will add for the chunk at column n (row i * 4 + lane / 8, columns (lane % 8) * 4 ..),
+// fetched ahead of time.  Nothing is loaded (and rv is left alone) when there is no residual or the chunk takes
+// the element-wise path.
+__device__ __forceinline__ void f32_chunk32_load_res(const float* out, const float* res, int64_t ldo, int M, int N, int m0,
+                                                     int n, int lane, float4 (&rv)[8]) {
+  if (res == nullptr || n >= N || !f32_chunk32_fast(out, res, ldo, N, n)) return;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int m = m0 + i * 4 + (lane >> 3);
+    rv[i] = (m < M) ? __ldcs(reinterpret_cast<const float4*>(res + (int64_t)m * ldo + n + (lane & 7) * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+}
 
 // out[m, n .. n+31] = v (+ res[m, n .. n+31]) for the 32 rows m0 + lane; out / res row stride ldo; rows >= M and
-// columns >= N are skipped.  res may alias out.
+// columns >= N are skipped.  res may alias out (a thread reads and writes exactly the same elements, so its loads
+// may be hoisted above its stores).  PRELOADED: rv already holds what f32_chunk32_load_res fetched for this chunk.
+// stage: EPI_STAGE_F32_BYTES of shared memory private to the warp.
+template <bool PRELOADED>
 __device__ __forceinline__ void f32_chunk32_staged(float* out, const float* res, int64_t ldo, int M, int N, int m0, int n,
-                                                   const float (&v)[32], unsigned char* stage, int lane) {
+                                                   const float (&v)[32], float4 (&rv)[8], unsigned char* stage, int lane) {
   if (n >= N) return;
-  const bool fast = (n + 32 <= N) && ((ldo & 3) == 0) && ((n & 3) == 0) &&
-                    (((uintptr_t)out & 15) == 0) && (res == nullptr || ((uintptr_t)res & 15) == 0);
-  if (!fast) {                                    // same decision in every lane: element-wise, one row per thread
+  if (!f32_chunk32_fast(out, res, ldo, N, n)) {   // same decision in every lane: element-wise, one row per thread
     const int m = m0 + lane;
     if (m < M) {
       const int64_t o = (int64_t)m * ldo + n;
@@ -221,22 +294,13 @@ __device__ __forceinline__ void f32_chunk32_staged(float* out, const float* res,
     }
     return;
   }
-  // residual first: eight independent 16-byte loads in flight while the tile turns around.  A thread reads and
-  // writes exactly the same elements, so hoisting the loads above the stores is safe when res aliases out.
-  const int cq = (lane & 7) * 4;                  // eight lanes cover the 128 bytes of one row
-  float4 rv[8];
-  if (res != nullptr) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int m = m0 + i * 4 + (lane >> 3);
-      rv[i] = (m < M) ? __ldcs(reinterpret_cast<const float4*>(res + (int64_t)m * ldo + n + cq)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-  }
+  if (!PRELOADED) f32_chunk32_load_res(out, res, ldo, M, N, m0, n, lane, rv);
   float* tile = reinterpret_cast<float*>(stage);
 #pragma unroll
   for (int q = 0; q < 8; ++q)
     *reinterpret_cast<float4*>(tile + lane * 36 + 4 * q) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
   __syncwarp();
+  const int cq = (lane & 7) * 4;                  // eight lanes cover the 128 bytes of one row
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int rr = i * 4 + (lane >> 3);
@@ -252,25 +316,8 @@ __device__ __forceinline__ void f32_chunk32_staged(float* out, const float* res,
 
 __device__ __forceinline__ void epi_f32_chunk32_staged(const LinearParams& p, int m0, int n, const float (&v)[32],
                                                        unsigned char* stage, int lane) {
-  f32_chunk32_staged(p.out_f32, p.res, p.ldo, p.M, p.N, m0, n, v, stage, lane);
-}
-
-// 32 fp16 values per row (o) to dst (nullptr = skip the row): four lanes cover the 64 bytes of one row
-__device__ __forceinline__ void rows16_store_staged(__half* dst, const uint4 (&o)[4], unsigned char* stage, int lane) {
-  uint4* tile = reinterpret_cast<uint4*>(stage);                      // rows of 5 x 16 bytes (4 used)
-  unsigned long long* rowptr = reinterpret_cast<unsigned long long*>(stage + 32 * 36 * 4);
-#pragma unroll
-  for (int q = 0; q < 4; ++q) tile[lane * 5 + q] = o[q];
-  rowptr[lane] = reinterpret_cast<unsigned long long>(dst);
-  __syncwarp();
-  const int piece = lane >> 3;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int rr = i * 8 + (lane & 7);
-    __half* d = reinterpret_cast<__half*>(rowptr[rr]);
-    if (d != nullptr) reinterpret_cast<uint4*>(d)[piece] = tile[rr * 5 + piece];
-  }
-  __syncwarp();
+  float4 rv[8];
+  f32_chunk32_staged<false>(p.out_f32, p.res, p.ldo, p.M, p.N, m0, n, v, rv, stage, lane);
 }
 
 __device__ __forceinline__ void epi_swiglu_chunk32_staged(const LinearParams& p, int m0, int n, const float (&g)[32],
@@ -286,8 +333,9 @@ __device__ __forceinline__ void epi_swiglu_chunk32_staged(const LinearParams& p,
   rows16_store_staged(dst, o, stage, lane);
 }
 
-__device__ __forceinline__ void epi_qkv_chunk32_staged(const LinearParams& p, int m0, int n, const float (&v)[32],
-                                                       unsigned char* stage, int lane) {
+// row = qkv_row(p, m0 + lane), computed once per tile
+__device__ __forceinline__ void epi_qkv_chunk32_staged(const LinearParams& p, const QkvRow& row, int m0, int n,
+                                                       const float (&v)[32], unsigned char* stage, int lane) {
   if (n >= p.N) return;
   if (!qkv_chunk32_fast(p, n)) {
     epi_qkv_chunk32(p, m0 + lane, n, v);
@@ -295,7 +343,7 @@ __device__ __forceinline__ void epi_qkv_chunk32_staged(const LinearParams& p, in
   }
   uint4 o[4];
   __half* dst;
-  qkv_pack32(p, m0 + lane, n, v, o, dst);
+  qkv_pack32_row(p, row, n, v, o, dst);
   rows16_store_staged(dst, o, stage, lane);
 }
 

@@ -38,7 +38,7 @@ template <int BN> struct TileCfg {
   static constexpr int STAGES = (200 * 1024) / (A_STAGE_BYTES + B_STAGE_BYTES) > 8 ? 8 : (200 * 1024) / (A_STAGE_BYTES + B_STAGE_BYTES);
   static constexpr int TMEM_COLS = BN;                                       // one accumulator buffer
   static constexpr int TMEM_ALLOC = 2 * BN <= 64 ? 64 : 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512;   // two buffers, power of two
-  static constexpr size_t SMEM = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 4 * EPI_STAGE_BYTES + 256;
+  static constexpr size_t SMEM = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 4 * EPI_STAGE_F32_BYTES + 256;
 };
 
 struct TmapSet {
@@ -64,7 +64,7 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
   unsigned char* a_tiles = smem;
   unsigned char* b_tiles = smem + (size_t)STAGES * A_STAGE_BYTES;
   unsigned char* epi_stage = b_tiles + (size_t)STAGES * Cfg::B_STAGE_BYTES;   // one store-staging tile per epilogue warp
-  uint64_t* bars = (uint64_t*)(epi_stage + 4 * EPI_STAGE_BYTES);
+  uint64_t* bars = (uint64_t*)(epi_stage + 4 * EPI_STAGE_F32_BYTES);
   uint64_t* full_bar = bars;
   uint64_t* empty_bar = bars + STAGES;
   uint64_t* acc_full = bars + 2 * STAGES;        // [2]
@@ -200,7 +200,7 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
       tile_origin(tile - ks * mn_tiles, m0, n0);
       const int mw = m0 + quarter * 32;              // row of lane 0
       const uint32_t trow = tmem_base + (uint32_t)(buf * ACC_COLS) + ((uint32_t)(quarter * 32) << 16);
-      unsigned char* stage = epi_stage + (size_t)(warp - 2) * EPI_STAGE_BYTES;
+      unsigned char* stage = epi_stage + (size_t)(warp - 2) * EPI_STAGE_F32_BYTES;   // large enough for either kind of chunk
       if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
         for (int c = 0; c < BN_OUT; c += 32) {
@@ -209,18 +209,23 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
           tmem_ld32(trow + BN_OUT + c, u);
           epi_swiglu_chunk32_staged(p, mw, n0 + c, g, u, stage, lane);
         }
-      } else {
+      } else if (EPI == EPI_QKV) {
+        const QkvRow row = qkv_row(p, mw + lane);      // the row's place in the q output and the KV pages, once per tile
 #pragma unroll 1
         for (int c = 0; c < BN; c += 32) {
           float v[32];
           tmem_ld32(trow + c, v);
-          if (EPI == EPI_F32) {
-            // split-K: the raw accumulator goes to slice ks of the workspace [k_splits, M, N]
-            if (k_splits > 1) f32_chunk32_staged(p.part + (int64_t)ks * p.M * p.N, nullptr, p.N, p.M, p.N, mw, n0 + c, v, stage, lane);
-            else epi_f32_chunk32_staged(p, mw, n0 + c, v, stage, lane);
-          } else {
-            epi_qkv_chunk32_staged(p, mw, n0 + c, v, stage, lane);
-          }
+          epi_qkv_chunk32_staged(p, row, mw, n0 + c, v, stage, lane);
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          float v[32];
+          float4 rv[8];
+          tmem_ld32(trow + c, v);
+          // split-K: the raw accumulator goes to slice ks of the workspace [k_splits, M, N]
+          if (k_splits > 1) f32_chunk32_staged<false>(p.part + (int64_t)ks * p.M * p.N, nullptr, p.N, p.M, p.N, mw, n0 + c, v, rv, stage, lane);
+          else f32_chunk32_staged<false>(p.out_f32, p.res, p.ldo, p.M, p.N, mw, n0 + c, v, rv, stage, lane);
         }
       }
       // this warp has read its quarter of the buffer: hand it back to the MMA issuer

@@ -32,12 +32,12 @@ constexpr int BM2 = 128;          // rows per CTA (256 per pair)
 constexpr int BN2 = 256;
 constexpr int BK2 = 64, UK2 = 16;
 constexpr int W_BOX = 32;
-constexpr int T2_THREADS = 192;
 constexpr int A_BYTES2 = BM2 * BK2 * 2;          // 16 KB
 constexpr int B_BYTES2 = (BN2 / 2) * BK2 * 2;    // this CTA's half of one 256-row W tile, 16 KB
 constexpr int RING_BYTES2 = 192 * 1024;          // 6 stages of 32 KB (NACC = 1) or 4 of 48 KB (NACC = 2)
 constexpr int MAX_STAGES2 = 6;
-constexpr size_t SMEM2 = 1024 + (size_t)RING_BYTES2 + 4 * EPI_STAGE_BYTES + 256;
+constexpr int EPI_AREA2 = 8 * EPI_STAGE_BYTES > 4 * EPI_STAGE_F32_BYTES ? 8 * EPI_STAGE_BYTES : 4 * EPI_STAGE_F32_BYTES;
+constexpr size_t SMEM2 = 1024 + (size_t)RING_BYTES2 + EPI_AREA2 + 256;   // eight small or four large store-staging tiles
 
 struct TmapSet2 {
   CUtensorMap a;
@@ -45,8 +45,17 @@ struct TmapSet2 {
 };
 static_assert(sizeof(TmapSet2) == sizeof(TcMaps), "TcMaps must hold four tensor maps");
 
+// Threads: warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner, then the epilogue warps (TMEM lane quarter =
+// warp % 4): four per accumulator for the fp16 epilogues; four in all for the fp32 one, whose store-staging tiles
+// are larger (each warp then drains both accumulators of its quarter).
+template <int EPI, int NACC> struct PairCfg {
+  static constexpr int EPI_WARPS = (EPI == EPI_F32) ? 4 : 4 * NACC;
+  static constexpr int THREADS = 64 + 32 * EPI_WARPS;
+  static constexpr int STAGE = (EPI == EPI_F32) ? EPI_STAGE_F32_BYTES : EPI_STAGE_BYTES;
+};
+
 template <int EPI, int NACC>
-__global__ void __launch_bounds__(T2_THREADS, 1)
+__global__ void __launch_bounds__(PairCfg<EPI, NACC>::THREADS, 1)
 linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, int* status, int m_tiles, int n_tiles) {
   constexpr int ACC_OUT = (EPI == EPI_SWIGLU) ? BN2 / 2 : BN2;   // output columns of one accumulator
   constexpr int BN_OUT = NACC * ACC_OUT;                           // output columns of a tile
@@ -60,11 +69,11 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* ring = smem;                    // stage s: A tile, then NACC half W tiles
   unsigned char* epi_stage = smem + RING_BYTES2;
-  uint64_t* bars = (uint64_t*)(epi_stage + 4 * EPI_STAGE_BYTES);
+  uint64_t* bars = (uint64_t*)(epi_stage + EPI_AREA2);
   uint64_t* full_bar = bars;                         // used in rank 0 only
   uint64_t* empty_bar = bars + MAX_STAGES2;          // one copy per CTA
   uint64_t* acc_full = bars + 2 * MAX_STAGES2;       // [2], one copy per CTA
-  uint64_t* acc_empty = bars + 2 * MAX_STAGES2 + 2;  // [2], used in rank 0 only (8 arrivals)
+  uint64_t* acc_empty = bars + 2 * MAX_STAGES2 + 2;  // [2], used in rank 0 only (every epilogue warp of both CTAs arrives)
   uint32_t* tmem_slot = (uint32_t*)(bars + 2 * MAX_STAGES2 + 4);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
@@ -92,7 +101,7 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&acc_full[b]), 1);
-      mbar_init(smem_u32(&acc_empty[b]), 8);       // four epilogue warps in each CTA of the pair
+      mbar_init(smem_u32(&acc_empty[b]), 2 * PairCfg<EPI, NACC>::EPI_WARPS);   // the epilogue warps of both CTAs
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -184,38 +193,58 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
     }
   } else {
     // ---- epilogue warps (both CTAs): own 128 rows x 256 columns ----
+    using PC = PairCfg<EPI, NACC>;
     const int quarter = warp & 3;
-    unsigned char* stage = epi_stage + (size_t)(warp - 2) * EPI_STAGE_BYTES;
+    const int a0 = (EPI == EPI_F32) ? 0 : (warp - 2) >> 2;       // first accumulator of this warp
+    constexpr int N_MY = (EPI == EPI_F32) ? NACC : 1;            // accumulators this warp drains
+    unsigned char* stage = epi_stage + (size_t)(warp - 2) * PC::STAGE;
     int local = 0;
     for (int tile = pair; tile < num_tiles; tile += n_pairs, ++local) {
       const int buf = local % NBUF;
       const uint32_t use = (uint32_t)(local / NBUF);
-      if (!mbar_wait(smem_u32(&acc_full[buf]), use & 1, abort_flag, status, 33)) break;
-      tc_fence_after();
       int m0, n0;
       tile_origin(tile, m0, n0);
       const int mw = m0 + (int)rank * BM2 + quarter * 32;          // row of lane 0
-      const uint32_t trow = tmem_base + (uint32_t)(buf * BN2) + ((uint32_t)(quarter * 32) << 16);
+      const int na = n0 + a0 * ACC_OUT;                            // first output column of this warp
+      // what does not depend on the accumulator is fetched before it is complete: the row's place in the q output
+      // and the KV pages, or the first chunk of the residual
+      QkvRow row;
+      float4 rv[2][8];
+      if (EPI == EPI_QKV) row = qkv_row(p, mw + lane);
+      if (EPI == EPI_F32) {
+        f32_chunk32_load_res(p.out_f32, p.res, p.ldo, p.M, p.N, mw, na, lane, rv[0]);
+      }
+      if (!mbar_wait(smem_u32(&acc_full[buf]), use & 1, abort_flag, status, 33)) break;
+      tc_fence_after();
+      const uint32_t tacc = tmem_base + (uint32_t)(buf * BN2 + a0 * BN2) + ((uint32_t)(quarter * 32) << 16);
+      if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
-      for (int a = 0; a < NACC; ++a) {
-        const uint32_t tacc = trow + (uint32_t)(a * BN2);
-        const int na = n0 + a * ACC_OUT;
-        if (EPI == EPI_SWIGLU) {
+        for (int c = 0; c < ACC_OUT; c += 32) {
+          float g[32], u[32];
+          tmem_ld32(tacc + c, g);
+          tmem_ld32(tacc + ACC_OUT + c, u);
+          epi_swiglu_chunk32_staged(p, mw, na + c, g, u, stage, lane);
+        }
+      } else if (EPI == EPI_QKV) {
 #pragma unroll 1
-          for (int c = 0; c < ACC_OUT; c += 32) {
-            float g[32], u[32];
-            tmem_ld32(tacc + c, g);
-            tmem_ld32(tacc + ACC_OUT + c, u);
-            epi_swiglu_chunk32_staged(p, mw, na + c, g, u, stage, lane);
-          }
-        } else {
+        for (int c = 0; c < BN2; c += 32) {
+          float v[32];
+          tmem_ld32(tacc + c, v);
+          epi_qkv_chunk32_staged(p, row, mw, na + c, v, stage, lane);
+        }
+      } else {
+        // accumulator columns and output columns coincide (ACC_OUT == BN2); the residual of the next chunk is
+        // requested before the current one is stored (two register sets, two chunks per trip of a rolled loop)
+        constexpr int NCH = N_MY * (BN2 / 32);
 #pragma unroll 1
-          for (int c = 0; c < BN2; c += 32) {
-            float v[32];
-            tmem_ld32(tacc + c, v);
-            if (EPI == EPI_F32) epi_f32_chunk32_staged(p, mw, na + c, v, stage, lane);
-            else epi_qkv_chunk32_staged(p, mw, na + c, v, stage, lane);
-          }
+        for (int c = 0; c < NCH; c += 2) {
+          float v[32];
+          f32_chunk32_load_res(p.out_f32, p.res, p.ldo, p.M, p.N, mw, na + (c + 1) * 32, lane, rv[1]);
+          tmem_ld32(tacc + c * 32, v);
+          f32_chunk32_staged<true>(p.out_f32, p.res, p.ldo, p.M, p.N, mw, na + c * 32, v, rv[0], stage, lane);
+          if (c + 2 < NCH) f32_chunk32_load_res(p.out_f32, p.res, p.ldo, p.M, p.N, mw, na + (c + 2) * 32, lane, rv[0]);
+          tmem_ld32(tacc + (c + 1) * 32, v);
+          f32_chunk32_staged<true>(p.out_f32, p.res, p.ldo, p.M, p.N, mw, na + (c + 1) * 32, v, rv[1], stage, lane);
         }
       }
       tc_fence_before();
@@ -256,7 +285,7 @@ es_status_t launch_pair(const TmapSet2& maps, const LinearParams& p, int* status
   if (pairs > tiles) pairs = tiles;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * pairs);
-  cfg.blockDim = dim3(T2_THREADS);
+  cfg.blockDim = dim3(PairCfg<EPI, NACC>::THREADS);
   cfg.dynamicSmemBytes = SMEM2;
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
