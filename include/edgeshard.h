@@ -128,6 +128,20 @@ ES_API es_status_t es_shard_create(const es_model_desc_t *desc, int32_t layer_be
 ES_API es_status_t es_shard_prefill(es_shard_t *shard, const int32_t *ids, const es_tensor_t *hidden_in,
                              int32_t B, int32_t T, const int32_t *slots);
 
+/* Prefill of prompts of different lengths in one batch (Sec. "Generative LLM Inference": requests are
+ * padded to a common length).  Arguments as for es_shard_prefill; the B prompts are RIGHT-padded to T
+ * rows each, and
+ *   lens       host int32 [B], 1 <= lens[b] <= T: the real tokens of sequence b are its first lens[b] rows.
+ * Padding ids must be valid token ids (their values do not matter).  All B * T rows are computed; causal
+ * attention keeps padding out of every real row.  Slot b then holds lens[b] positions, so the next
+ * es_shard_decode_step continues each sequence at its own position (the padded rows' K/V beyond it are
+ * overwritten as the sequence grows and are never read).  With the output layer, logits and the greedy
+ * token are those of row lens[b] - 1 of each sequence.  es_shard_handoff() gives hidden [B, T, d_model];
+ * rows at or beyond lens[b] are padding, and the next shard must be given the same lens.
+ * ES_ERR_RANGE if a length is outside [1, T]. */
+ES_API es_status_t es_shard_prefill_ragged(es_shard_t *shard, const int32_t *ids, const es_tensor_t *hidden_in,
+                                    int32_t B, int32_t T, const int32_t *slots, const int32_t *lens);
+
 /* One autoregressive step for B sequences: each consumes one token (ids dev int32 [B]) or one
  * activation row (hidden_in fp32 [B, d_model]) at its slot's next position and attends to the
  * slot's cached keys/values.  ES_ERR_STATE if a slot has no prefilled context, ES_ERR_KV_FULL if

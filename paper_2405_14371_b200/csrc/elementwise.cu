@@ -53,12 +53,15 @@ template <int THREADS, int REGS>
 __global__ void __launch_bounds__(THREADS) rmsnorm_kernel(const float* __restrict__ x,
                                                               const __half* __restrict__ gain,
                                                               __half* __restrict__ y, int d, float eps,
-                                                              int64_t row_stride, int64_t row_offset) {
+                                                              int64_t row_stride, int64_t row_offset,
+                                                              const int* __restrict__ last_of) {
   __shared__ float red[32];
   pdl_launch_dependents();
   pdl_wait();
   const int r = blockIdx.x;
-  const float4* src = reinterpret_cast<const float4*>(x + ((int64_t)r * row_stride + row_offset) * d);
+  // source row: r * row_stride + row_offset, or with last_of the last of the first last_of[r] rows of block r
+  const int64_t off = last_of ? (int64_t)last_of[r] - 1 : row_offset;
+  const float4* src = reinterpret_cast<const float4*>(x + ((int64_t)r * row_stride + off) * d);
   const int n4 = d / 4;
   float4 v[REGS];
   float ss = 0.f;
@@ -200,14 +203,15 @@ __global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ l
   }
 }
 
-// ctx_len[slots[b]] = add ? ctx_len[..] + value : value
-__global__ void set_ctx_kernel(int* ctx_len, const int* slots, int B, int value, int add) {
+// ctx_len[slots[b]] = add ? ctx_len[..] + value : value; with `values` the value of row b is values[b]
+__global__ void set_ctx_kernel(int* ctx_len, const int* slots, int B, int value, int add, const int* values) {
   pdl_launch_dependents();
   pdl_wait();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < B) {
     const int s = slots[b];
-    ctx_len[s] = add ? ctx_len[s] + value : value;
+    const int v = values ? values[b] : value;
+    ctx_len[s] = add ? ctx_len[s] + v : v;
   }
 }
 
@@ -222,12 +226,13 @@ es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, i
 }
 
 es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M, int d, float eps,
-                           int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches, bool pdl) {
+                           int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches, bool pdl,
+                           const int* last_of) {
   if (M <= 0) return ES_OK;
   if (M <= WIDE_ROWS_MAX)
-    ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset));
+    ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset, last_of));
   else
-    ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset));
+    ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset, last_of));
   if (launches) ++*launches;
   return ES_OK;
 }
@@ -252,9 +257,9 @@ es_status_t launch_splitk_reduce(const float* part, int k_splits, const float* r
 }
 
 es_status_t launch_set_ctx(int* ctx_len, const int* slots, int B, int value, int add, cudaStream_t s,
-                           int64_t* launches, bool pdl) {
+                           int64_t* launches, bool pdl, const int* values) {
   if (B <= 0) return ES_OK;
-  ES_CUDA_CHECK(launch_kernel(set_ctx_kernel, dim3((B + 63) / 64), dim3(64), 0, s, pdl, ctx_len, slots, B, value, add));
+  ES_CUDA_CHECK(launch_kernel(set_ctx_kernel, dim3((B + 63) / 64), dim3(64), 0, s, pdl, ctx_len, slots, B, value, add, values));
   if (launches) ++*launches;
   return ES_OK;
 }

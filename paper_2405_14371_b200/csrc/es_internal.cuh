@@ -126,14 +126,16 @@ bool tma_available();
 // ---- element-wise / reductions ---------------------------------------------------------------
 es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, int d, int vocab,
                          cudaStream_t s, int64_t* launches, bool pdl = false);
-// row r of y = rmsnorm(row (r * row_stride + row_offset) of x)
+// row r of y = rmsnorm(row (r * row_stride + row_offset) of x); with last_of (device, [M]) the source row is
+// r * row_stride + last_of[r] - 1 instead (the last of the first last_of[r] rows of block r)
 es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M, int d, float eps,
                            int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches,
-                           bool pdl = false);
+                           bool pdl = false, const int* last_of = nullptr);
 es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches,
                           bool pdl = false);
+// ctx_len[slots[b]] = (add ? ctx_len[slots[b]] : 0) + (values ? values[b] : value)
 es_status_t launch_set_ctx(int* ctx_len, const int* slots, int B, int value, int add, cudaStream_t s,
-                           int64_t* launches, bool pdl = false);
+                           int64_t* launches, bool pdl = false, const int* values = nullptr);
 
 // ---- attention -------------------------------------------------------------------------------
 // K/V addressing shared by both attention kernels: token t of sequence b, kv head g lives at

@@ -122,7 +122,7 @@ Layout make_layout(const es_model_desc_t& d, int begin, int end) {
   L.off_sin = take((size_t)d.max_seq * (d.head_dim / 2) * 4);
   L.off_table = take((size_t)L.n_pages * 4);
   L.off_ctx = take((size_t)d.max_slots * 4);
-  L.off_slots = take(B * 4);
+  L.off_slots = take(2 * B * 4);       // slots, then the prompt lengths of a ragged prefill
   L.off_status = take(256);
   L.off_splitk = take(d.max_tokens > 2 ? linear_tc_split_workspace_bytes() : 0);   // split-K partial sums of short prefills
   L.scratch_bytes = o;
@@ -172,10 +172,11 @@ struct es_shard {
   float* x;
   __half *h, *q, *ao, *act, *h_last;
   float *logits, *part, *rope_cos, *rope_sin;
-  int *next_ids, *block_table, *ctx_len, *slots_dev, *status;
+  int *next_ids, *block_table, *ctx_len, *slots_dev, *lens_dev, *status;
   float* splitk = nullptr;      // split-K workspace (nullptr when the shard never runs more than 2 rows)
   std::vector<int> ctx;         // host mirror of ctx_len, -1 = never prefilled
   std::vector<int> slots_host;  // slots currently uploaded to slots_dev
+  std::vector<int> lens_host;   // prompt lengths of the last ragged prefill (source of the upload)
   int last_B = 0, last_T = 0;
   bool last_valid = false;
   int64_t launches = 0;
@@ -357,7 +358,9 @@ inline void prof_mark(es_shard* s, int idx, int which) {
 
 // The launch sequence of one pass (prefill: T tokens per sequence; decode: T == 1 at each slot's
 // next position).  Everything is enqueued on s->stream.
-es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in, int B, int T, bool decode) {
+// lens (device, [B]) != nullptr: a prefill of right-padded prompts; sequence b has lens[b] <= T real tokens
+es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in, int B, int T, bool decode,
+                         const int* lens = nullptr) {
   const es_model_desc_t& d = s->d;
   const int M = B * T;
   int pi = 0;
@@ -472,10 +475,10 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   if (s->has_head) {
     prof_mark(s, pi, 0);
     // last position of every sequence only
-    const bool fuse_head = linear_stream_can_fuse_norm(B);
+    const bool fuse_head = lens == nullptr && linear_stream_can_fuse_norm(B);
     if (!fuse_head) {
       ES_TRY(kt_begin(s));
-      ES_TRY(launch_rmsnorm(s->x, s->fnorm, s->h_last, B, d.d_model, d.rms_eps, T, T - 1, s->stream, &s->launches, pdl));
+      ES_TRY(launch_rmsnorm(s->x, s->fnorm, s->h_last, B, d.d_model, d.rms_eps, T, T - 1, s->stream, &s->launches, pdl, lens));
       ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)B * d.d_model * 6.0));
     }
     for (int b0 = 0; b0 < B; b0 += 16) {
@@ -497,7 +500,7 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   }
   // the slots' contexts now hold T (prefill) or one more (decode) position
   ES_TRY(kt_begin(s));
-  ES_TRY(launch_set_ctx(s->ctx_len, s->slots_dev, B, decode ? 1 : T, decode ? 1 : 0, s->stream, &s->launches, pdl));
+  ES_TRY(launch_set_ctx(s->ctx_len, s->slots_dev, B, decode ? 1 : T, decode ? 1 : 0, s->stream, &s->launches, pdl, lens));
   ES_TRY(kt_end(s, ES_KT_SET_CTX, 0.0));
   s->pdl_now = false;
   return ES_OK;
@@ -600,6 +603,7 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
   s->block_table = (int*)(sb + L.off_table);
   s->ctx_len = (int*)(sb + L.off_ctx);
   s->slots_dev = (int*)(sb + L.off_slots);
+  s->lens_dev = s->slots_dev + desc->max_batch;
   s->status = (int*)(sb + L.off_status);
   s->splitk = desc->max_tokens > 2 ? (float*)(sb + L.off_splitk) : nullptr;
   s->ctx.assign(desc->max_slots, -1);
@@ -695,6 +699,31 @@ es_status_t es_shard_prefill(es_shard_t* s, const int32_t* ids, const es_tensor_
   s->last_valid = false;
   ES_TRY(enqueue_pass(s, ids, hin, B, T, false));
   for (int b = 0; b < B; ++b) s->ctx[slots[b]] = T;
+  s->last_B = B; s->last_T = T; s->last_valid = true;
+  if (s->profiling) { s->pending = true; s->pending_prefill = true; }
+  return ES_OK;
+}
+
+es_status_t es_shard_prefill_ragged(es_shard_t* s, const int32_t* ids, const es_tensor_t* hidden_in, int32_t B, int32_t T,
+                                    const int32_t* slots, const int32_t* lens) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  if (!lens) return fail(ES_ERR_INVALID_ARG, "lens is null");
+  if (B <= 0 || T <= 0) return fail(ES_ERR_INVALID_ARG, "B and T must be positive");
+  if (B > s->d.max_batch) return fail(ES_ERR_RANGE, "B = %d exceeds max_batch = %d", B, s->d.max_batch);
+  if ((int64_t)B * T > s->d.max_tokens) return fail(ES_ERR_RANGE, "B*T = %lld exceeds max_tokens = %d", (long long)B * T, s->d.max_tokens);
+  if (T > s->d.max_seq) return fail(ES_ERR_KV_FULL, "prompt of %d tokens exceeds max_seq = %d", T, s->d.max_seq);
+  for (int b = 0; b < B; ++b)
+    if (lens[b] < 1 || lens[b] > T) return fail(ES_ERR_RANGE, "lens[%d] = %d outside [1, %d]", b, lens[b], T);
+  ES_TRY(check_slots(s, slots, B));
+  const float* hin;
+  ES_TRY(check_inputs(s, ids, hidden_in, (int64_t)B * T, &hin));
+  if (s->profiling) ES_TRY(harvest_profile(s));
+  ES_TRY(upload_slots(s, slots, B));
+  s->lens_host.assign(lens, lens + B);
+  ES_CUDA_CHECK(cudaMemcpyAsync(s->lens_dev, s->lens_host.data(), B * sizeof(int), cudaMemcpyHostToDevice, s->stream));
+  s->last_valid = false;
+  ES_TRY(enqueue_pass(s, ids, hin, B, T, false, s->lens_dev));
+  for (int b = 0; b < B; ++b) s->ctx[slots[b]] = lens[b];
   s->last_B = B; s->last_T = T; s->last_valid = true;
   if (s->profiling) { s->pending = true; s->pending_prefill = true; }
   return ES_OK;

@@ -68,6 +68,7 @@ def test_description_validation(binding, kw, begin, end, status):
 def test_null_arguments_are_rejected_without_a_gpu(binding):
     lib = binding.lib
     assert lib.es_shard_prefill(None, None, None, 1, 1, None) == 1
+    assert lib.es_shard_prefill_ragged(None, None, None, 1, 1, None, None) == 1
     assert lib.es_shard_decode_step(None, None, None, 1, None) == 1
     assert lib.es_shard_handoff(None, None, None, None) == 1
     assert lib.es_layer_profile(None, None, 0, None) == 1

@@ -273,6 +273,57 @@ def test_edge_shapes_match_oracle(B, tiny, Bn, T, P):
         assert rel_err(ls[S][b], want_l) < TOL
 
 
+@pytest.mark.parametrize("P,split", [(64, None), (16, 1)])
+def test_ragged_prompts_and_sequences_that_stop_early(B, tiny, P, split):
+    """Right-padded prompts of different lengths in one batch (one of them the full width, one a single token, one
+    ending on a page boundary), then greedy decoding in which sequences leave the batch at different steps (the
+    caller's EOS handling: a finished sequence's slot is simply no longer passed).  Every sequence must match the
+    oracle run on that sequence alone; with `split` the model runs as two shards handing padded activations over."""
+    wd, wh = tiny
+    T, lens, stop_after = 40, [40, 1, 16, 23], [4, 1, 6, 3]        # decode steps each sequence stays for
+    Bn = len(lens)
+    ids = prompt_ids(0, Bn, T, TINY.vocab, seed=33)
+    S = max(stop_after)
+    slots = [2, 0, 3, 1]
+    kw = dict(max_slots=Bn, max_seq=T + S, max_tokens=Bn * T, kv_page_tokens=P)
+    if split is None:
+        shards = [B.Shard(TINY, 0, 2, wd, **kw)]
+    else:
+        shards = [B.Shard(TINY, 0, split, slice_weights(wd, TINY, 0, split), **kw),
+                  B.Shard(TINY, split, 2, slice_weights(wd, TINY, split, 2), **kw)]
+    x = None
+    for i, sh in enumerate(shards):
+        sh.es_shard_prefill_ragged(ids.cuda() if i == 0 else None, x, Bn, T, slots, lens)
+        x, logits, nxt = sh.es_shard_handoff()
+    pre_h, step_logits = x.clone(), [logits.clone()]
+    tokens = [nxt.clone().cpu()]                                   # tokens[s][row of the batch at step s]
+    alive = list(range(Bn))
+    rows_at = [list(alive)]
+    for s_ in range(S):
+        alive = [b for b in alive if stop_after[b] > s_]
+        if not alive:
+            break
+        prev_rows = rows_at[-1]
+        feed = torch.tensor([int(tokens[-1][prev_rows.index(b)]) for b in alive], dtype=torch.int32).cuda()
+        x = None
+        for i, sh in enumerate(shards):
+            sh.es_shard_decode_step(feed if i == 0 else None, x, len(alive), [slots[b] for b in alive])
+            x, logits, nxt = sh.es_shard_handoff()
+        step_logits.append(logits.clone()); tokens.append(nxt.clone().cpu()); rows_at.append(list(alive))
+    for sh in shards:
+        sh.es_shard_device_status()
+        sh.close()
+    for b in range(Bn):
+        fed = [int(tokens[s_][rows_at[s_].index(b)]) for s_ in range(len(rows_at) - 1) if b in rows_at[s_] and b in rows_at[s_ + 1]]
+        seq = torch.cat([ids[b, :lens[b]], torch.tensor(fed, dtype=torch.int32)])
+        want_h, _ = O.shard_forward_full(TINY, wh, 0, 2, ids=seq)
+        assert rel_err(pre_h[b, :lens[b]], want_h[:lens[b]]) < TOL
+        for s_ in range(len(fed) + 1):                            # logits after the prompt and after every fed token
+            _, want_l = O.shard_forward_full(TINY, wh, 0, 2, ids=seq[:lens[b] + s_])
+            got = step_logits[s_][rows_at[s_].index(b)]
+            assert rel_err(got, want_l) < TOL
+
+
 def test_profile_feeds_the_partition_planners(B, tiny):
     """The per-layer profile is the planners' input: measured times for this GPU plus two synthetic slower
     devices (scaled times), activation and memory sizes from the profile."""
