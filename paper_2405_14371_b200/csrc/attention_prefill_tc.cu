@@ -261,19 +261,25 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
         const uint4 val = make_uint4(packed[4 * c8], packed[4 * c8 + 1], packed[4 * c8 + 2], packed[4 * c8 + 3]);
         *reinterpret_cast<uint4*>(prow + ((c8 ^ (r & 7)) << 4)) = val;
       }
-      // rescale the accumulator rows of this warp if any of them moved its reference (not before the previous P V
-      // has landed); on the first tile there is nothing to rescale: P V(0) overwrites O
-      if (j > 0 && __any_sync(0xffffffffu, move)) {
+      // The previous P V must have landed before this warp signals tile j: every warp then follows pv_done phase by
+      // phase (the parity test can only tell "this phase" from "the next", so a phase must never be skipped; waiting
+      // for two phases at the end instead deadlocked whenever both had already completed).  P V(j - 1) was issued
+      // before this tile's softmax began, so the wait is normally over at once.
+      if (j > 0) {
         ok = mbar_wait(smem_u32(pv_done), (uint32_t)((j - 1) & 1), abort_flag, a.status, 16);
         if (!ok) break;
         tc_fence_after();
+        // rescale the accumulator rows of this warp if any of them moved its reference; on the first tile there is
+        // nothing to rescale: P V(0) overwrites O
+        if (__any_sync(0xffffffffu, move)) {
 #pragma unroll 1
-        for (int c = 0; c < HD; c += 32) {
-          float o[32];
-          tmem_ld32(tmem_o + lane_off + c, o);
+          for (int c = 0; c < HD; c += 32) {
+            float o[32];
+            tmem_ld32(tmem_o + lane_off + c, o);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] *= alpha;
-          tmem_st32(tmem_o + lane_off + c, o);
+            for (int i = 0; i < 32; ++i) o[i] *= alpha;
+            tmem_st32(tmem_o + lane_off + c, o);
+          }
         }
       }
       fence_proxy_async_smem();      // P (generic stores) must be visible to the tensor cores' reads
@@ -281,10 +287,7 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&p_full[j & 1]));
     }
-    // The last two P V products may still be in flight: the score product of the last tile was issued before
-    // P V(n_kv - 2), so having seen it complete only proves P V(n_kv - 3).  Phase by phase, so that the parity
-    // test cannot mistake "two behind" for "done".
-    if (ok && n_kv >= 2) ok = mbar_wait(smem_u32(pv_done), (uint32_t)((n_kv - 2) & 1), abort_flag, a.status, 17);
+    // every earlier phase of pv_done has been waited for inside the loop; the last one remains
     if (ok) ok = mbar_wait(smem_u32(pv_done), (uint32_t)((n_kv - 1) & 1), abort_flag, a.status, 17);
     if (ok) {
       tc_fence_after();
