@@ -254,6 +254,7 @@ ES_API es_status_t es_op_linear(const void *A, const void *W, const float *R, fl
  * Every (tile, slice) pair is computed by its own CTA into `workspace` ([k_splits, M, N] fp32,
  * device, 16-byte aligned, at least es_op_linear_splitk_workspace_bytes bytes); a second kernel adds
  * the slices in ascending order and the residual, so the result does not depend on scheduling.
+ * With 256 or more rows the slices are computed by CTA pairs (256 x 256 tiles), below that by single CTAs.
  * k_splits = 0 lets the library choose (1 = no split, no workspace needed).  Slices must not be
  * empty: (k_splits - 1) * ceil(ceil(K / 64) / k_splits) < ceil(K / 64), else ES_ERR_INVALID_ARG.
  * N must be a multiple of 4, K of 8.  R may be NULL and may alias C.

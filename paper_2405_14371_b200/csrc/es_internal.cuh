@@ -32,6 +32,7 @@ struct Tunables {
   int stream_deep;   // ES_STREAM_DEEP: weight-streaming kernel chunk depth, 1 = 4 KB per warp per buffer (default), 0 = 2 KB
   int tc_pair;       // ES_TC_PAIR: CTA-pair tensor-core kernel for large prefill products (1, default) or never (0)
   int tc_pair_wide;  // ES_TC_PAIR_WIDE: 256 x 512 pair tiles: chosen per shape (1, default), never (0), always (2)
+  int split_pairs;   // ES_SPLIT_PAIRS: split-K products with 256 or more rows run on CTA pairs (1, default) or on single CTAs (0)
   int pdl;           // ES_PDL: programmatic dependent launch in decode steps (1, default) or plain stream order (0)
   int attn_mma;      // ES_ATTN_MMA: tensor-core decode attention for launches with many items (1, default) or never (0)
   int split_k;       // ES_SPLIT_K: split-K for the O and down projections of short prefills (1, default) or never (0)
@@ -88,6 +89,8 @@ struct LinearParams {
   float* part;
   // CTA-pair tensor-core kernel: accumulators per tile, 1 = 256 x 256 tiles, 2 = 256 x 512 tiles, 0 = chosen per shape
   int pair_nacc;
+  // k_splits > 1 on the tensor-core path: the CTA-pair kernel computes the slices (else the single-CTA kernel)
+  int split_on_pairs;
 };
 
 // Kernel families.  Each returns after enqueuing; `launches` is incremented per kernel launched.
@@ -114,6 +117,7 @@ es_status_t launch_splitk_reduce(const float* part, int k_splits, const float* r
                                  const __half* gain, __half* y, float eps, cudaStream_t s, int64_t* launches, bool pdl = false);
 // CTA-pair (cta_group::2) variant for large M; uses the same tensor maps
 bool linear_tc2_supported(const LinearParams& p, int epi);
+int linear_tc2_splits(const LinearParams& p, int epi);   // K slices for a plain product on CTA pairs (1 = not this way)
 es_status_t launch_linear_tc2(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word, bool pdl = false);
 // Encodes the tensor maps for p's operands; the A map covers a_rows rows (the buffer's capacity).
 es_status_t tc_build_maps(const LinearParams& p, int epi, int64_t a_rows, TcMaps* out);

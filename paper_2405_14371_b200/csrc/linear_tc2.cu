@@ -80,8 +80,13 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-  const int num_tiles = m_tiles * n_tiles;
+  // split-K (plain epilogue only): every (tile, K slice) pair is a work item, slice-major, and the raw accumulator
+  // goes to slice ks of the workspace [k_splits, M, N]
+  const int k_splits = (EPI == EPI_F32 && p.k_splits > 1) ? p.k_splits : 1;
+  const int mn_tiles = m_tiles * n_tiles;
+  const int num_tiles = mn_tiles * k_splits;
   const int num_kb = (p.K + BK2 - 1) / BK2;
+  const int kb_per = (num_kb + k_splits - 1) / k_splits;
 
   auto tile_origin = [&](int tile, int& m0, int& n0) {
     constexpr int GM = 16;                         // 16 row tiles of 256 share a column tile in L2 (8 measured 2-3 % slower, 32 the same)
@@ -122,7 +127,9 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
         int m0, n0;
-        tile_origin(tile, m0, n0);
+        const int ks = tile / mn_tiles;
+        tile_origin(tile - ks * mn_tiles, m0, n0);
+        const int kb0 = ks * kb_per, kb1 = min(num_kb, kb0 + kb_per);
         // W rows this CTA stages for accumulator a: SwiGLU - rank 0 the gate rows, rank 1 the up rows of the same
         // 128 columns; otherwise rows [r * 128, r * 128 + 128) of the accumulator's 256 columns, inside one segment
         const CUtensorMap* wmap[NACC];
@@ -139,7 +146,7 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
             wrow[a] = n + (int)rank * (BN2 / 2);
           }
         }
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES2;
           const uint32_t ph = (it / STAGES2) & 1;
           if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1, abort_flag, status, 31)) { ok = false; break; }
@@ -170,7 +177,9 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
         if (!ok) break;
         tc_fence_after();
         const uint32_t tacc = tmem_base + (uint32_t)(buf * BN2);
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        const int ks = tile / mn_tiles;
+        const int kb0 = ks * kb_per, kb1 = min(num_kb, kb0 + kb_per);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES2;
           const uint32_t ph = (it / STAGES2) & 1;
           ok = mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag, status, 32);
@@ -184,7 +193,7 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
 #pragma unroll
             for (int a = 0; a < NACC; ++a)
               umma_f16_pair(tacc + (uint32_t)(a * BN2), adesc, umma_desc_sw128(b0 + a * B_BYTES2 + k * UK2 * 2), idesc,
-                            (kb > 0 || k > 0) ? 1u : 0u);
+                            (kb > kb0 || k > 0) ? 1u : 0u);
           }
           umma_commit_pair(smem_u32(&empty_bar[s]));
         }
@@ -203,16 +212,22 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
       const int buf = local % NBUF;
       const uint32_t use = (uint32_t)(local / NBUF);
       int m0, n0;
-      tile_origin(tile, m0, n0);
+      const int ks = tile / mn_tiles;
+      tile_origin(tile - ks * mn_tiles, m0, n0);
       const int mw = m0 + (int)rank * BM2 + quarter * 32;          // row of lane 0
       const int na = n0 + a0 * ACC_OUT;                            // first output column of this warp
+      // plain epilogue: where the rows go and what is added to them (split-K: raw sums to the workspace slice)
+      float* f_out = p.out_f32;
+      const float* f_res = p.res;
+      int64_t f_ld = p.ldo;
+      if (k_splits > 1) { f_out = p.part + (int64_t)ks * p.M * p.N; f_res = nullptr; f_ld = p.N; }
       // what does not depend on the accumulator is fetched before it is complete: the row's place in the q output
       // and the KV pages, or the first chunk of the residual
       QkvRow row;
       float4 rv[2][8];
       if (EPI == EPI_QKV) row = qkv_row(p, mw + lane);
       if (EPI == EPI_F32) {
-        f32_chunk32_load_res(p.out_f32, p.res, p.ldo, p.M, p.N, mw, na, lane, rv[0]);
+        f32_chunk32_load_res(f_out, f_res, f_ld, p.M, p.N, mw, na, lane, rv[0]);
       }
       if (!mbar_wait(smem_u32(&acc_full[buf]), use & 1, abort_flag, status, 33)) break;
       tc_fence_after();
@@ -239,12 +254,12 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
 #pragma unroll 1
         for (int c = 0; c < NCH; c += 2) {
           float v[32];
-          f32_chunk32_load_res(p.out_f32, p.res, p.ldo, p.M, p.N, mw, na + (c + 1) * 32, lane, rv[1]);
+          f32_chunk32_load_res(f_out, f_res, f_ld, p.M, p.N, mw, na + (c + 1) * 32, lane, rv[1]);
           tmem_ld32(tacc + c * 32, v);
-          f32_chunk32_staged<true>(p.out_f32, p.res, p.ldo, p.M, p.N, mw, na + c * 32, v, rv[0], stage, lane);
-          if (c + 2 < NCH) f32_chunk32_load_res(p.out_f32, p.res, p.ldo, p.M, p.N, mw, na + (c + 2) * 32, lane, rv[0]);
+          f32_chunk32_staged<true>(f_out, f_res, f_ld, p.M, p.N, mw, na + c * 32, v, rv[0], stage, lane);
+          if (c + 2 < NCH) f32_chunk32_load_res(f_out, f_res, f_ld, p.M, p.N, mw, na + (c + 2) * 32, lane, rv[0]);
           tmem_ld32(tacc + (c + 1) * 32, v);
-          f32_chunk32_staged<true>(p.out_f32, p.res, p.ldo, p.M, p.N, mw, na + (c + 1) * 32, v, rv[1], stage, lane);
+          f32_chunk32_staged<true>(f_out, f_res, f_ld, p.M, p.N, mw, na + (c + 1) * 32, v, rv[1], stage, lane);
         }
       }
       tc_fence_before();
@@ -280,7 +295,7 @@ es_status_t launch_pair(const TmapSet2& maps, const LinearParams& p, int* status
     ES_CUDA_CHECK(cudaGetDevice(&dev));
     ES_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   }
-  const int tiles = m_tiles * n_tiles;
+  const int tiles = m_tiles * n_tiles * ((EPI == EPI_F32 && p.k_splits > 1) ? p.k_splits : 1);
   int pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
   cudaLaunchConfig_t cfg = {};
@@ -306,6 +321,7 @@ es_status_t launch_pair(const TmapSet2& maps, const LinearParams& p, int* status
 // rows): K = 4096 +-2 %, K = 8192 +7 % (+1 % with a residual to read), K = 28672 +13 % (+10 %).  It is taken
 // for K >= 8192 when its waves, discounted for the traffic saved, come out shorter.
 int pair_nacc(const LinearParams& p, int epi) {
+  if (p.k_splits > 1) return 1;
   if (p.pair_nacc == 1 || p.pair_nacc == 2) return p.pair_nacc;
   const int force = tunables().tc_pair_wide;
   if (force == 0) return 1;
@@ -335,8 +351,34 @@ bool linear_tc2_supported(const LinearParams& p, int epi) {
   return p.M >= 2 * BM2 && tiles >= 74;
 }
 
+// K slices for a plain product with too few 256 x 256 tiles for the machine's 74 pairs (1 = do not use the pair
+// kernel this way): as many slices as keep every (tile, slice) item in one wave, at least four K blocks each, and a
+// workspace of linear_tc_split_workspace_bytes() must hold the partial sums.  Against the single-CTA split kernel
+// a CTA pulls a third fewer operand bytes through L2 for the same output.
+int linear_tc2_splits(const LinearParams& p, int epi) {
+  if (epi != EPI_F32 || p.M < 2 * BM2 || p.N % 4 != 0 || !linear_tc_supported(p, epi)) return 1;
+  const int tiles = ((p.M + 2 * BM2 - 1) / (2 * BM2)) * ((p.N + BN2 - 1) / BN2);
+  if (tiles >= 74) return 1;
+  const int num_kb = (p.K + BK2 - 1) / BK2;
+  int s = 74 / tiles;
+  if (s > 8) s = 8;
+  if (s > num_kb / 4) s = num_kb / 4;
+  while (s > 1 && (size_t)s * p.M * p.N * sizeof(float) > linear_tc_split_workspace_bytes()) --s;
+  if (s < 2) return 1;
+  const int kb_per = (num_kb + s - 1) / s;
+  return (num_kb + kb_per - 1) / kb_per;       // no empty slice
+}
+
 es_status_t launch_linear_tc2(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word, bool pdl) {
-  if (!linear_tc2_supported(p, epi)) return fail(ES_ERR_UNSUPPORTED, "pair kernel does not take this shape");
+  if (p.k_splits > 1) {
+    if (epi != EPI_F32 || p.part == nullptr || p.N % 4 != 0 || p.M < 2 * BM2 || !linear_tc_supported(p, epi))
+      return fail(ES_ERR_INVALID_ARG, "split-K on CTA pairs needs the plain epilogue, a workspace, N %% 4 == 0 and M >= 256");
+    const int num_kb = (p.K + BK2 - 1) / BK2;
+    const int kb_per = (num_kb + p.k_splits - 1) / p.k_splits;
+    if ((p.k_splits - 1) * kb_per >= num_kb) return fail(ES_ERR_INVALID_ARG, "split-K: %d slices leave one empty (K = %d)", p.k_splits, p.K);
+  } else if (!linear_tc2_supported(p, epi)) {
+    return fail(ES_ERR_UNSUPPORTED, "pair kernel does not take this shape");
+  }
   TcMaps local;
   const TcMaps* maps = p.tc_maps;
   if (!maps) {

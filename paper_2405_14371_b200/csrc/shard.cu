@@ -40,7 +40,7 @@ static int env_int(const char* name, int dflt) {
 }
 
 const Tunables& tunables() {
-  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_TC_PAIR_WIDE", 1), env_int("ES_PDL", 1), env_int("ES_ATTN_MMA", 1), env_int("ES_SPLIT_K", 1)};
+  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_TC_PAIR_WIDE", 1), env_int("ES_SPLIT_PAIRS", 1), env_int("ES_PDL", 1), env_int("ES_ATTN_MMA", 1), env_int("ES_SPLIT_K", 1)};
   return t;
 }
 
@@ -241,7 +241,9 @@ es_status_t dispatch_linear(es_shard* s, const LinearParams& p, int epi) {
   if (p.M > 2 && p.M <= 16 && linear_stream_mma_supported(p, epi))
     return launch_linear_stream_mma(p, epi, s->stream, &s->launches, s->pdl_now);
   if (p.M <= 16) return launch_linear_stream(p, epi, s->stream, &s->launches, s->pdl_now);
-  if (p.k_splits > 1) return launch_linear_tc(p, epi, s->stream, &s->launches, s->status, s->pdl_now);
+  if (p.k_splits > 1)
+    return p.split_on_pairs ? launch_linear_tc2(p, epi, s->stream, &s->launches, s->status, s->pdl_now)
+                            : launch_linear_tc(p, epi, s->stream, &s->launches, s->status, s->pdl_now);
   if (tunables().tc_pair && linear_tc2_supported(p, epi)) return launch_linear_tc2(p, epi, s->stream, &s->launches, s->status, s->pdl_now);
   if (linear_tc_supported(p, epi)) return launch_linear_tc(p, epi, s->stream, &s->launches, s->status, s->pdl_now);
   return launch_linear_reference(p, epi, s->stream, &s->launches);
@@ -296,10 +298,15 @@ LinearParams base_params(const es_shard* s, int M, int T, bool decode) {
 }
 
 // K slices for a product on the tensor-core path (1 = whole K range per tile).
-int split_k_for(const es_shard* s, const LinearParams& p, int epi) {
+int split_k_for(const es_shard* s, LinearParams& p, int epi) {
+  p.split_on_pairs = 0;
   if (s->splitk == nullptr || p.M <= 2 || tunables().split_k == 0) return 1;
   if (p.M <= 16) return linear_stream_mma_splits(p, epi, linear_tc_split_workspace_bytes());   // decode with several sequences
   if (!linear_tc_supported(p, epi)) return 1;
+  if (tunables().tc_pair && tunables().split_pairs) {
+    const int ps = linear_tc2_splits(p, epi);        // 256 or more rows: slices on CTA pairs
+    if (ps > 1) { p.split_on_pairs = 1; return ps; }
+  }
   return linear_tc_splits(p, epi);
 }
 
@@ -992,7 +999,11 @@ es_status_t es_op_linear_splitk(const void* A, const void* W, const float* R, fl
     if (k_splits == 0) k_splits = linear_stream_mma_splits(p, EPI_F32, workspace ? workspace_bytes : 0);
   } else {
     if (!linear_tc_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "tensor-core kernel does not take this shape");
-    if (k_splits == 0) k_splits = linear_tc_splits(p, EPI_F32);
+    p.split_on_pairs = (M >= 256 && tunables().tc_pair && tunables().split_pairs) ? 1 : 0;   // 256 or more rows: slices on CTA pairs
+    if (k_splits == 0) {
+      k_splits = p.split_on_pairs ? linear_tc2_splits(p, EPI_F32) : 1;
+      if (k_splits <= 1) { p.split_on_pairs = 0; k_splits = linear_tc_splits(p, EPI_F32); }
+    }
   }
   if (k_splits < 1 || k_splits > 64) return fail(ES_ERR_INVALID_ARG, "k_splits must be 0 (automatic) or 1..64");
   if (k_splits == 1)
@@ -1007,7 +1018,8 @@ es_status_t es_op_linear_splitk(const void* A, const void* W, const float* R, fl
     return launch_splitk_reduce(p.part, k_splits, R, C, M, N, N, nullptr, nullptr, 0.f, st, nullptr);
   }
   p.k_splits = k_splits; p.part = (float*)workspace;
-  ES_TRY(launch_linear_tc(p, EPI_F32, st, nullptr, nullptr));
+  if (p.split_on_pairs) ES_TRY(launch_linear_tc2(p, EPI_F32, st, nullptr, nullptr));
+  else ES_TRY(launch_linear_tc(p, EPI_F32, st, nullptr, nullptr));
   return launch_splitk_reduce(p.part, k_splits, R, C, M, N, N, nullptr, nullptr, 0.f, st, nullptr);
 }
 

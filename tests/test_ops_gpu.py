@@ -104,7 +104,7 @@ def test_linear_tensor_core_cta_pairs(B, M, N, K):
 
 @pytest.mark.parametrize("M,N,K,S", [(128, 4096, 4096, 0), (128, 4096, 11008, 0), (256, 5120, 5120, 0), (100, 260, 1096, 3),
                                      (17, 36, 512, 2), (300, 1000, 4096, 5), (128, 512, 256, 4), (512, 4096, 4096, 0),
-                                     (128, 4096, 4096, 1)])
+                                     (128, 4096, 4096, 1), (512, 4096, 11008, 0), (700, 1000, 2080, 3), (256, 5120, 13824, 0)])
 def test_linear_tensor_core_split_k(B, M, N, K, S):
     """K range cut into slices (automatic count and fixed counts), ragged M / N / K, residual aliasing the output."""
     A = _randn(M, K, seed=22)
