@@ -18,8 +18,12 @@
 //     tokens' rows (a warp-wide load touches 128 contiguous bytes of 4 rows) and builds the pairs
 //     with one byte-permute each; MMA number i then produces dimensions 8g + i and 64 + 8g + i.
 //
-// K for the next 16 tokens is requested as soon as the score MMAs have consumed the registers, V as
-// soon as the output MMAs have, so loads and arithmetic overlap without extra registers.  The four
+// A register set is refilled with a later block as soon as it has been consumed (K after the score MMAs, V
+// after the output MMAs), so loads and arithmetic overlap.  With one or two query heads per KV head (DB) a
+// warp keeps two 16-token blocks in registers — while it works on one, the other is on its way — at two CTAs
+// per SM; with larger groups, whose blocks carry more arithmetic, one block per warp at three CTAs per SM
+// measured faster (config 4 shape 30.5 against 33.7 us; 8 sequences x 32 heads x 680 keys 27.1 -> 25.0 us
+// with two).  The four
 // warps of a CTA are merged through shared memory in warp order and the result is written as the
 // final row (one split) or as an unnormalised partial (o, max, sum) for the merge kernel, exactly
 // like the CUDA-core kernel, so results do not depend on scheduling.
@@ -58,8 +62,8 @@ __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
-template <int G>
-__global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const DecodeAttnParams p) {
+template <int G, bool DB>
+__global__ void __launch_bounds__(MW * 32, DB ? 2 : 3) decode_attn_mma_kernel(const DecodeAttnParams p) {
   pdl_launch_dependents();
   constexpr int HD = MHD;
   __shared__ float sm_o[MW][G][HD];
@@ -87,8 +91,7 @@ __global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const Decod
     const int page = table ? table[lp] : slot * p.kv.pages_per_slot + lp;
     return (int64_t)page * p.kv.page_stride + kv_head_off + (int64_t)(T - lp * p.kv.P) * p.kv.tok_stride;
   };
-  uint4 kreg[2][4], vreg[4][2];
-  auto load_k = [&](int T) {
+  auto load_k = [&](int T, uint4 (&kreg)[2][4]) {
     const int64_t base = block_base(T);
     const int last = t_end - 1 - T;                      // tokens past the end re-read the last valid row (masked below)
 #pragma unroll
@@ -99,7 +102,7 @@ __global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const Decod
       for (int j = 0; j < 4; ++j) kreg[nt][j] = ld_kv(row + (4 * j + t) * 8);
     }
   };
-  auto load_v = [&](int T) {
+  auto load_v = [&](int T, uint4 (&vreg)[4][2]) {
     const int64_t base = block_base(T);
     const int last = t_end - 1 - T;
 #pragma unroll
@@ -116,11 +119,15 @@ __global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const Decod
   for (int i = 0; i < 8; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
   float m_run = -INFINITY, l_run = 0.f;      // head g (replicated in the 4 threads of the group)
 
-  // The first block's K and V rows are requested before the dependency wait when every one of its
-  // tokens was cached by an earlier pass (the newest token's rows come from the kernel just before).
-  int T = t_begin + warp * 16;
-  const bool early = T < t_end && T + 16 <= ctx_old;
-  if (early) { load_k(T); load_v(T); }
+  // A block's K and V rows are requested before the dependency wait when every one of its tokens was cached
+  // by an earlier pass (the newest token's rows come from the kernel just before).
+  constexpr int STEP = MW * 16;              // tokens between consecutive blocks of one warp
+  uint4 kA[2][4], vA[4][2], kB[2][4], vB[4][2];
+  const int T0 = t_begin + warp * 16;
+  const bool earlyA = T0 < t_end && T0 + 16 <= ctx_old;
+  const bool earlyB = DB && T0 + STEP < t_end && T0 + STEP + 16 <= ctx_old;
+  if (earlyA) { load_k(T0, kA); load_v(T0, vA); }
+  if (earlyB) { load_k(T0 + STEP, kB); load_v(T0 + STEP, vB); }
 
   pdl_wait();
 
@@ -131,9 +138,11 @@ __global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const Decod
 #pragma unroll
     for (int j = 0; j < 4; ++j) qa[j] = (g < G) ? *reinterpret_cast<const uint4*>(qrow + (4 * j + t) * 8) : make_uint4(0, 0, 0, 0);
   }
-  if (T < t_end && !early) { load_k(T); load_v(T); }
-  for (; T < t_end; T += MW * 16) {
-    const int Tn = T + MW * 16;
+  if (T0 < t_end && !earlyA) { load_k(T0, kA); load_v(T0, vA); }
+  if (DB && T0 + STEP < t_end && !earlyB) { load_k(T0 + STEP, kB); load_v(T0 + STEP, vB); }
+
+  // one block of 16 tokens at T out of (kreg, vreg); the registers are refilled with the block at Tn
+  auto block = [&](int T, int Tn, uint4 (&kreg)[2][4], uint4 (&vreg)[4][2]) {
     // ---- scores of 16 tokens ----
     float s[2][4];
 #pragma unroll
@@ -145,7 +154,7 @@ __global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const Decod
         mma_f16(s[nt], qa[j].z, 0u, qa[j].w, 0u, kreg[nt][j].z, kreg[nt][j].w);
       }
     }
-    if (Tn < t_end) load_k(Tn);
+    if (Tn < t_end) load_k(Tn, kreg);
     // ---- online softmax: this thread holds head g, tokens T + 2t, T + 2t + 1, T + 8 + 2t, T + 9 + 2t ----
     float sv[4];
 #pragma unroll
@@ -176,7 +185,15 @@ __global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const Decod
       mma_f16(oacc[i], pair_of(vreg[0][0], vreg[1][0], i), pair_of(vreg[0][1], vreg[1][1], i),
               pair_of(vreg[2][0], vreg[3][0], i), pair_of(vreg[2][1], vreg[3][1], i), pb0, pb1);
     }
-    if (Tn < t_end) load_v(Tn);
+    if (Tn < t_end) load_v(Tn, vreg);
+  };
+  if (DB) {
+    for (int T = T0; T < t_end; T += 2 * STEP) {
+      block(T, T + 2 * STEP, kA, vA);
+      if (T + STEP < t_end) block(T + STEP, T + 3 * STEP, kB, vB);
+    }
+  } else {
+    for (int T = T0; T < t_end; T += STEP) block(T, T + STEP, kA, vA);
   }
 
   // ---- merge the warps in warp order ----
@@ -212,7 +229,7 @@ __global__ void __launch_bounds__(MW * 32, 3) decode_attn_mma_kernel(const Decod
 
 template <int G>
 es_status_t launch_g(const DecodeAttnParams& p, cudaStream_t s, bool pdl) {
-  ES_CUDA_CHECK(launch_kernel(decode_attn_mma_kernel<G>, dim3(p.n_splits, p.Hkv, p.B), dim3(MW * 32), 0, s, pdl, p));
+  ES_CUDA_CHECK(launch_kernel(decode_attn_mma_kernel<G, (G <= 2)>, dim3(p.n_splits, p.Hkv, p.B), dim3(MW * 32), 0, s, pdl, p));
   return ES_OK;
 }
 
