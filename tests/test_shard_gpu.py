@@ -324,6 +324,41 @@ def test_ragged_prompts_and_sequences_that_stop_early(B, tiny, P, split):
             assert rel_err(got, want_l) < TOL
 
 
+def test_pipeline_stage_drives_the_library_on_one_gpu(B, tiny):
+    """The multi-device stage object with a single rank: it must drive the real shard (device tensors, greedy
+    feedback, several micro-batches in their own KV slots) to the oracle's tokens.  The message flow between ranks
+    is tested on the CPU (tests/test_stage.py); more than one GPU is not available to these tests."""
+    import socket
+    import torch.distributed as dist
+    from paper_2405_14371_b200.stage import PipelineStage
+
+    wd, wh = tiny
+    sock = socket.socket(); sock.bind(("127.0.0.1", 0)); port = sock.getsockname()[1]; sock.close()
+    os.environ.update(RANK="0", WORLD_SIZE="1", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo")
+    try:
+        MB, Bn, T, S = 2, 2, 16, 5
+        seed, _ = _golden_cfg0()
+        ids = prompt_ids(0, MB * Bn, T, TINY.vocab, seed=seed).reshape(MB, Bn, T)
+        sh = B.Shard(TINY, 0, 2, wd, max_slots=MB * Bn, max_seq=T + S, max_tokens=Bn * T, max_batch=Bn)
+        slots = [[mb * Bn + b for b in range(Bn)] for mb in range(MB)]
+        stage = PipelineStage(sh, TINY.d_model, MB, Bn, slots, torch.device("cuda"))
+        gen = stage.prefill_and_decode([ids[mb].cuda() for mb in range(MB)], T, S).cpu()
+        sh.es_shard_device_status()
+        sh.close()
+    finally:
+        dist.destroy_process_group()
+    want, _, _ = O.generate_greedy(TINY, wh, ids[0, 0], S)          # the golden prompt: margins known to be wide
+    assert gen[:, 0, 0].tolist() == want.tolist()
+    for mb in range(MB):
+        for b in range(Bn):
+            w_t, w_l, _ = O.generate_greedy(TINY, wh, ids[mb, b], S)
+            top2 = w_l.topk(2, dim=-1).values
+            wide = bool(((top2[:, 0] - top2[:, 1]) > 1e-2 * w_l.abs().max()).all())
+            if wide:                                                # near-ties may legitimately flip under fp16
+                assert gen[:, mb, b].tolist() == w_t.tolist()
+
+
 def test_profile_feeds_the_partition_planners(B, tiny):
     """The per-layer profile is the planners' input: measured times for this GPU plus two synthetic slower
     devices (scaled times), activation and memory sizes from the profile."""
