@@ -243,7 +243,7 @@ ES_API es_status_t es_op_rmsnorm(const float *x, const void *gain, void *y, int3
 /* C = A * W^T (+ R):  A fp16 [M, K], W fp16 [N, K], C fp32 [M, N], R fp32 [M, N] or NULL.
  * path: 0 = automatic, 1 = tensor-core (tcgen05) kernel, 2 = weight-streaming kernel (M <= 16),
  * 3 = plain reference kernel, 4 = weight-streaming kernel on tensor cores (M <= 16, K % 256 == 0),
- * 5 = tensor-core kernel on CTA pairs (needs M >= 256 and at least 74 tiles of 256 x 256),
+ * 5 = tensor-core kernel on CTA pairs (needs M >= 256 and at least 40 tiles of 256 x 256),
  * 6 = the same with 256 x 512 tiles per pair. */
 ES_API es_status_t es_op_linear(const void *A, const void *W, const float *R, float *C, int32_t M, int32_t N,
                          int32_t K, int32_t path, void *stream);

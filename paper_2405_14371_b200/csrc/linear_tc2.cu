@@ -341,14 +341,17 @@ es_status_t launch_pair_epi(const TmapSet2& maps, const LinearParams& p, int* st
 
 }  // namespace
 
-// The pair kernel pays off when there are enough 256 x 256 tiles to keep every pair busy.
+// The pair kernel pays off from about 40 tiles of 256 x 256 on: with fewer than the machine's 74 pairs' worth some
+// SMs idle, but a CTA of a pair stages 128 + 128 rows per K block where a single CTA stages 128 + 256, and these
+// launches are bound by what a CTA pulls through L2 (measured: 7B layers at 256 / 768 / 1024 tokens +3 / +3.5 / +6.5 %,
+// 13B layers at 256 tokens +3 %, against a threshold of 74).
 bool linear_tc2_supported(const LinearParams& p, int epi) {
   if (!linear_tc_supported(p, epi)) return false;
   const int out = (epi == EPI_SWIGLU) ? BN2 / 2 : BN2;
   if (epi == EPI_QKV)
     for (int s = 0; s < 3; ++s) if (p.seg_rows[s] % out) return false;
   const long long tiles = (long long)((p.M + 2 * BM2 - 1) / (2 * BM2)) * ((p.N + out - 1) / out);
-  return p.M >= 2 * BM2 && tiles >= 74;
+  return p.M >= 2 * BM2 && tiles >= 40;
 }
 
 // K slices for a plain product with too few 256 x 256 tiles for the machine's 74 pairs (1 = do not use the pair
