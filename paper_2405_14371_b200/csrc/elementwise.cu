@@ -117,9 +117,8 @@ __global__ void __launch_bounds__(THREADS) splitk_reduce_kernel(const float* __r
   const float4* src = reinterpret_cast<const float4*>(part + (int64_t)r * N);
   const float4* rs = res ? reinterpret_cast<const float4*>(res + (int64_t)r * ldo) : nullptr;
   float4* dst = reinterpret_cast<float4*>(out + (int64_t)r * ldo);
-  auto finish = [&](int c) {
-    float4 a = rs ? rs[c] : make_float4(0.f, 0.f, 0.f, 0.f);
-    // eight slices are requested at a time and then added in slice order
+  // a = the residual element; then the slices, eight requested at a time and added in slice order
+  auto finish = [&](int c, float4 a) {
     for (int s0 = 0; s0 < k_splits; s0 += 8) {
       float4 v[8];
 #pragma unroll
@@ -134,16 +133,24 @@ __global__ void __launch_bounds__(THREADS) splitk_reduce_kernel(const float* __r
   };
   float4 v[REGS];
   float ss = 0.f;
+  // The residual may alias the output, so the compiler cannot move a column's residual load above the previous
+  // column's store and a thread would wait out one memory round trip per column; a thread reads and writes only
+  // its own elements, so all its residual elements are requested up front.
+#pragma unroll
+  for (int i = 0; i < REGS; ++i) {
+    const int c = threadIdx.x + i * THREADS;
+    v[i] = (rs && c < n4) ? rs[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
 #pragma unroll
   for (int i = 0; i < REGS; ++i) {
     const int c = threadIdx.x + i * THREADS;
     if (c < n4) {
-      v[i] = finish(c);
+      v[i] = finish(c, v[i]);
       ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
     }
   }
   for (int c = threadIdx.x + REGS * THREADS; c < n4; c += THREADS) {
-    const float4 t = finish(c);
+    const float4 t = finish(c, rs ? rs[c] : make_float4(0.f, 0.f, 0.f, 0.f));
     ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
   }
   if (gain == nullptr) return;                       // uniform over the CTA
