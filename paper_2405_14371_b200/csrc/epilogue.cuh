@@ -218,6 +218,39 @@ __device__ __forceinline__ void epi_qkv_chunk32(const LinearParams& p, int m, in
   for (int q = 0; q < 4; ++q) reinterpret_cast<uint4*>(dst)[q] = o[q];
 }
 
+// epi_qkv_pair with the row's lookups (slot, position, page) done once by the caller: row = qkv_row(p, m).
+__device__ __forceinline__ void epi_qkv_pair_row(const LinearParams& p, const QkvRow& row, int n, float v0, float v1) {
+  if (!row.valid || n >= p.N) return;
+  const int nq = p.Hq * p.hd, nkv = p.Hkv * p.hd;
+  if (n < nq + nkv) {
+    const int c = (n < nq ? n : n - nq) % p.hd;
+    const int i = c >> 1;
+    const float cs = p.rope_cos[row.rope_off + i];
+    const float sn = p.rope_sin[row.rope_off + i];
+    const float r0 = v0 * cs - v1 * sn;
+    const float r1 = v0 * sn + v1 * cs;
+    v0 = r0;
+    v1 = r1;
+  }
+  const __half2 hv = __floats2half2_rn(v0, v1);
+  if (n < nq) {
+    *reinterpret_cast<__half2*>(p.out_f16 + row.q_off + n) = hv;
+    return;
+  }
+  const bool is_k = n < nq + nkv;
+  const int kn = is_k ? n - nq : n - nq - nkv;
+  const int g = kn / p.hd;
+  const int c = kn - g * p.hd;
+  *reinterpret_cast<__half2*>((is_k ? p.k_cache : p.v_cache) + row.kv_off + (int64_t)g * p.P * p.hd + c) = hv;
+}
+
+// epi_pair for a caller that finishes many pairs of the same row m: row = qkv_row(p, m) (used by the QKV form only)
+template <int EPI>
+__device__ __forceinline__ void epi_pair_row(const LinearParams& p, const QkvRow& row, int m, int n, float v0, float v1) {
+  if (EPI == EPI_QKV) epi_qkv_pair_row(p, row, n, v0, v1);
+  else epi_pair<EPI>(p, m, n, v0, v1);
+}
+
 // ---- the same chunks stored through a per-warp shared-memory tile -------------------------------
 // A thread that owns 32 adjacent columns of ONE row would store 16 bytes into a row of its own: 32 rows per
 // instruction, half a 32-byte sector each.  The variants below are called by a whole warp whose lane l owns

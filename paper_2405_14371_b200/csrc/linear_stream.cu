@@ -192,6 +192,10 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
     __syncthreads();
   }
 
+  // lane m finishes activation row m: its slot, position and KV page are looked up once, not per pair of columns
+  QkvRow qrow;
+  if (EPI == EPI_QKV) qrow = qkv_row(p, lane < MB ? lane : p.M);
+
   // ---- "chunk being consumed" cursor ----
   int cur_i = 0, cur_cc = 0;
   float acc0[MB], acc1[MB];
@@ -230,7 +234,7 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
         if (lane == m) { v0 = acc0[m]; v1 = acc1[m]; }
       const int u = u0 + warp + cur_i * WARPS;
       const int n = (EPI == EPI_SWIGLU) ? u : u * 2;
-      if (lane < MB) epi_pair<EPI>(p, lane, n, v0, v1);
+      if (lane < MB) epi_pair_row<EPI>(p, qrow, lane, n, v0, v1);
 #pragma unroll
       for (int m = 0; m < MB; ++m) acc0[m] = acc1[m] = 0.f;
       cur_cc = 0;

@@ -131,6 +131,12 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
     __syncthreads();
   }
 
+  // In the unit epilogue below thread i always finishes activation row (i / 8) % (NT * 8) (the loop over idx runs
+  // at most once: RG * 8 * NT * 8 <= MTHREADS): its slot, position and KV page are looked up once.
+  static_assert(RG * 8 * NT * 8 <= MTHREADS, "one epilogue element per thread");
+  QkvRow qrow;
+  if (EPI == EPI_QKV) qrow = qkv_row(p, (threadIdx.x >> 3) % (NT * 8));
+
   float acc[RG][NT][4];
 #pragma unroll
   for (int rg = 0; rg < RG; ++rg)
@@ -191,7 +197,7 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
         }
         const int u = u0 + cur_i;
         const int n = (EPI == EPI_SWIGLU) ? u * COLS + rg * 8 + pr : u * COLS + rg * 16 + 2 * pr;
-        epi_pair<EPI>(p, m, n, v0, v1);
+        epi_pair_row<EPI>(p, qrow, m, n, v0, v1);       // idx == threadIdx.x: the row is the one looked up before the loop
       }
       cur_cc = 0;
       ++cur_i;
