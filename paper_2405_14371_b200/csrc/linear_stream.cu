@@ -202,8 +202,17 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
 #pragma unroll
   for (int m = 0; m < MB; ++m) acc0[m] = acc1[m] = 0.f;
 
+  // plain epilogue: the two residual elements lane m will add at the end of a unit are requested when the unit
+  // begins (the same lane reads and later writes them, so this is safe when the residual aliases the output)
+  float rpre0 = 0.f, rpre1 = 0.f;
   auto consume = [&](const uint4 (&w0)[U], const uint4 (&w1)[U]) {
     const int kb = cur_cc * CHUNK_K + lane * 8;
+    if (EPI == EPI_F32 && cur_cc == 0 && p.res != nullptr && lane < MB && lane < p.M) {
+      const int n = (u0 + warp + cur_i * WARPS) * 2;
+      const int64_t o = (int64_t)lane * p.ldo + n;
+      if (n < p.N) rpre0 = p.res[o];
+      if (n + 1 < p.N) rpre1 = p.res[o + 1];
+    }
 #pragma unroll
     for (int j = 0; j < U; ++j) {
       const int k = kb + j * 256;
@@ -234,7 +243,20 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
         if (lane == m) { v0 = acc0[m]; v1 = acc1[m]; }
       const int u = u0 + warp + cur_i * WARPS;
       const int n = (EPI == EPI_SWIGLU) ? u : u * 2;
-      if (lane < MB) epi_pair_row<EPI>(p, qrow, lane, n, v0, v1);
+      if (lane < MB) {
+        if (EPI == EPI_F32) {
+          // epi_f32_pair with the residual already in registers
+          if (lane < p.M && n < p.N) {
+            const int64_t o = (int64_t)lane * p.ldo + n;
+            const bool two = (n + 1 < p.N);
+            if (p.res != nullptr) { v0 += rpre0; if (two) v1 += rpre1; }
+            p.out_f32[o] = v0;
+            if (two) p.out_f32[o + 1] = v1;
+          }
+        } else {
+          epi_pair_row<EPI>(p, qrow, lane, n, v0, v1);
+        }
+      }
 #pragma unroll
       for (int m = 0; m < MB; ++m) acc0[m] = acc1[m] = 0.f;
       cur_cc = 0;
