@@ -33,7 +33,9 @@ Pins (tests/test_oracle_pins.py): brute-force scalar-loop attention on tiny inpu
 rows sum to 1, RoPE identity at position 0 / norm preservation / relative-position property /
 hand-computed rotation, RMSNorm closed form on constant vectors, silu special values, zeroed
 Wo/Wd make a layer the identity, zero Wq gives running means of v, GQA == MHA with repeated kv
-weights, form A == form B, split invariance at every cut, batch-row independence, the
+weights, form A == form B, split invariance at every cut, batch-row independence, the output
+layer against closed forms and hand-computed numbers (constant vector, a 2 x 3 case, a square
+matrix, identity layers so the logits are the output layer of the last token's embedding), the
 parameter counts behind the paper's memory table, and greedy tie-breaking on a hand-made tie.
 Absolute logits of random-weight models have no printed reference value in the paper: for
 those the parity is unpinned beyond the invariants above.

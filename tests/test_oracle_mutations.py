@@ -18,7 +18,9 @@ def _all_pins():
              "test_rmsnorm_constant_vector_closed_form", "test_rmsnorm_unit_rms_scale_invariance_and_gain",
              "test_rmsnorm_eps_inside_sqrt", "test_silu_special_values", "test_zero_output_projections_make_layers_identity",
              "test_layer_against_handwritten_single_token", "test_decode_step_equals_prefill_of_extended_sequence",
-             "test_causality_future_tokens_do_not_matter", "test_greedy_lowest_index_on_tie"]
+             "test_causality_future_tokens_do_not_matter", "test_greedy_lowest_index_on_tie",
+             "test_lm_head_constant_vector_closed_form", "test_lm_head_hand_computed_two_by_three",
+             "test_lm_head_square_matrix_is_used_row_by_row", "test_shard_logits_are_the_output_layer_of_the_last_position"]
     fns = [getattr(pins, n) for n in names]
     fns += [lambda hq=hq, hkv=hkv: pins.test_attention_matches_bruteforce(hq, hkv) for hq, hkv in ((4, 4), (4, 2), (4, 1))]
     fns += [pins.test_attention_with_query_offset_matches_bruteforce]
@@ -108,7 +110,27 @@ def _greedy_last(logits):
     return torch.where(logits == m, idx, torch.full_like(idx, -1)).max(dim=-1).values
 
 
+def _lm_head_no_norm(x_last, final_norm, w_lm, eps, dtype=torch.float32):
+    return x_last.to(dtype) @ w_lm.to(dtype).T
+
+
+def _lm_head_gain_before_division(x_last, final_norm, w_lm, eps, dtype=torch.float32):
+    y = x_last * final_norm.to(dtype)
+    return (y / torch.sqrt((y * y).mean(dim=-1, keepdim=True) + eps)) @ w_lm.to(dtype).T
+
+
+def _lm_head_untransposed(x_last, final_norm, w_lm, eps, dtype=torch.float32):
+    w = w_lm.to(dtype)
+    return O.rmsnorm(x_last, final_norm.to(dtype), eps) @ (w if w.shape[0] == w.shape[1] else w.T)
+
+
+def _lm_head_no_gain(x_last, final_norm, w_lm, eps, dtype=torch.float32):
+    return O.rmsnorm(x_last, torch.ones_like(final_norm, dtype=dtype), eps) @ w_lm.to(dtype).T
+
+
 MUTANTS = [
+    ("lm_head", _lm_head_no_norm), ("lm_head", _lm_head_gain_before_division), ("lm_head", _lm_head_untransposed),
+    ("lm_head", _lm_head_no_gain),
     ("rmsnorm", _rms_eps_outside), ("rmsnorm", _rms_no_gain), ("rmsnorm", _rms_sum_not_mean),
     ("apply_rope", _rope_wrong_sign), ("apply_rope", _rope_split_half), ("rope_cos_sin", _rope_wrong_frequency),
     ("causal_attention_matrix", _attn_variant(scale_pow=1.0)), ("causal_attention_matrix", _attn_variant(scale_pow=0.0)),
@@ -144,3 +166,46 @@ def _layer_mutant(kind):
 def test_layer_level_mistakes_are_caught(monkeypatch, kind):
     monkeypatch.setattr(O, "layer_forward_full", _layer_mutant(kind))
     assert _pins_fail(), kind
+
+
+def _wrong_gain_vector(form):
+    """The output layer normalised with the last decoder layer's attention-norm gains instead of its own."""
+    if form == "A":
+        orig = O.shard_forward_full
+
+        def f(model, weights, layer_begin, layer_end, **kw):
+            w = dict(weights)
+            if "final_norm" in w:
+                w["final_norm"] = w["layers"][-1]["attn_norm"]
+            return orig(model, w, layer_begin, layer_end, **kw)
+        return "shard_forward_full", f
+    orig_cls = O.IncrementalShard
+
+    class Wrong(orig_cls):
+        def __init__(self, model, weights, layer_begin, layer_end, dtype=torch.float32):
+            w = dict(weights)
+            if "final_norm" in w:
+                w["final_norm"] = w["layers"][-1]["attn_norm"]
+            super().__init__(model, w, layer_begin, layer_end, dtype)
+    return "IncrementalShard", Wrong
+
+
+@pytest.mark.parametrize("form", ["A", "B"])
+def test_output_layer_with_the_wrong_gain_vector_is_caught(monkeypatch, form):
+    name, mutant = _wrong_gain_vector(form)
+    monkeypatch.setattr(O, name, mutant)
+    assert _pins_fail(), form
+
+
+def test_last_position_rule_of_the_logits_is_pinned(monkeypatch):
+    """Logits taken from the first position instead of the last must fail a pin."""
+    orig = O.lm_head
+    orig_full = O.shard_forward_full
+
+    def f(model, weights, layer_begin, layer_end, **kw):
+        x, logits = orig_full(model, weights, layer_begin, layer_end, **kw)
+        if logits is not None:
+            logits = orig(x[:1, :], weights["final_norm"], weights["lm_head"], model.rms_eps, kw.get("dtype", torch.float32))[0]
+        return x, logits
+    monkeypatch.setattr(O, "shard_forward_full", f)
+    assert _pins_fail()

@@ -286,6 +286,78 @@ def test_greedy_lowest_index_on_tie():
     assert O.greedy(l).tolist() == [1, 0, 0]
 
 
+# ---- output layer ------------------------------------------------------------------------
+
+def test_lm_head_constant_vector_closed_form():
+    # x = c*1: mean of squares is c^2, so logit v = c / sqrt(c^2 + eps) * sum_j g_j W[v, j]
+    c, eps, d = 1.5, 1e-5, 6
+    g = [0.5, 1.0, 1.5, 2.0, 0.25, 3.0]
+    W = [[1, 0, 0, 0, 0, 0], [0, 2, 0, 0, 0, -1], [1, 1, 1, 1, 1, 1], [0.5, -0.5, 0.25, -0.25, 2.0, 0.0]]
+    x = torch.full((1, d), c, dtype=torch.float64)
+    got = O.lm_head(x, torch.tensor(g, dtype=torch.float64), torch.tensor(W, dtype=torch.float64), eps, torch.float64)
+    assert got.shape == (1, 4)
+    for v in range(4):
+        want = c / math.sqrt(c * c + eps) * sum(g[j] * W[v][j] for j in range(d))
+        assert abs(float(got[0, v]) - want) < 1e-12
+
+
+def test_lm_head_hand_computed_two_by_three():
+    # d = 3, V = 2, non-constant x, two rows; every number below is written out by hand with scalar arithmetic
+    eps = 0.25
+    xs = [[1.0, -2.0, 3.0], [0.5, 0.0, -1.5]]
+    g = [2.0, 0.5, -1.0]
+    W = [[1.0, 2.0, 3.0], [-1.0, 0.5, 4.0]]
+    got = O.lm_head(torch.tensor(xs, dtype=torch.float64), torch.tensor(g, dtype=torch.float64),
+                    torch.tensor(W, dtype=torch.float64), eps, torch.float64)
+    assert got.shape == (2, 2)
+    for b, x in enumerate(xs):
+        r = math.sqrt((x[0] * x[0] + x[1] * x[1] + x[2] * x[2]) / 3.0 + eps)
+        n = [x[0] / r * g[0], x[1] / r * g[1], x[2] / r * g[2]]
+        for v in range(2):
+            want = n[0] * W[v][0] + n[1] * W[v][1] + n[2] * W[v][2]
+            assert abs(float(got[b, v]) - want) < 1e-12
+    # row 0 spelled out once more as plain numbers: mean of squares 14/3, r = sqrt(14/3 + 1/4)
+    r0 = math.sqrt(14.0 / 3.0 + 0.25)
+    assert abs(float(got[0, 0]) - (2.0 - 2.0 - 9.0) / r0) < 1e-12
+    assert abs(float(got[0, 1]) - (-2.0 - 0.5 - 12.0) / r0) < 1e-12
+
+
+def test_lm_head_square_matrix_is_used_row_by_row():
+    # V == d: logit v is the product with ROW v of the matrix (a transposed operand changes the result)
+    eps, d = 1e-5, 4
+    W = torch.tensor([[1.0, 2.0, 3.0, 4.0], [0.0, 1.0, 0.0, 0.0], [5.0, 0.0, 0.0, 0.0], [0.0, 0.0, 0.0, 7.0]], dtype=torch.float64)
+    x = torch.tensor([[1.0, 1.0, -1.0, 2.0]], dtype=torch.float64)
+    r = math.sqrt((1.0 + 1.0 + 1.0 + 4.0) / 4.0 + eps)
+    got = O.lm_head(x, torch.ones(d, dtype=torch.float64), W, eps, torch.float64)[0]
+    want = [(1.0 + 2.0 - 3.0 + 8.0) / r, 1.0 / r, 5.0 / r, 14.0 / r]
+    for v in range(4):
+        assert abs(float(got[v]) - want[v]) < 1e-12
+
+
+def test_shard_logits_are_the_output_layer_of_the_last_position():
+    # Wo = Wd = 0 makes every decoder layer the identity, so the logits of both forms must be the output
+    # layer (final-norm gains, not a decoder layer's) applied to the LAST prompt token's embedding row
+    w = _rand_weights(SMALL, 3)
+    for lw in w["layers"]:
+        lw["wo"].zero_(); lw["w_down"].zero_()
+    ids = torch.tensor([3, 1, 4, 1, 5])
+    d, V, eps = SMALL.d_model, SMALL.vocab, SMALL.rms_eps
+    e = w["tok_embedding"][5].double().tolist()
+    g = w["final_norm"].double().tolist()
+    Wl = w["lm_head"].double().tolist()
+    r = math.sqrt(sum(t * t for t in e) / d + eps)
+    want = torch.tensor([sum(e[j] / r * g[j] * Wl[v][j] for j in range(d)) for v in range(V)], dtype=torch.float64)
+    _, la = O.shard_forward_full(SMALL, w, 0, 3, ids=ids, dtype=torch.float64)
+    assert la.shape == (V,) and torch.allclose(la, want, atol=1e-12)
+    sh = O.IncrementalShard(SMALL, w, 0, 3, torch.float64)
+    for t in ids.tolist():
+        _, lb = sh.step(token=t)
+    assert torch.allclose(lb, want, atol=1e-12)
+    # a shard that does not end at the last layer has no output layer
+    wa = dict(w); wa["layers"] = w["layers"][:2]
+    assert O.shard_forward_full(SMALL, wa, 0, 2, ids=ids)[1] is None
+
+
 # ---- shapes: the paper's memory table ------------------------------------------------------
 
 def test_parameter_counts_match_paper_memory_table():
