@@ -190,7 +190,10 @@ ES_API es_status_t es_shard_device_status(es_shard_t *shard);
  * bytes those launches had to read (N*K*2 each) and their number. */
 typedef enum {
   ES_KT_EMBED = 0, ES_KT_RMSNORM = 1, ES_KT_QKV = 2, ES_KT_ATTENTION = 3, ES_KT_O = 4, ES_KT_GATE_UP = 5,
-  ES_KT_DOWN = 6, ES_KT_LM_HEAD = 7, ES_KT_ARGMAX = 8, ES_KT_SET_CTX = 9, ES_KT_COUNT = 10
+  ES_KT_DOWN = 6, ES_KT_LM_HEAD = 7, ES_KT_ARGMAX = 8, ES_KT_SET_CTX = 9,
+  ES_KT_FINISH = 10,  /* epilogue kernel of a K-sliced product (SwiGLU / QKV forms) */
+  ES_KT_REDUCE = 11,  /* slice reduction + residual (+ RMSNorm for the next product) of a K-sliced product */
+  ES_KT_COUNT = 12
 } es_kernel_category_t;
 ES_API es_status_t es_shard_set_kernel_timing(es_shard_t *shard, int32_t enabled);
 /* The same record split by kernel category: three arrays of ES_KT_COUNT entries (any may be NULL):
@@ -199,6 +202,21 @@ ES_API es_status_t es_shard_set_kernel_timing(es_shard_t *shard, int32_t enabled
 ES_API es_status_t es_shard_kernel_timing_detail(es_shard_t *shard, double *ms, double *bytes, int64_t *launches);
 ES_API es_status_t es_shard_kernel_timing(es_shard_t *shard, double *total_ms, double *weight_bytes,
                                           int64_t *launches);
+
+/* Timing from inside a step (Sec. "Profiling" asks what each layer costs on the device; this is the same
+ * question one level down, per kernel of a replayed step).  While on, every kernel of a pass records the
+ * earliest time any of its CTAs started and the latest time any of its warps finished (%globaltimer,
+ * one atomic per CTA / warp) into a slot of the scratch buffer; decode steps are still replayed as graphs
+ * with programmatic dependent launch, so the overlap between consecutive kernels is what it is in a normal
+ * step (the stamps cost well under a microsecond per kernel).  Switching it on or off drops the captured
+ * graphs.  es_shard_step_timing synchronises and returns, for each launch of the most recently enqueued
+ * pass in launch order (up to `capacity`; *n = how many there were): its category, its start and end in
+ * microseconds relative to the first start of the pass, and its algorithmic bytes (as in
+ * es_shard_kernel_timing_detail).  A decode-attention entry covers the split and the merge kernel.
+ * At most 2048 launches per pass are stamped; later ones are left out. */
+ES_API es_status_t es_shard_set_step_timing(es_shard_t *shard, int32_t enabled);
+ES_API es_status_t es_shard_step_timing(es_shard_t *shard, int32_t capacity, int32_t *n, int32_t *category,
+                                        double *start_us, double *end_us, double *bytes);
 
 /* Number of kernels this shard has launched (graph replays count their nodes). */
 ES_API int64_t es_shard_launch_count(const es_shard_t *shard);
@@ -226,7 +244,11 @@ ES_API const char *es_version(void);
  * g(m, S + {j}, j) = min over (i, k) of max(g(i, S, k), O(i-1)/Bw(k, j), t_comp(i..m-1, j)), memory
  * Req(i..m-1) <= Mem(j) per device; the source device holds the first range, which contains layer 0 and
  * may contain more.  *bottleneck = the slowest stage's time (its reciprocal is the pipeline throughput).
- * Exact; cost O(N^2 2^M M^2), M <= 20. */
+ * Exact; cost O(N^2 2^M M^2), M <= 20.
+ *
+ * Both planners refuse (ES_ERR_UNSUPPORTED, nothing computed) a problem whose table would exceed 4 GiB of host
+ * memory — (N + 1) * 2^M * M cells of 12 bytes for es_partition_throughput (N = 82 layers: M <= 17), N * M cells
+ * of 12 + 8 M bytes for es_partition_latency — and report an allocation failure the same way. */
 ES_API es_status_t es_partition_latency(int32_t N, int32_t M, const double *t_comp, const double *O, const double *Req,
                                         const double *Mem, const double *Bw, int32_t *assign, double *latency);
 ES_API es_status_t es_partition_throughput(int32_t N, int32_t M, const double *t_comp, const double *O,

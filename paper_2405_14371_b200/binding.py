@@ -22,7 +22,8 @@ STATUS_NAMES = {
     9: "ES_ERR_UNSUPPORTED",
 }
 ES_DTYPE_F16, ES_DTYPE_F32, ES_DTYPE_I32 = 0, 1, 2
-KERNEL_CATEGORIES = ("embed", "rmsnorm", "qkv", "attention", "o", "gate_up", "down", "lm_head", "argmax", "set_ctx")
+KERNEL_CATEGORIES = ("embed", "rmsnorm", "qkv", "attention", "o", "gate_up", "down", "lm_head", "argmax", "set_ctx",
+                     "splitk_finish", "splitk_reduce")
 LAYER_KEYS = ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down")
 
 
@@ -82,6 +83,8 @@ def _load() -> C.CDLL:
         "es_shard_set_kernel_timing": (i32, [vp, i32]),
         "es_shard_kernel_timing": (i32, [vp, P(C.c_double), P(C.c_double), P(C.c_int64)]),
         "es_shard_kernel_timing_detail": (i32, [vp, P(C.c_double), P(C.c_double), P(C.c_int64)]),
+        "es_shard_set_step_timing": (i32, [vp, i32]),
+        "es_shard_step_timing": (i32, [vp, i32, P(i32), P(i32), P(C.c_double), P(C.c_double), P(C.c_double)]),
         "es_shard_destroy": (None, [vp]),
         "es_last_error": (C.c_char_p, []),
         "es_version": (C.c_char_p, []),
@@ -107,7 +110,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ("es_shard_workspace_bytes es_shard_create es_shard_prefill es_shard_prefill_ragged es_shard_decode_step es_shard_handoff "
            "es_layer_profile es_shard_set_profiling es_shard_reset_slots es_shard_set_page_table es_shard_set_graphs "
-           "es_partition_latency es_partition_throughput es_shard_device_status es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_kernel_timing_detail es_shard_destroy es_last_error es_version es_op_rmsnorm "
+           "es_partition_latency es_partition_throughput es_shard_device_status es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_kernel_timing_detail es_shard_set_step_timing es_shard_step_timing es_shard_destroy es_last_error es_version es_op_rmsnorm "
            "es_op_linear es_op_linear_splitk_workspace_bytes es_op_linear_splitk es_op_prefill_attention es_op_decode_attention_scratch_bytes es_op_decode_attention "
            "es_op_decode_attention_static_capacity es_op_decode_attention_static").split()
 
@@ -271,6 +274,19 @@ class Shard:
         ms, by, cnt = (C.c_double * n)(), (C.c_double * n)(), (C.c_int64 * n)()
         _check(lib.es_shard_kernel_timing_detail(self._handle, ms, by, cnt))
         return {name: {"ms": ms[i], "bytes": by[i], "launches": cnt[i]} for i, name in enumerate(KERNEL_CATEGORIES)}
+
+    def es_shard_set_step_timing(self, enabled: bool) -> None:
+        _check(lib.es_shard_set_step_timing(self._handle, int(enabled)))
+
+    def es_shard_step_timing(self) -> list:
+        """One dict per launch of the last enqueued pass, in launch order: category name, start / end in
+        microseconds from the first start of the pass, algorithmic bytes."""
+        cap = 2048
+        n = C.c_int32(0)
+        cat, t0, t1, by = (C.c_int32 * cap)(), (C.c_double * cap)(), (C.c_double * cap)(), (C.c_double * cap)()
+        _check(lib.es_shard_step_timing(self._handle, cap, C.byref(n), cat, t0, t1, by))
+        return [{"category": KERNEL_CATEGORIES[cat[i]], "start_us": t0[i], "end_us": t1[i], "bytes": by[i]}
+                for i in range(min(n.value, cap))]
 
     @property
     def n_pages(self) -> int:

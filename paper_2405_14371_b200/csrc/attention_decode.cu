@@ -26,6 +26,7 @@ constexpr int DWARPS = 8;
 template <int HD, int G, bool PRE>
 __global__ void __launch_bounds__(DWARPS * 32, PRE ? 1 : 2) decode_attn_split_kernel(const DecodeAttnParams p) {
   pdl_launch_dependents();
+  stamp_begin(p.stamp);
   constexpr int E = HD / 32;
   __shared__ __align__(16) float q_s[G][HD];
   __shared__ float sm_o[DWARPS][G][HD];
@@ -40,11 +41,20 @@ __global__ void __launch_bounds__(DWARPS * 32, PRE ? 1 : 2) decode_attn_split_ke
   // tokens cached by earlier passes.  The newest token's K / V and the query come from the kernel
   // just before this one and are read after the wait.
   const int slot = p.kv.slots ? p.kv.slots[b] : b;
-  const int ctx_old = p.ctx_len[slot];
+  // a context length beyond the sequence's page list is clamped to it: no page index is ever read past the row
+  const int ctx_old = min(p.ctx_len[slot], p.kv.pages_per_slot * p.kv.P - p.ctx_add);
   const int ctx = ctx_old + p.ctx_add;
   const int tokens_per_split = p.pages_per_split * p.kv.P;
   const int t_begin = split * tokens_per_split;
-  if (t_begin >= ctx) { pdl_wait(); return; }
+  if (t_begin >= ctx) {
+    pdl_wait();
+    // an empty context with a single split has no merge kernel behind it: the output rows are zeros
+    if (p.n_splits == 1)
+      for (int i = threadIdx.x; i < G * HD; i += DWARPS * 32)
+        p.out[((int64_t)b * p.Hq + (g * G + i / HD)) * HD + (i % HD)] = __float2half_rn(0.f);
+    stamp_end(p.stamp);
+    return;
+  }
   const int t_end = min(ctx, t_begin + tokens_per_split);
   const float scale = rsqrtf((float)HD);
   constexpr bool PRELOAD = PRE && (G <= 2);     // K row of the first block kept in registers across the wait
@@ -199,6 +209,7 @@ __global__ void __launch_bounds__(DWARPS * 32, PRE ? 1 : 2) decode_attn_split_ke
       if (c == 0) { dst[HD] = mm; dst[HD + 1] = ll; }
     }
   }
+  stamp_end(p.stamp);
 }
 
 template <int HD>
@@ -207,7 +218,7 @@ __global__ void __launch_bounds__(HD) decode_attn_merge_kernel(const DecodeAttnP
   const int h = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
   pdl_wait();
   const int slot = p.kv.slots ? p.kv.slots[b] : b;
-  const int ctx = p.ctx_len[slot] + p.ctx_add;
+  const int ctx = min(p.ctx_len[slot] + p.ctx_add, p.kv.pages_per_slot * p.kv.P);
   const int tokens_per_split = p.pages_per_split * p.kv.P;
   int active = (ctx + tokens_per_split - 1) / tokens_per_split;
   active = active < p.n_splits ? active : p.n_splits;
@@ -221,6 +232,7 @@ __global__ void __launch_bounds__(HD) decode_attn_merge_kernel(const DecodeAttnP
     ll += src[(int64_t)s * (HD + 2) + HD + 1] * f;
   }
   p.out[((int64_t)b * p.Hq + h) * HD + c] = __float2half_rn(active > 0 ? o / ll : 0.f);
+  stamp_end(p.stamp);
 }
 
 template <int HD, int G>

@@ -65,6 +65,7 @@ __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) {
 template <int G, bool DB>
 __global__ void __launch_bounds__(MW * 32, DB ? 2 : 3) decode_attn_mma_kernel(const DecodeAttnParams p) {
   pdl_launch_dependents();
+  stamp_begin(p.stamp);
   constexpr int HD = MHD;
   __shared__ float sm_o[MW][G][HD];
   __shared__ float sm_m[MW][G];
@@ -75,11 +76,20 @@ __global__ void __launch_bounds__(MW * 32, DB ? 2 : 3) decode_attn_mma_kernel(co
   const int g = lane >> 2, t = lane & 3;
   // read-only state of earlier passes (slot list, page map, context length) may be read before the wait
   const int slot = p.kv.slots ? p.kv.slots[b] : b;
-  const int ctx_old = p.ctx_len[slot];
+  // a context length beyond the sequence's page list is clamped to it: no page index is ever read past the row
+  const int ctx_old = min(p.ctx_len[slot], p.kv.pages_per_slot * p.kv.P - p.ctx_add);
   const int ctx = ctx_old + p.ctx_add;
   const int tokens_per_split = p.pages_per_split * p.kv.P;
   const int t_begin = split * tokens_per_split;
-  if (t_begin >= ctx) { pdl_wait(); return; }
+  if (t_begin >= ctx) {
+    pdl_wait();
+    // an empty context with a single split has no merge kernel behind it: the output rows are zeros
+    if (p.n_splits == 1)
+      for (int i = threadIdx.x; i < G * HD; i += MW * 32)
+        p.out[((int64_t)b * p.Hq + ((int64_t)kvh * G + i / HD)) * HD + (i % HD)] = __float2half_rn(0.f);
+    stamp_end(p.stamp);
+    return;
+  }
   const int t_end = min(ctx, t_begin + tokens_per_split);
   const float scale = rsqrtf((float)HD);
   const int64_t kv_head_off = (int64_t)kvh * p.kv.head_stride;
@@ -225,6 +235,7 @@ __global__ void __launch_bounds__(MW * 32, DB ? 2 : 3) decode_attn_mma_kernel(co
       if (c == 0) { dst[HD] = mm; dst[HD + 1] = ll; }
     }
   }
+  stamp_end(p.stamp);
 }
 
 template <int G>

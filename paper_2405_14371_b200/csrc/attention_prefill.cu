@@ -5,6 +5,7 @@
 // the running-softmax statistics are reduced with warp shuffles; for the value product the head
 // dimension is spread over the lanes and the 32 probabilities are broadcast lane by lane.
 #include "es_internal.cuh"
+#include "launch.cuh"
 
 namespace es {
 
@@ -23,13 +24,14 @@ __global__ void __launch_bounds__(PWARPS * 32) prefill_attn_simt_kernel(const Pr
   const int slot = p.kv.slots ? p.kv.slots[b] : b;
   const bool active = t < p.T;
   const float scale = rsqrtf((float)HD);
+  stamp_begin(p.stamp);
   if (active) {
     const __half* qrow = p.q + (((int64_t)b * p.T + t) * p.Hq + h) * HD;
 #pragma unroll
     for (int e = 0; e < E; ++e) q_s[warp][lane * E + e] = __half2float(qrow[lane * E + e]) * scale;
   }
   __syncwarp();
-  if (!active) return;
+  if (!active) { stamp_end(p.stamp); return; }
 
   float acc[E];
 #pragma unroll
@@ -88,6 +90,7 @@ __global__ void __launch_bounds__(PWARPS * 32) prefill_attn_simt_kernel(const Pr
   const float inv = 1.0f / l;
 #pragma unroll
   for (int e = 0; e < E; ++e) orow[e] = __float2half_rn(acc[e] * inv);
+  stamp_end(p.stamp);
 }
 
 }  // namespace

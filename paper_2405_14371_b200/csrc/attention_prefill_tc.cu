@@ -51,6 +51,7 @@ struct AttnArgs {
   int B, T, Hq, Hkv;
   int paged, P, pages_per_slot;
   float scale_log2e;         // log2(e) / sqrt(hd)
+  unsigned long long* stamp; // optional time stamps of the launch, nullptr = none
 };
 
 template <int HD>
@@ -69,6 +70,7 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
   using L = AttnSmem<HD>;
   constexpr int HALVES = L::HALVES;
   pdl_launch_dependents();
+  stamp_begin(a.stamp);
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* q_s = smem;                                   // [HALVES][128 rows][128 B]
@@ -322,6 +324,7 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
     if (*abort_flag) __nanosleep(100000);
     tmem_dealloc(tmem_base, TMEM_ALLOC);
   }
+  stamp_end(a.stamp);
 }
 
 bool is_paged(const PrefillAttnParams& p) { return p.kv.block_table != nullptr; }
@@ -335,6 +338,7 @@ es_status_t launch_hd(const AttnMaps& maps, const PrefillAttnParams& p, cudaStre
     configured = true;
   }
   AttnArgs a{};
+  a.stamp = p.stamp;
   a.out = p.out;
   a.block_table = p.kv.block_table;
   a.slots = p.kv.slots;

@@ -18,12 +18,16 @@ void* g_scratch_ptr[MAX_DEVICES] = {};
 
 // In host code `g_decode_scratch` is only a handle for the symbol, not a device address; the real
 // address is looked up once per device, with that device current.
-es_status_t scratch_address(void** out) {
+es_status_t scratch_address(void** out, cudaStream_t stream) {
   int dev = -1;
   ES_CUDA_CHECK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= MAX_DEVICES) return es::fail(ES_ERR_UNSUPPORTED, "device index %d not supported", dev);
   std::lock_guard<std::mutex> lock(g_mu);
   if (!g_scratch_ptr[dev]) {
+    // the look-up may load the module, which a stream capture in progress does not survive
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) == cudaSuccess && cap != cudaStreamCaptureStatusNone)
+      return es::fail(ES_ERR_STATE, "the first call on a device must come before any stream capture");
     void* p = nullptr;
     ES_CUDA_CHECK(cudaGetSymbolAddress(&p, g_decode_scratch));
     if (!p) return es::fail(ES_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
@@ -48,6 +52,11 @@ es_status_t es_op_decode_attention_static(const void* q, const void* k_pages, co
   if (B <= 0 || Hq <= 0 || Hkv <= 0 || page_tokens <= 0 || pages_per_seq <= 0 || max_ctx <= 0)
     return fail(ES_ERR_INVALID_ARG, "bad sizes");
   if (max_ctx > page_tokens * pages_per_seq) return fail(ES_ERR_RANGE, "max_ctx exceeds the block table");
+  // shapes first: the capacity test below computes with them
+  if (hd != 64 && hd != 128) return fail(ES_ERR_SHAPE, "head_dim must be 64 or 128");
+  if (Hq % Hkv != 0) return fail(ES_ERR_SHAPE, "Hq must be a multiple of Hkv");
+  const int group = Hq / Hkv;
+  if (group != 1 && group != 2 && group != 4 && group != 8) return fail(ES_ERR_SHAPE, "Hq / Hkv must be 1, 2, 4 or 8");
   DecodeAttnParams p{};
   p.q = (const __half*)q; p.out = (__half*)out; p.ctx_len = ctx_len; p.ctx_add = 0;
   p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.hd = hd;
@@ -60,7 +69,7 @@ es_status_t es_op_decode_attention_static(const void* q, const void* k_pages, co
     return fail(ES_ERR_WORKSPACE, "this call needs %zu bytes of split-KV scratch but the built-in array holds %zu; "
                 "use es_op_decode_attention with a caller buffer", need, STATIC_SCRATCH_BYTES);
   void* scratch = nullptr;
-  ES_TRY(scratch_address(&scratch));
+  ES_TRY(scratch_address(&scratch, (cudaStream_t)stream));
   // Nothing has to be cleared: every split that the merge step reads is written earlier in this same call.
   p.part = (float*)scratch;
   return launch_decode_attention(p, (cudaStream_t)stream, nullptr);

@@ -8,8 +8,9 @@ namespace {
 
 // x[m, :] = table[ids[m], :] widened to fp32.  One CTA per row.
 __global__ void embed_kernel(const int* __restrict__ ids, const __half* __restrict__ table,
-                             float* __restrict__ x, int d, int vocab) {
+                             float* __restrict__ x, int d, int vocab, unsigned long long* stamp) {
   pdl_launch_dependents();
+  stamp_begin(stamp);
   pdl_wait();
   const int m = blockIdx.x;
   int id = ids[m];
@@ -24,6 +25,7 @@ __global__ void embed_kernel(const int* __restrict__ ids, const __half* __restri
     dst[2 * c] = make_float4(a.x, a.y, b.x, b.y);
     dst[2 * c + 1] = make_float4(e.x, e.y, f.x, f.y);
   }
+  stamp_end(stamp);
 }
 
 __device__ __forceinline__ float block_sum(float v, float* red) {
@@ -54,9 +56,10 @@ __global__ void __launch_bounds__(THREADS) rmsnorm_kernel(const float* __restric
                                                               const __half* __restrict__ gain,
                                                               __half* __restrict__ y, int d, float eps,
                                                               int64_t row_stride, int64_t row_offset,
-                                                              const int* __restrict__ last_of) {
+                                                              const int* __restrict__ last_of, unsigned long long* stamp) {
   __shared__ float red[32];
   pdl_launch_dependents();
+  stamp_begin(stamp);
   pdl_wait();
   const int r = blockIdx.x;
   // source row: r * row_stride + row_offset, or with last_of the last of the first last_of[r] rows of block r
@@ -96,6 +99,7 @@ __global__ void __launch_bounds__(THREADS) rmsnorm_kernel(const float* __restric
     dst[2 * c] = __floats2half2_rn(t.x * inv * ga.x, t.y * inv * ga.y);
     dst[2 * c + 1] = __floats2half2_rn(t.z * inv * gb.x, t.w * inv * gb.y);
   }
+  stamp_end(stamp);
 }
 
 // Finishes a split-K product: out[r, :] = (res ? res[r, :] : 0) + part[0, r, :] + part[1, r, :] + ...
@@ -107,9 +111,10 @@ template <int THREADS, int REGS>
 __global__ void __launch_bounds__(THREADS) splitk_reduce_kernel(const float* __restrict__ part, int k_splits,
                                                                 const float* res, float* out, int M, int N,
                                                                 int64_t ldo, const __half* __restrict__ gain,
-                                                                __half* __restrict__ y, float eps) {
+                                                                __half* __restrict__ y, float eps, unsigned long long* stamp) {
   __shared__ float red[32];
   pdl_launch_dependents();
+  stamp_begin(stamp);
   pdl_wait();
   const int r = blockIdx.x;
   const int n4 = N / 4;
@@ -153,7 +158,7 @@ __global__ void __launch_bounds__(THREADS) splitk_reduce_kernel(const float* __r
     const float4 t = finish(c, rs ? rs[c] : make_float4(0.f, 0.f, 0.f, 0.f));
     ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
   }
-  if (gain == nullptr) return;                       // uniform over the CTA
+  if (gain == nullptr) { stamp_end(stamp); return; }   // uniform over the CTA
   const float total = block_sum(ss, red);
   const float inv = 1.0f / sqrtf(total / (float)N + eps);
   __half2* yd = reinterpret_cast<__half2*>(y + (int64_t)r * N);
@@ -173,13 +178,16 @@ __global__ void __launch_bounds__(THREADS) splitk_reduce_kernel(const float* __r
     yd[2 * c] = __floats2half2_rn(t.x * inv * ga.x, t.y * inv * ga.y);
     yd[2 * c + 1] = __floats2half2_rn(t.z * inv * gb.x, t.w * inv * gb.y);
   }
+  stamp_end(stamp);
 }
 
 // Greedy token: index of the largest logit, the lowest index on ties.  One CTA per sequence.
-__global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ logits, int* __restrict__ out, int V) {
+__global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ logits, int* __restrict__ out, int V,
+                                                      unsigned long long* stamp) {
   __shared__ float bv[8];
   __shared__ int bi[8];
   pdl_launch_dependents();
+  stamp_begin(stamp);
   pdl_wait();
   const float* row = logits + (int64_t)blockIdx.x * V;
   float best = -INFINITY;
@@ -208,11 +216,14 @@ __global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ l
     }
     if (lane == 0) out[blockIdx.x] = (idx == 0x7fffffff) ? 0 : idx;
   }
+  stamp_end(stamp);
 }
 
 // ctx_len[slots[b]] = add ? ctx_len[..] + value : value; with `values` the value of row b is values[b]
-__global__ void set_ctx_kernel(int* ctx_len, const int* slots, int B, int value, int add, const int* values) {
+__global__ void set_ctx_kernel(int* ctx_len, const int* slots, int B, int value, int add, const int* values,
+                               unsigned long long* stamp) {
   pdl_launch_dependents();
+  stamp_begin(stamp);
   pdl_wait();
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < B) {
@@ -220,53 +231,56 @@ __global__ void set_ctx_kernel(int* ctx_len, const int* slots, int B, int value,
     const int v = values ? values[b] : value;
     ctx_len[s] = add ? ctx_len[s] + v : v;
   }
+  stamp_end(stamp);
 }
 
 }  // namespace
 
 es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, int d, int vocab,
-                         cudaStream_t s, int64_t* launches, bool pdl) {
+                         cudaStream_t s, int64_t* launches, bool pdl, unsigned long long* stamp) {
   if (M <= 0) return ES_OK;
-  ES_CUDA_CHECK(launch_kernel(embed_kernel, dim3(M), dim3(128), 0, s, pdl, ids, table, x, d, vocab));
+  ES_CUDA_CHECK(launch_kernel(embed_kernel, dim3(M), dim3(128), 0, s, pdl, ids, table, x, d, vocab, stamp));
   if (launches) ++*launches;
   return ES_OK;
 }
 
 es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M, int d, float eps,
                            int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches, bool pdl,
-                           const int* last_of) {
+                           const int* last_of, unsigned long long* stamp) {
   if (M <= 0) return ES_OK;
   if (M <= WIDE_ROWS_MAX)
-    ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset, last_of));
+    ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset, last_of, stamp));
   else
-    ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset, last_of));
+    ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset, last_of, stamp));
   if (launches) ++*launches;
   return ES_OK;
 }
 
-es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches, bool pdl) {
+es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches, bool pdl,
+                          unsigned long long* stamp) {
   if (B <= 0) return ES_OK;
-  ES_CUDA_CHECK(launch_kernel(argmax_kernel, dim3(B), dim3(256), 0, s, pdl, logits, out, V));
+  ES_CUDA_CHECK(launch_kernel(argmax_kernel, dim3(B), dim3(256), 0, s, pdl, logits, out, V, stamp));
   if (launches) ++*launches;
   return ES_OK;
 }
 
 es_status_t launch_splitk_reduce(const float* part, int k_splits, const float* res, float* out, int M, int N, int64_t ldo,
-                                 const __half* gain, __half* y, float eps, cudaStream_t s, int64_t* launches, bool pdl) {
+                                 const __half* gain, __half* y, float eps, cudaStream_t s, int64_t* launches, bool pdl,
+                                 unsigned long long* stamp) {
   if (M <= 0 || N <= 0) return ES_OK;
   if (N % 4 != 0 || ldo % 4 != 0) return fail(ES_ERR_SHAPE, "split-K reduction needs N and the row stride to be multiples of 4");
   if (M <= WIDE_ROWS_MAX)
-    ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps));
+    ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps, stamp));
   else
-    ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps));
+    ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps, stamp));
   if (launches) ++*launches;
   return ES_OK;
 }
 
 es_status_t launch_set_ctx(int* ctx_len, const int* slots, int B, int value, int add, cudaStream_t s,
-                           int64_t* launches, bool pdl, const int* values) {
+                           int64_t* launches, bool pdl, const int* values, unsigned long long* stamp) {
   if (B <= 0) return ES_OK;
-  ES_CUDA_CHECK(launch_kernel(set_ctx_kernel, dim3((B + 63) / 64), dim3(64), 0, s, pdl, ctx_len, slots, B, value, add, values));
+  ES_CUDA_CHECK(launch_kernel(set_ctx_kernel, dim3((B + 63) / 64), dim3(64), 0, s, pdl, ctx_len, slots, B, value, add, values, stamp));
   if (launches) ++*launches;
   return ES_OK;
 }

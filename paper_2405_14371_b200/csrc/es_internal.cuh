@@ -91,6 +91,8 @@ struct LinearParams {
   int pair_nacc;
   // k_splits > 1 on the tensor-core path: the CTA-pair kernel computes the slices (else the single-CTA kernel)
   int split_on_pairs;
+  // optional time stamps of this launch (see launch.cuh), nullptr = none
+  unsigned long long* stamp;
 };
 
 // Kernel families.  Each returns after enqueuing; `launches` is incremented per kernel launched.
@@ -114,7 +116,8 @@ size_t linear_tc_split_workspace_bytes();
 // out[m, :] = (res ? res[m, :] : 0) + sum over slices (ascending) of part[s, m, :]; with gain != nullptr also
 // y[m, :] = rmsnorm(out[m, :]) * gain in fp16.  N % 4 == 0.  res may alias out.
 es_status_t launch_splitk_reduce(const float* part, int k_splits, const float* res, float* out, int M, int N, int64_t ldo,
-                                 const __half* gain, __half* y, float eps, cudaStream_t s, int64_t* launches, bool pdl = false);
+                                 const __half* gain, __half* y, float eps, cudaStream_t s, int64_t* launches, bool pdl = false,
+                                 unsigned long long* stamp = nullptr);
 // CTA-pair (cta_group::2) variant for large M; uses the same tensor maps
 bool linear_tc2_supported(const LinearParams& p, int epi);
 int linear_tc2_splits(const LinearParams& p, int epi);   // K slices for a plain product on CTA pairs (1 = not this way)
@@ -129,17 +132,18 @@ bool tma_available();
 
 // ---- element-wise / reductions ---------------------------------------------------------------
 es_status_t launch_embed(const int* ids, const __half* table, float* x, int M, int d, int vocab,
-                         cudaStream_t s, int64_t* launches, bool pdl = false);
+                         cudaStream_t s, int64_t* launches, bool pdl = false, unsigned long long* stamp = nullptr);
 // row r of y = rmsnorm(row (r * row_stride + row_offset) of x); with last_of (device, [M]) the source row is
 // r * row_stride + last_of[r] - 1 instead (the last of the first last_of[r] rows of block r)
 es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M, int d, float eps,
                            int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches,
-                           bool pdl = false, const int* last_of = nullptr);
+                           bool pdl = false, const int* last_of = nullptr, unsigned long long* stamp = nullptr);
 es_status_t launch_argmax(const float* logits, int* out, int B, int V, cudaStream_t s, int64_t* launches,
-                          bool pdl = false);
+                          bool pdl = false, unsigned long long* stamp = nullptr);
 // ctx_len[slots[b]] = (add ? ctx_len[slots[b]] : 0) + (values ? values[b] : value)
 es_status_t launch_set_ctx(int* ctx_len, const int* slots, int B, int value, int add, cudaStream_t s,
-                           int64_t* launches, bool pdl = false, const int* values = nullptr);
+                           int64_t* launches, bool pdl = false, const int* values = nullptr,
+                           unsigned long long* stamp = nullptr);
 
 // ---- attention -------------------------------------------------------------------------------
 // K/V addressing shared by both attention kernels: token t of sequence b, kv head g lives at
@@ -169,6 +173,7 @@ struct PrefillAttnParams {
   int64_t kv_rows;          // rows of the K / V matrices as 2-D [rows, row width] views (tensor-core kernel)
   const TcMaps* tc_maps;    // pre-encoded maps {q, k, v} or nullptr: encode per launch
   int* status;
+  unsigned long long* stamp;   // optional time stamps of this launch, nullptr = none
 };
 // path: 0 = automatic, 1 = tensor-core (tcgen05) kernel, 2 = CUDA-core kernel
 es_status_t launch_prefill_attention(const PrefillAttnParams& p, cudaStream_t s, int64_t* launches, int path = 0, bool pdl = false);
@@ -186,6 +191,7 @@ struct DecodeAttnParams {
   float* part;            // scratch [B, Hq, n_splits, hd + 2]
   int B, Hq, Hkv, hd;
   int n_splits, pages_per_split;
+  unsigned long long* stamp;   // optional time stamps of the launch (split and merge kernels share them), nullptr = none
 };
 size_t decode_attention_scratch_bytes(int B, int Hq, int hd, int n_splits);
 void choose_splits(int max_ctx, int P, int B, int Hkv, int group, int* n_splits, int* pages_per_split);

@@ -16,6 +16,26 @@ namespace es {
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Optional time stamps of a launch: slot[0] takes the earliest %globaltimer value any CTA of the launch saw at
+// its start, slot[STAMP_SLOTS] the latest any warp saw at its end (nanoseconds): the slots of a pass form two
+// arrays, so that one fill can reset the starts to "never" and another the ends to 0.  nullptr (the default) =
+// no stamps.
+// With them the time a replayed step spends in each of its kernels can be read from inside the step, with the
+// programmatic overlap between consecutive kernels left as it is.
+constexpr int STAMP_SLOTS = 2048;
+__device__ __forceinline__ unsigned long long stamp_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void stamp_begin(unsigned long long* slot) {
+  if (slot != nullptr && threadIdx.x == 0) atomicMin(slot, stamp_now());
+}
+// called by every thread that leaves the kernel (one atomic per warp)
+__device__ __forceinline__ void stamp_end(unsigned long long* slot) {
+  if (slot != nullptr && (threadIdx.x & 31) == 0) atomicMax(slot + STAMP_SLOTS, stamp_now());
+}
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
                                  bool pdl, Args&&... args) {

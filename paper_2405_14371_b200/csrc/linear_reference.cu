@@ -3,6 +3,7 @@
 // as the path for shapes the tensor-core kernel does not take.  64x64 output tile, 16-deep K
 // slices staged through shared memory as fp32, 4x4 outputs per thread.
 #include "epilogue.cuh"
+#include "launch.cuh"
 
 namespace es {
 
@@ -19,6 +20,7 @@ __global__ void __launch_bounds__(256) linear_reference_kernel(const LinearParam
   const int tid = threadIdx.x;
   const int tx = tid & 15, ty = tid >> 4;
   const int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
+  stamp_begin(p.stamp);
 
   float acc[DUAL ? 2 : 1][4][4];
 #pragma unroll
@@ -83,6 +85,7 @@ __global__ void __launch_bounds__(256) linear_reference_kernel(const LinearParam
       epi_pair<EPI>(p, m, n + 2, acc[0][i][2], acc[0][i][3]);
     }
   }
+  stamp_end(p.stamp);
 }
 
 }  // namespace

@@ -51,6 +51,7 @@ __device__ __forceinline__ void fma8(float& acc, const uint4& w, const uint4& a)
 template <int MB, int EPI, bool NORM, int U, bool A_SMEM>
 __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_stream_kernel(const LinearParams p) {
   pdl_launch_dependents();
+  stamp_begin(p.stamp);
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __half* a_s = reinterpret_cast<__half*>(smem_raw);
   __shared__ float red[WARPS];
@@ -274,6 +275,7 @@ __global__ void __launch_bounds__(THREADS, (U == 2 && MB <= 2) ? 4 : 2) linear_s
       if (c + 3 < total) issue(b1w0, b1w1);
     }
   }
+  stamp_end(p.stamp);
 }
 
 template <int MB, int EPI, bool NORM, int U, bool A_SMEM>

@@ -53,6 +53,7 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
 template <int NT, int EPI, bool A_SMEM, int RG>
 __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const LinearParams p, int a_stride) {
   pdl_launch_dependents();
+  stamp_begin(p.stamp);
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __half* a_s = reinterpret_cast<__half*>(smem_raw);                 // [NT*8][a_stride], padded rows
   __shared__ float red[2][MW][RG][NT][32][4];
@@ -212,6 +213,7 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
       if (c + 3 < total) issue(b1w0, b1w1);
     }
   }
+  stamp_end(p.stamp);
 }
 
 // ---- K sliced across CTAs (activations too large for shared memory) ---------------------------------
@@ -222,6 +224,7 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
 template <int NT, int EPI>
 __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_ks_kernel(const LinearParams p, int a_stride, int n_col_ctas) {
   pdl_launch_dependents();
+  stamp_begin(p.stamp);
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __half* a_s = reinterpret_cast<__half*>(smem_raw);                 // [NT*8][a_stride]: this CTA's K slice of the activations
 
@@ -350,6 +353,7 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_ks_kernel(const
       if (c + 3 < total) issue(b1w0, b1w1);
     }
   }
+  stamp_end(p.stamp);
 }
 
 // Adds the K slices of one output pair in slice order and applies the epilogue (SwiGLU / QKV forms;
@@ -357,6 +361,7 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_ks_kernel(const
 template <int EPI>
 __global__ void __launch_bounds__(256) splitk_finish_kernel(const LinearParams p) {
   pdl_launch_dependents();
+  stamp_begin(p.stamp);
   pdl_wait();
   const int pairs = (EPI == EPI_SWIGLU) ? p.N : (p.N + 1) / 2;
   const int64_t part_cols = (EPI == EPI_SWIGLU) ? 2 * (int64_t)p.N : p.N;
@@ -383,6 +388,7 @@ __global__ void __launch_bounds__(256) splitk_finish_kernel(const LinearParams p
     }
     epi_pair<EPI>(p, m, n, v0, v1);
   }
+  stamp_end(p.stamp);
 }
 
 template <int NT, int EPI>

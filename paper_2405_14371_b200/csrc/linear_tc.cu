@@ -59,6 +59,7 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
   constexpr int ACC_COLS = Cfg::TMEM_COLS;                    // TMEM columns of one accumulator buffer
 
   pdl_launch_dependents();
+  stamp_begin(p.stamp);
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   unsigned char* a_tiles = smem;
@@ -243,6 +244,7 @@ linear_tc_kernel(const __grid_constant__ TmapSet maps, const LinearParams p, int
     if (*abort_flag) __nanosleep(100000);     // let copies still in flight land before the CTA's memory is released
     tmem_dealloc(tmem_base, Cfg::TMEM_ALLOC);
   }
+  stamp_end(p.stamp);
 }
 
 // ---- host side -----------------------------------------------------------------------------------

@@ -64,6 +64,7 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
   constexpr int NBUF = 2 / NACC;                                   // accumulator buffers in the 512 TMEM columns
   static_assert(STAGES2 <= MAX_STAGES2 && STAGES2 * STAGE_BYTES == RING_BYTES2, "ring layout");
   pdl_launch_dependents();
+  stamp_begin(p.stamp);
 
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -277,6 +278,7 @@ linear_tc2_kernel(const __grid_constant__ TmapSet2 maps, const LinearParams p, i
     if (*abort_flag) __nanosleep(100000);
     tmem_dealloc_pair(tmem_base, 512);
   }
+  stamp_end(p.stamp);
 }
 
 template <int EPI, int NACC>

@@ -5,6 +5,7 @@
 #include <math.h>
 
 #include <limits>
+#include <new>
 #include <vector>
 
 #include "es_internal.cuh"
@@ -27,13 +28,15 @@ es_status_t check_common(int N, int M, const double* t_comp, const double* O, co
   return ES_OK;
 }
 
-}  // namespace
+// Largest dynamic-programming table either planner will allocate; beyond it the call is refused with
+// ES_ERR_UNSUPPORTED instead of exhausting host memory.
+constexpr double TABLE_BYTES_MAX = 4.0 * 1024 * 1024 * 1024;
 
-extern "C" {
-
-es_status_t es_partition_latency(int32_t N, int32_t M, const double* t_comp, const double* O, const double* Req,
-                                 const double* Mem, const double* Bw, int32_t* assign, double* latency) {
+es_status_t latency_impl(int32_t N, int32_t M, const double* t_comp, const double* O, const double* Req,
+                         const double* Mem, const double* Bw, int32_t* assign, double* latency) {
   ES_TRY(check_common(N, M, t_comp, O, Req, Mem, Bw, assign, latency));
+  if ((double)N * M * (12.0 + 8.0 * M) > TABLE_BYTES_MAX)
+    return es::fail(ES_ERR_UNSUPPORTED, "N x M cells with M memory budgets each would exceed 4 GiB (N = %d, M = %d)", N, M);
   // DP(i, j): least time of layers 0..i with layer i on device j (Eq. 4); choice(i, j): device of layer i-1.
   // Each cell also carries the memory its own best path has placed on every device, which is how the
   // algorithm's "update memory" step is read: a move to device j is allowed only if that path still has room.
@@ -83,11 +86,15 @@ es_status_t es_partition_latency(int32_t N, int32_t M, const double* t_comp, con
   return ES_OK;
 }
 
-es_status_t es_partition_throughput(int32_t N, int32_t M, const double* t_comp, const double* O, const double* Req,
-                                    const double* Mem, const double* Bw, int32_t* assign, double* bottleneck) {
+es_status_t throughput_impl(int32_t N, int32_t M, const double* t_comp, const double* O, const double* Req,
+                            const double* Mem, const double* Bw, int32_t* assign, double* bottleneck) {
   ES_TRY(check_common(N, M, t_comp, O, Req, Mem, Bw, assign, bottleneck));
   if (M > 20) return es::fail(ES_ERR_UNSUPPORTED, "the subset table is 2^M: at most 20 devices");
+  if (N >= (1 << 24)) return es::fail(ES_ERR_UNSUPPORTED, "at most 2^24 layers");
   const int S_ALL = 1 << M;
+  // (N + 1) x 2^M x M cells of one double and one packed back-pointer
+  if ((double)(N + 1) * S_ALL * M * 12.0 > TABLE_BYTES_MAX)
+    return es::fail(ES_ERR_UNSUPPORTED, "the table of (N + 1) x 2^M x M cells would exceed 4 GiB (N = %d, M = %d)", N, M);
   // prefix sums of time per device and of memory: t_comp^{i->m, j} and Req_{i->m}
   std::vector<double> tp((size_t)(N + 1) * M, 0.0), rp(N + 1, 0.0);
   for (int i = 0; i < N; ++i) {
@@ -99,7 +106,7 @@ es_status_t es_partition_throughput(int32_t N, int32_t M, const double* t_comp, 
   // contiguous range, in the order used) with k last.  c counts layers, 1 <= c <= N.
   auto idx = [&](int c, int S, int k) { return ((size_t)c * S_ALL + S) * M + k; };
   std::vector<double> g((size_t)(N + 1) * S_ALL * M, INF);
-  std::vector<int> from_c((size_t)(N + 1) * S_ALL * M, -1), from_k((size_t)(N + 1) * S_ALL * M, -1);
+  std::vector<int> from((size_t)(N + 1) * S_ALL * M, -1);      // previous (layer count, last device) as count * 32 + device
   // the source device holds the first shard: layer 0 is pinned to it, and it may keep more layers
   for (int c = 1; c <= N; ++c)
     if (rp[c] - rp[0] <= Mem[0]) g[idx(c, 1, 0)] = seg_t(0, c, 0);
@@ -118,7 +125,7 @@ es_status_t es_partition_throughput(int32_t N, int32_t M, const double* t_comp, 
             if (rp[m] - rp[c] > Mem[j]) break;
             const double t = fmax(cur, fmax(tc, seg_t(c, m, j)));
             const size_t at = idx(m, S2, j);
-            if (t < g[at]) { g[at] = t; from_c[at] = c; from_k[at] = k; }
+            if (t < g[at]) { g[at] = t; from[at] = c * 32 + k; }
           }
         }
       }
@@ -133,16 +140,39 @@ es_status_t es_partition_throughput(int32_t N, int32_t M, const double* t_comp, 
   int c = N, S = bS, k = bk;
   while (c > 0) {
     const size_t at = idx(c, S, k);
-    const int pc = from_c[at] < 0 ? 0 : from_c[at];
+    const int pc = from[at] < 0 ? 0 : from[at] / 32;
     for (int i = pc; i < c; ++i) assign[i] = k;
-    if (from_c[at] < 0) break;
-    const int pk = from_k[at];
+    if (from[at] < 0) break;
+    const int pk = from[at] % 32;
     S &= ~(1 << k);
     k = pk;
     c = pc;
   }
   *bottleneck = best;
   return ES_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+// Nothing is thrown across the C boundary: running out of host memory is reported as a status.
+es_status_t es_partition_latency(int32_t N, int32_t M, const double* t_comp, const double* O, const double* Req,
+                                 const double* Mem, const double* Bw, int32_t* assign, double* latency) {
+  try {
+    return latency_impl(N, M, t_comp, O, Req, Mem, Bw, assign, latency);
+  } catch (const std::bad_alloc&) {
+    return es::fail(ES_ERR_UNSUPPORTED, "out of host memory for the planner's table (N = %d, M = %d)", N, M);
+  }
+}
+
+es_status_t es_partition_throughput(int32_t N, int32_t M, const double* t_comp, const double* O, const double* Req,
+                                    const double* Mem, const double* Bw, int32_t* assign, double* bottleneck) {
+  try {
+    return throughput_impl(N, M, t_comp, O, Req, Mem, Bw, assign, bottleneck);
+  } catch (const std::bad_alloc&) {
+    return es::fail(ES_ERR_UNSUPPORTED, "out of host memory for the planner's table (N = %d, M = %d)", N, M);
+  }
 }
 
 }  // extern "C"

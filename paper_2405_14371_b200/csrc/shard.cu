@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "es_internal.cuh"
+#include "launch.cuh"
 
 namespace es {
 
@@ -71,7 +72,7 @@ struct Layout {
   size_t page_elems;   // halves in one page of one of K / V
   size_t kv_bytes;
   size_t off_x, off_h, off_q, off_ao, off_act, off_logits, off_next, off_hlast, off_part, off_cos, off_sin,
-      off_table, off_ctx, off_slots, off_status, off_splitk;
+      off_table, off_ctx, off_slots, off_status, off_splitk, off_stamps;
   size_t scratch_bytes;
 };
 
@@ -125,6 +126,7 @@ Layout make_layout(const es_model_desc_t& d, int begin, int end) {
   L.off_slots = take(2 * B * 4);       // slots, then the prompt lengths of a ragged prefill
   L.off_status = take(256);
   L.off_splitk = take(d.max_tokens > 2 ? linear_tc_split_workspace_bytes() : 0);   // split-K partial sums of short prefills
+  L.off_stamps = take((size_t)2 * STAMP_SLOTS * sizeof(unsigned long long));
   L.scratch_bytes = o;
   return L;
 }
@@ -198,6 +200,12 @@ struct es_shard {
   std::vector<double> kt_pair_bytes;    // algorithmic bytes of each pair
   size_t kt_used = 0;
   int kt_next_cat = 0;
+  // time stamps written by the kernels of the last enqueued (or captured) pass: see es_shard_set_step_timing
+  unsigned long long* stamps = nullptr;   // device: STAMP_SLOTS earliest starts, then STAMP_SLOTS latest ends
+  bool step_timing = false;
+  int st_used = 0;
+  std::vector<int> st_cat;
+  std::vector<double> st_bytes;
 
   __half* k_pages(int li) const { return kv + (size_t)(2 * li) * lay.n_pages * lay.page_elems; }
   __half* v_pages(int li) const { return kv + (size_t)(2 * li + 1) * lay.n_pages * lay.page_elems; }
@@ -263,6 +271,14 @@ es_status_t kt_begin(es_shard* s) {
   return ES_OK;
 }
 
+// Time-stamp slot for the next launch (nullptr unless step timing is on), tagged like an event pair.
+unsigned long long* next_stamp(es_shard* s, int cat, double bytes) {
+  if (!s->step_timing || s->st_used >= STAMP_SLOTS) return nullptr;
+  s->st_cat.push_back(cat);
+  s->st_bytes.push_back(bytes);
+  return s->stamps + s->st_used++;
+}
+
 es_status_t kt_end(es_shard* s, int cat, double bytes) {
   if (!s->kernel_timing) return ES_OK;
   ES_CUDA_CHECK(cudaEventRecord(s->kt_events[s->kt_used + 1], s->stream));
@@ -272,10 +288,13 @@ es_status_t kt_end(es_shard* s, int cat, double bytes) {
   return ES_OK;
 }
 
-es_status_t run_linear(es_shard* s, const LinearParams& p, int epi) {
+es_status_t run_linear(es_shard* s, const LinearParams& p0, int epi) {
+  LinearParams p = p0;
+  const double bytes = (double)p.N * p.K * 2.0 * (epi == EPI_SWIGLU ? 2.0 : 1.0);
+  p.stamp = next_stamp(s, s->kt_next_cat, bytes);
   ES_TRY(kt_begin(s));
   ES_TRY(dispatch_linear(s, p, epi));
-  return kt_end(s, s->kt_next_cat, (double)p.N * p.K * 2.0 * (epi == EPI_SWIGLU ? 2.0 : 1.0));
+  return kt_end(s, s->kt_next_cat, bytes);
 }
 
 LinearParams base_params(const es_shard* s, int M, int T, bool decode) {
@@ -317,9 +336,10 @@ es_status_t run_linear_sliced(es_shard* s, LinearParams& p, int epi, bool pdl) {
   p.k_splits = splits;
   p.part = s->splitk;
   ES_TRY(run_linear(s, p, epi));
+  p.stamp = next_stamp(s, ES_KT_FINISH, 0.0);
   ES_TRY(kt_begin(s));
   ES_TRY(launch_splitk_finish(p, epi, s->stream, &s->launches, pdl));
-  return kt_end(s, s->kt_next_cat, 0.0);
+  return kt_end(s, ES_KT_FINISH, 0.0);
 }
 
 // Parameters of the four linear layers of decoder layer li (kind: 0 qkv, 1 o, 2 gate/up, 3 down).
@@ -376,12 +396,20 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   s->pdl_now = pdl;
   const bool fuse_norm = M <= 16 && linear_stream_can_fuse_norm(M);
   bool h_ready = false;   // s->h already holds the normalised input of the coming layer
+  if (s->step_timing) {
+    s->st_used = 0;
+    s->st_cat.clear();
+    s->st_bytes.clear();
+    ES_CUDA_CHECK(cudaMemsetAsync(s->stamps, 0xFF, STAMP_SLOTS * sizeof(unsigned long long), s->stream));
+    ES_CUDA_CHECK(cudaMemsetAsync(s->stamps + STAMP_SLOTS, 0, STAMP_SLOTS * sizeof(unsigned long long), s->stream));
+  }
   if (s->has_emb) {
     prof_mark(s, pi, 0);
     ES_TRY(kt_begin(s));
     // the first kernel of a pass is launched with a full dependency: everything from earlier passes
     // has completed before any kernel of this pass begins
-    ES_TRY(launch_embed(ids, s->emb, s->x, M, d.d_model, d.vocab, s->stream, &s->launches, false));
+    ES_TRY(launch_embed(ids, s->emb, s->x, M, d.d_model, d.vocab, s->stream, &s->launches, false,
+                        next_stamp(s, ES_KT_EMBED, (double)M * d.d_model * 6.0)));
     ES_TRY(kt_end(s, ES_KT_EMBED, (double)M * d.d_model * 6.0));
     prof_mark(s, pi, 1);
     ++pi;
@@ -394,7 +422,8 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     const bool pdl0 = (li == 0 && !s->has_emb) ? false : pdl;     // first kernel of the pass: full dependency
     if (!fuse_norm && !h_ready) {
       ES_TRY(kt_begin(s));
-      ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl0));
+      ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl0,
+                            nullptr, next_stamp(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0)));
       ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0));
     }
     h_ready = false;
@@ -418,6 +447,7 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       a.q = s->q; a.out = s->ao; a.kv = kvv; a.ctx_len = s->ctx_len; a.ctx_add = 1; a.part = s->part;
       a.B = B; a.Hq = d.n_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim;
       a.n_splits = s->lay.n_splits; a.pages_per_split = s->lay.pages_per_split;
+      a.stamp = next_stamp(s, ES_KT_ATTENTION, 0.0);
       ES_TRY(launch_decode_attention(a, s->stream, &s->launches, pdl));
     } else {
       PrefillAttnParams a{};
@@ -425,6 +455,7 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       a.kv_rows = (int64_t)s->lay.n_pages * d.n_kv_heads * d.kv_page_tokens;
       a.status = s->status;
       a.tc_maps = s->attn_maps_valid ? &s->attn_maps[li] : nullptr;
+      a.stamp = next_stamp(s, ES_KT_ATTENTION, 0.0);
       ES_TRY(launch_prefill_attention(a, s->stream, &s->launches, 0, pdl));
     }
     ES_TRY(kt_end(s, ES_KT_ATTENTION, 0.0));
@@ -439,8 +470,9 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
         ES_TRY(run_linear(s, p, epi));
         ES_TRY(kt_begin(s));
         ES_TRY(launch_splitk_reduce(s->splitk, splits, p.res, p.out_f32, M, p.N, p.ldo, (const __half*)w.ffn_norm, s->h,
-                                    d.rms_eps, s->stream, &s->launches, pdl));
-        ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * (8.0 + 4.0 * splits + 2.0)));
+                                    d.rms_eps, s->stream, &s->launches, pdl,
+                                    next_stamp(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + 2.0))));
+        ES_TRY(kt_end(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + 2.0)));
         o_split = true;
       } else {
         ES_TRY(run_linear(s, p, epi));
@@ -449,7 +481,8 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     xin = s->x;
     if (!fuse_norm && !o_split) {
       ES_TRY(kt_begin(s));
-      ES_TRY(launch_rmsnorm(s->x, (const __half*)w.ffn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl));
+      ES_TRY(launch_rmsnorm(s->x, (const __half*)w.ffn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl,
+                            nullptr, next_stamp(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0)));
       ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0));
     }
     {
@@ -470,8 +503,9 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
         ES_TRY(kt_begin(s));
         ES_TRY(launch_splitk_reduce(s->splitk, splits, p.res, p.out_f32, M, p.N, p.ldo,
                                     more ? (const __half*)s->lw[li + 1].attn_norm : nullptr, s->h, d.rms_eps, s->stream,
-                                    &s->launches, pdl));
-        ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * (8.0 + 4.0 * splits + (more ? 2.0 : 0.0))));
+                                    &s->launches, pdl,
+                                    next_stamp(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + (more ? 2.0 : 0.0)))));
+        ES_TRY(kt_end(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + (more ? 2.0 : 0.0))));
         h_ready = more;
       } else {
         ES_TRY(run_linear(s, p, epi));
@@ -485,7 +519,8 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     const bool fuse_head = lens == nullptr && linear_stream_can_fuse_norm(B);
     if (!fuse_head) {
       ES_TRY(kt_begin(s));
-      ES_TRY(launch_rmsnorm(s->x, s->fnorm, s->h_last, B, d.d_model, d.rms_eps, T, T - 1, s->stream, &s->launches, pdl, lens));
+      ES_TRY(launch_rmsnorm(s->x, s->fnorm, s->h_last, B, d.d_model, d.rms_eps, T, T - 1, s->stream, &s->launches, pdl, lens,
+                            next_stamp(s, ES_KT_RMSNORM, (double)B * d.d_model * 6.0)));
       ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)B * d.d_model * 6.0));
     }
     for (int b0 = 0; b0 < B; b0 += 16) {
@@ -501,13 +536,15 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       ES_TRY(run_linear(s, p, EPI_F32));
     }
     ES_TRY(kt_begin(s));
-    ES_TRY(launch_argmax(s->logits, s->next_ids, B, d.vocab, s->stream, &s->launches, pdl));
+    ES_TRY(launch_argmax(s->logits, s->next_ids, B, d.vocab, s->stream, &s->launches, pdl,
+                         next_stamp(s, ES_KT_ARGMAX, (double)B * d.vocab * 4.0)));
     ES_TRY(kt_end(s, ES_KT_ARGMAX, (double)B * d.vocab * 4.0));
     prof_mark(s, pi, 1);
   }
   // the slots' contexts now hold T (prefill) or one more (decode) position
   ES_TRY(kt_begin(s));
-  ES_TRY(launch_set_ctx(s->ctx_len, s->slots_dev, B, decode ? 1 : T, decode ? 1 : 0, s->stream, &s->launches, pdl, lens));
+  ES_TRY(launch_set_ctx(s->ctx_len, s->slots_dev, B, decode ? 1 : T, decode ? 1 : 0, s->stream, &s->launches, pdl, lens,
+                        next_stamp(s, ES_KT_SET_CTX, 0.0)));
   ES_TRY(kt_end(s, ES_KT_SET_CTX, 0.0));
   s->pdl_now = false;
   return ES_OK;
@@ -613,6 +650,7 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
   s->lens_dev = s->slots_dev + desc->max_batch;
   s->status = (int*)(sb + L.off_status);
   s->splitk = desc->max_tokens > 2 ? (float*)(sb + L.off_splitk) : nullptr;
+  s->stamps = (unsigned long long*)(sb + L.off_stamps);
   s->ctx.assign(desc->max_slots, -1);
 
   auto bail = [&](es_status_t st) { delete s; return st; };
@@ -901,6 +939,42 @@ es_status_t es_shard_set_kernel_timing(es_shard_t* s, int32_t enabled) {
   s->kt_used = 0;
   s->kt_cat.clear();
   s->kt_pair_bytes.clear();
+  return ES_OK;
+}
+
+es_status_t es_shard_set_step_timing(es_shard_t* s, int32_t enabled) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  if ((enabled != 0) == s->step_timing) return ES_OK;
+  // captured steps carry (or lack) the stamp slots of their launches: capture afresh
+  ES_CUDA_CHECK(cudaStreamSynchronize(s->stream));
+  for (auto& g : s->graph_cache) if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
+  s->graph_cache.clear();
+  s->step_timing = enabled != 0;
+  s->st_used = 0;
+  s->st_cat.clear();
+  s->st_bytes.clear();
+  return ES_OK;
+}
+
+es_status_t es_shard_step_timing(es_shard_t* s, int32_t capacity, int32_t* n, int32_t* category, double* start_us,
+                                 double* end_us, double* bytes) {
+  if (!s || !n) return fail(ES_ERR_INVALID_ARG, "null argument");
+  if (capacity > 0 && (!category || !start_us || !end_us || !bytes)) return fail(ES_ERR_INVALID_ARG, "null output array");
+  *n = s->st_used;
+  if (s->st_used == 0 || capacity <= 0) return ES_OK;
+  std::vector<unsigned long long> host(2 * (size_t)STAMP_SLOTS);
+  ES_CUDA_CHECK(cudaStreamSynchronize(s->stream));
+  ES_CUDA_CHECK(cudaMemcpy(host.data(), s->stamps, host.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+  unsigned long long t0 = ~0ull;
+  for (int i = 0; i < s->st_used; ++i) if (host[i] < t0) t0 = host[i];
+  for (int i = 0; i < s->st_used && i < capacity; ++i) {
+    const unsigned long long a = host[i], b = host[STAMP_SLOTS + i];
+    category[i] = s->st_cat[i];
+    bytes[i] = s->st_bytes[i];
+    // a launch that never ran (or whose stamps were lost) reports a negative start
+    start_us[i] = (a == ~0ull) ? -1.0 : (double)(a - t0) * 1e-3;
+    end_us[i] = (a == ~0ull || b < t0) ? -1.0 : (double)(b - t0) * 1e-3;
+  }
   return ES_OK;
 }
 

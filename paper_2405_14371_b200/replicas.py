@@ -10,6 +10,19 @@ import os
 import torch
 
 
+def launch_plan(n_gpus: int, environ, argv):
+    """How a benchmark asked for `n_gpus` replicas should start them.  None: run in this process (one GPU, or
+    this process already is a rank of a running job: WORLD_SIZE is set).  Otherwise the command line that
+    starts the same script with the same arguments as `n_gpus` ranks of one node under torch.distributed.run
+    (rendezvous on 127.0.0.1: the host name of a container may not resolve)."""
+    import sys
+
+    if n_gpus <= 1 or "WORLD_SIZE" in environ:
+        return None
+    return [sys.executable, "-m", "torch.distributed.run", "--standalone", "--nnodes=1", f"--nproc-per-node={n_gpus}",
+            "--local-addr", "127.0.0.1"] + list(argv)
+
+
 def setup(backend: str | None = None):
     """(rank, local_rank, world_size); initialises torch.distributed when WORLD_SIZE > 1."""
     rank = int(os.environ.get("RANK", "0"))

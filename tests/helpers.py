@@ -33,6 +33,20 @@ def rel_err(got: torch.Tensor, want: torch.Tensor) -> float:
     return float((got - want).abs().max() / want.abs().max())
 
 
+def report_err(label: str, value: float) -> float:
+    """Prints a measured parity error (pytest -s / -rP shows it) and, when ES_PARITY_LOG names a file,
+    appends it there as one JSON line, so the worst error per configuration can be tabulated."""
+    import json
+    import os
+
+    print(f"parity {label}: {value:.3e}")
+    path = os.environ.get("ES_PARITY_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps({"label": label, "rel_err": value}) + "\n")
+    return value
+
+
 def host_layer(lw: dict) -> dict:
     return {k: v.cpu() for k, v in lw.items()}
 

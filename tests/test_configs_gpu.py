@@ -7,7 +7,7 @@ import pytest
 import torch
 
 from oracle import decoder as O
-from tests.helpers import device_weights, rel_err
+from tests.helpers import device_weights, rel_err, report_err
 from workload import WORKLOADS, prompt_ids, forced_decode_ids, shard_weights
 
 pytestmark = pytest.mark.gpu
@@ -48,11 +48,11 @@ def test_cfg1_prefill_and_every_decode_step(B):
         sh.es_shard_device_status()
         sh.close()
     torch.cuda.synchronize()
-    assert rel_err(got_prefill, want[:T]) < TOL
+    assert report_err("cfg1 prefill handoff", rel_err(got_prefill, want[:T])) < TOL
     got_dec = torch.stack(rows)
-    assert rel_err(got_dec, want[T:]) < TOL
+    assert report_err("cfg1 decode handoff", rel_err(got_dec, want[T:])) < TOL
     worst = max(rel_err(got_dec[s], want[T + s]) for s in range(S))
-    assert worst < TOL, worst
+    assert report_err("cfg1 decode handoff, worst single step", worst) < TOL, worst
 
 
 def _run_generation(B, wl, wd, batch, stream, decode_steps=None):
@@ -86,8 +86,8 @@ def _run_generation(B, wl, wd, batch, stream, decode_steps=None):
     return pre, torch.stack(rows), (torch.stack(logits) if logits is not None else None), torch.stack(fed), ids
 
 
-@pytest.mark.parametrize("batch,row", [(1, 0), (8, 7)])
-def test_cfg2_full_7b_with_head(B, batch, row):
+@pytest.mark.parametrize("batch,rows", [(1, (0,)), (8, (0, 7))])
+def test_cfg2_full_7b_with_head(B, batch, rows):
     """Full Llama-2-7B, prompt 512, 256 greedy steps.  The oracle is teacher-forced with the tokens the
     GPU generated (near-ties may legitimately flip an argmax under fp16), and checks the sampled batch
     row at every position: hidden states after prefill and after each step, logits of each step."""
@@ -98,14 +98,15 @@ def test_cfg2_full_7b_with_head(B, batch, row):
     stream = torch.cuda.Stream()
     torch.cuda.synchronize()
     pre, dec, logits, fed, ids = _run_generation(B, wl, wd, batch, stream)
-    seq = torch.cat([ids[row].cpu(), fed[:, row].cpu()])                 # T + S tokens actually consumed
-    xs, ls = oracle_streamed(m, wd, 0, m.n_layers, [seq], logits_from=T - 1)
-    want_h, want_l = xs[0], ls[0]                                         # [T+S, d], [S+1, V]
-    assert rel_err(pre[row], want_h[:T]) < TOL
-    assert rel_err(dec[:, row], want_h[T:]) < TOL
-    assert rel_err(logits[:, row], want_l) < TOL
-    agree = (logits[:, row].argmax(-1).cpu() == want_l.argmax(-1)).float().mean()
-    assert agree > 0.9, float(agree)
+    seqs = [torch.cat([ids[row].cpu(), fed[:, row].cpu()]) for row in rows]   # T + S tokens actually consumed
+    xs, ls = oracle_streamed(m, wd, 0, m.n_layers, seqs, logits_from=T - 1)
+    for row, want_h, want_l in zip(rows, xs, ls):                              # [T+S, d], [S+1, V]
+        tag = f"cfg2 batch {batch} row {row}"
+        assert report_err(tag + " prefill hidden", rel_err(pre[row], want_h[:T])) < TOL
+        assert report_err(tag + " decode hidden", rel_err(dec[:, row], want_h[T:])) < TOL
+        assert report_err(tag + " logits", rel_err(logits[:, row], want_l)) < TOL
+        agree = (logits[:, row].argmax(-1).cpu() == want_l.argmax(-1)).float().mean()
+        assert agree > 0.9, float(agree)
 
 
 def test_cfg3_pipeline_of_four_shards(B):
@@ -158,16 +159,23 @@ def test_cfg3_pipeline_of_four_shards(B):
     for mb in (0, MB - 1):
         seq = torch.cat([ids[mb].cpu(), fed[:, mb]])
         xs, ls = oracle_streamed(m, wd, 0, m.n_layers, [seq], logits_from=T - 1)
-        assert rel_err(pre_h[mb], xs[0][:T]) < TOL
-        assert rel_err(hid[:, mb], xs[0][T:]) < TOL
-        assert rel_err(logits[:, mb], ls[0]) < TOL
+        assert report_err(f"cfg3 micro-batch {mb} prefill hidden", rel_err(pre_h[mb], xs[0][:T])) < TOL
+        assert report_err(f"cfg3 micro-batch {mb} decode hidden", rel_err(hid[:, mb], xs[0][T:])) < TOL
+        assert report_err(f"cfg3 micro-batch {mb} logits", rel_err(logits[:, mb], ls[0])) < TOL
 
 
 def test_cfg4_gqa_shard_batch16(B):
     """Llama-2-70B-architecture layers 0-39 (8 KV heads for 64 query heads), batch 16, prompt 1024, 128
-    teacher-forced steps.  The 68 GB of weights exceed what the oracle can hold, so the oracle checks
-    layers 0-3 (a 4-layer shard at the full batch and lengths) on rows 0 and 15 at every position, and
-    the 40-layer shard is checked for the split invariance [0,4) -> [4,40) == [0,40), bit for bit."""
+    teacher-forced steps.  The 68 GB of weights exceed what the host can hold, so the oracle streams them
+    layer by layer.  Three checks:
+    * layers 0-3 (a 4-layer shard at the full batch and lengths) against a live oracle run on rows 0 and 15 at
+      every position, and the split invariance [0,4) -> [4,40) == [0,40), bit for bit;
+    * the full 40-layer handoff of rows 0 and 15, after the prefill and after every decode step, against the
+      oracle's stored digest (tests/golden/cfg4_handoff_digest.npz, written by make_cfg4_golden.py from the
+      oracle alone): the 64 stored columns of every position, and the magnitude and place of every position's
+      largest element;
+    * the first 96 prompt positions of rows 0 and 15 through all 40 layers against a live oracle run (causality
+      makes a prefix self-contained), every column."""
     from tests.helpers import oracle_streamed, slice_weights
     from workload import forced_decode_ids
     wl = WORKLOADS["cfg4"]
@@ -185,16 +193,19 @@ def test_cfg4_gqa_shard_batch16(B):
         a = B.Shard(m, 0, k, slice_weights(wd, m, 0, k), **kw)
         b = B.Shard(m, k, wl.layer_end, slice_weights(wd, m, k, wl.layer_end), **kw)
         full.es_shard_prefill(ids, None, Bn, T, slots)
+        hf = full.es_shard_handoff()[0]
+        pre_full = {r: hf[r].clone() for r in (0, Bn - 1)}
         a.es_shard_prefill(ids, None, Bn, T, slots)
         ha = a.es_shard_handoff()[0]
         pre_a = {r: ha[r].clone() for r in (0, Bn - 1)}
         b.es_shard_prefill(None, ha, Bn, T, slots)
         assert torch.equal(full.es_shard_handoff()[0], b.es_shard_handoff()[0])
         cur = torch.zeros(Bn, dtype=torch.int32, device="cuda")
-        dec_a = []
+        dec_a, dec_full = [], []
         for s in range(S):
             cur.copy_(forced[s])
             full.es_shard_decode_step(cur, None, Bn, slots)
+            dec_full.append(full.es_shard_handoff()[0][:, 0].clone())
             a.es_shard_decode_step(cur, None, Bn, slots)
             ha = a.es_shard_handoff()[0]
             dec_a.append(ha[:, 0].clone())
@@ -209,8 +220,38 @@ def test_cfg4_gqa_shard_batch16(B):
     seqs = [torch.cat([ids[r].cpu(), forced[:, r].cpu()]) for r in (0, Bn - 1)]
     xs, _ = oracle_streamed(m, wd, 0, k, seqs)
     for x, r in zip(xs, (0, Bn - 1)):
-        assert rel_err(pre_a[r], x[:T]) < TOL
-        assert rel_err(dec_a[:, r], x[T:]) < TOL
+        assert report_err(f"cfg4 layers 0-3 row {r} prefill handoff", rel_err(pre_a[r], x[:T])) < TOL
+        assert report_err(f"cfg4 layers 0-3 row {r} decode handoff", rel_err(dec_a[:, r], x[T:])) < TOL
+
+    # full depth, every position, against the stored oracle digest
+    import os
+    import numpy as np
+    g = np.load(os.path.join(os.path.dirname(__file__), "golden", "cfg4_handoff_digest.npz"))
+    assert int(g["n_layers"]) == wl.layer_end and g["rows"].tolist() == [0, Bn - 1]
+    cols = torch.from_numpy(g["cols"]).long()
+    dec_full = torch.stack(dec_full)                                       # [S, Bn, d]
+    for i, r in enumerate((0, Bn - 1)):
+        got = torch.cat([pre_full[r], dec_full[:, r]]).cpu()               # [T+S, d]
+        want_vals = torch.from_numpy(g["values"][i])                       # [T+S, 64]
+        want_max = torch.from_numpy(g["max_abs"][i])                       # [T+S]
+        scale = float(want_max.max())
+        for name, sl in (("prefill", slice(0, T)), ("decode", slice(T, T + S))):
+            e = float((got[sl][:, cols] - want_vals[sl]).abs().max()) / float(want_max[sl].max())
+            assert report_err(f"cfg4 layers 0-39 row {r} {name} handoff (64 stored columns)", e) < TOL
+        gmax = got.abs().max(dim=-1)
+        assert report_err(f"cfg4 layers 0-39 row {r} per-position max |x|",
+                          float((gmax.values - want_max).abs().max()) / scale) < TOL
+        # the place of a position's largest element is unique unless a runner-up is within rounding of it
+        where = torch.from_numpy(g["argmax_abs"][i]).long()
+        at_golden = got.abs().gather(1, where[:, None])[:, 0]
+        assert float(((gmax.values - at_golden) / scale).max()) < TOL
+
+    # full depth, every column, on a prefix of the prompt against a live oracle run
+    P = 96
+    xs, _ = oracle_streamed(m, wd, 0, wl.layer_end, [ids[r, :P].cpu() for r in (0, Bn - 1)])
+    for x, r in zip(xs, (0, Bn - 1)):
+        assert report_err(f"cfg4 layers 0-39 row {r} first {P} positions, all columns",
+                          rel_err(pre_full[r][:P], x)) < TOL
 
 
 @pytest.mark.parametrize("name,layers,Bn,T", [("cfg2_b1", 2, 2, 512), ("cfg4", 1, 2, 1024)])

@@ -203,3 +203,26 @@ def test_decode_attention_paged(B, Bn, Hq, Hkv, hd, P, ctxs):
     for b in range(Bn):
         want = O.causal_attention_matrix(q[b:b + 1].double(), ks[b].double(), vs[b].double(), q_pos0=ctxs[b] - 1)
         assert rel_err(got[b], want.reshape(-1)) < 2e-3
+
+
+@pytest.mark.parametrize("Bn,Hq,Hkv,hd,P,pps", [(2, 4, 4, 64, 16, 3), (9, 32, 8, 128, 64, 5)])
+def test_decode_attention_clamps_context_lengths_to_the_page_list(B, Bn, Hq, Hkv, hd, P, pps):
+    """A context length on the device that exceeds what the sequence's row of the page table can hold is read as
+    "the whole row" (no page index past the row is ever followed), and an empty context gives zeros."""
+    cap = P * pps
+    n_pages = Bn * pps
+    g = torch.Generator().manual_seed(5)
+    perm = torch.randperm(n_pages, generator=g).to(torch.int32).reshape(Bn, pps)
+    kp = torch.randn(n_pages, Hkv, P, hd, generator=g).half()
+    vp = torch.randn(n_pages, Hkv, P, hd, generator=g).half()
+    q = _randn(Bn, Hq, hd, seed=6)
+    ctx_dev = [cap + 1000 * (b + 1) for b in range(Bn)]
+    ctx_dev[-1] = 0                                                       # an empty sequence
+    got = B.es_op_decode_attention(q.cuda(), kp.cuda(), vp.cuda(), perm.cuda(),
+                                   torch.tensor(ctx_dev, dtype=torch.int32).cuda(), cap)
+    for b in range(Bn - 1):
+        k = torch.cat([kp[int(perm[b, i])] for i in range(pps)], dim=1).transpose(0, 1)      # [cap, Hkv, hd]
+        v = torch.cat([vp[int(perm[b, i])] for i in range(pps)], dim=1).transpose(0, 1)
+        want = O.causal_attention_matrix(q[b:b + 1].double(), k.double(), v.double(), q_pos0=cap - 1)
+        assert rel_err(got[b], want.reshape(-1)) < 2e-3
+    assert torch.count_nonzero(got[Bn - 1]) == 0

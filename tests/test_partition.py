@@ -115,3 +115,15 @@ def test_planner_argument_errors(B):
     with pytest.raises(B.EsError) as e:
         B.es_partition_throughput([[1.0]], [1.0, 2.0], [1.0], [1.0], [[0.0]])
     assert e.value.status == 2
+
+
+def test_planners_refuse_tables_beyond_their_memory_cap_instead_of_throwing():
+    """20 devices and 82 layers would need a 20 GB table: the call must come back with a status, not die."""
+    import numpy as np
+    from paper_2405_14371_b200 import binding as B
+
+    N, M = 82, 20
+    t = np.ones((N, M)); O = np.ones(N); Req = np.ones(N); Mem = np.full(M, 1e9); Bw = np.ones((M, M))
+    with pytest.raises(B.EsError) as e:
+        B.es_partition_throughput(t, O, Req, Mem, Bw)
+    assert e.value.status == 9 and "4 GiB" in e.value.message

@@ -102,3 +102,62 @@ def test_schedules_agree_bit_for_bit(with_head):
                 assert (x is None) == (y is None)
                 if x is not None:
                     assert torch.equal(x, y), schedule
+
+
+@pytest.mark.gpu
+def test_schedules_at_the_13b_shapes_of_the_timed_pipeline():
+    """The configuration the benchmark times for the 13B pipeline — four shards, eight micro-batches of one
+    sequence, 256-token prompts, one stream per shard with event dependencies — at the 13B layer shapes with two
+    layers per shard: both pipelined schedules must reproduce the one-stream order bit for bit, and micro-batches
+    0 and 7 must match the oracle (greedy tokens fed back on the device, the oracle teacher-forced with them)."""
+    from paper_2405_14371_b200 import binding as B
+    from paper_2405_14371_b200.pipeline import ShardPipeline
+    from tests.helpers import oracle_streamed, rel_err, report_err, slice_weights
+    from workload import LLAMA2_13B, ModelShape, prompt_ids, shard_weights
+
+    full = LLAMA2_13B
+    m = ModelShape("llama2-13b-8layers", 8, full.d_model, full.n_heads, full.n_kv_heads, full.head_dim, full.d_ffn, full.vocab)
+    n_sh, per, MB, T, S = 4, 2, 8, 256, 6
+    wd = shard_weights(3, m, 0, m.n_layers, device="cuda")
+    ids = prompt_ids(3, MB, T, m.vocab).cuda().reshape(MB, 1, T)
+    kw = dict(max_slots=MB, max_seq=T + S, max_tokens=T, max_batch=1)
+
+    def run(schedule):
+        torch.cuda.synchronize()
+        first = torch.cuda.Stream()
+        streams = [first if schedule == "sequential" else torch.cuda.Stream() for _ in range(n_sh)]
+        shards = [B.Shard(m, i * per, (i + 1) * per, slice_weights(wd, m, i * per, (i + 1) * per), stream=streams[i], **kw)
+                  for i in range(n_sh)]
+        pipe = ShardPipeline(shards, [[mb] for mb in range(MB)], 1, schedule)
+        got = {}
+
+        def keep(p, out):
+            got[(p.iteration, p.micro_batch)] = [t.clone() for t in out]
+
+        pipe.prefill(ids, T, on_output=keep)
+        pipe.decode(S, on_output=keep)
+        pipe.join(torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        for sh in shards:
+            sh.es_shard_device_status()
+            sh.close()
+        return got
+
+    ref = run("sequential")
+    assert len(ref) == MB * (S + 1)
+    for schedule in ("bubbles", "no_bubbles"):
+        got = run(schedule)
+        assert got.keys() == ref.keys()
+        for key in ref:
+            for x, y in zip(ref[key], got[key]):
+                assert torch.equal(x, y), (schedule, key)
+    for mb in (0, MB - 1):
+        fed = torch.stack([ref[(it, mb)][2][0] for it in range(S)]).cpu()              # token produced by iteration it
+        seq = torch.cat([ids[mb, 0].cpu(), fed])
+        xs, ls = oracle_streamed(m, wd, 0, m.n_layers, [seq], logits_from=T - 1)
+        want_h, want_l = xs[0], ls[0]
+        assert report_err(f"13B pipeline shapes micro-batch {mb} prefill hidden", rel_err(ref[(0, mb)][0][0], want_h[:T])) < 1e-2
+        dec_h = torch.stack([ref[(it, mb)][0][0, 0] for it in range(1, S + 1)])
+        assert report_err(f"13B pipeline shapes micro-batch {mb} decode hidden", rel_err(dec_h, want_h[T:])) < 1e-2
+        logits = torch.stack([ref[(it, mb)][1][0] for it in range(S + 1)])
+        assert report_err(f"13B pipeline shapes micro-batch {mb} logits", rel_err(logits, want_l)) < 1e-2

@@ -56,3 +56,16 @@ def test_single_process_needs_no_group():
         os.environ.pop(k, None)
     assert replicas.max_over_ranks(3.5, 1) == 3.5
     assert replicas.job_throughput(10.0, 500.0, 1) == pytest.approx(20.0)
+
+
+def test_launch_plan_starts_ranks_only_when_asked_for_several_gpus_outside_a_job():
+    from paper_2405_14371_b200 import replicas
+
+    argv = ["bench.py", "--gpus", "4", "--steps", "2"]
+    assert replicas.launch_plan(1, {}, argv) is None                       # one GPU: this process
+    assert replicas.launch_plan(4, {"WORLD_SIZE": "4", "RANK": "1"}, argv) is None   # already a rank of a job
+    cmd = replicas.launch_plan(4, {}, argv)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=4" in cmd and "--standalone" in cmd
+    assert cmd[cmd.index("--local-addr") + 1] == "127.0.0.1"
+    assert cmd[-len(argv):] == argv                                        # same script, same arguments
+    assert replicas.launch_plan(0, {}, argv) is None

@@ -359,6 +359,50 @@ def test_pipeline_stage_drives_the_library_on_one_gpu(B, tiny):
                 assert gen[:, mb, b].tolist() == w_t.tolist()
 
 
+@pytest.mark.parametrize("Bn", [1, 8])
+def test_step_timing_from_inside_a_replayed_step(B, tiny, Bn):
+    """Time stamps written by the kernels of a decode step: every launch of the step is listed in launch order
+    with a start and an end inside the step, the step's results are the same bits with and without the stamps,
+    and the prefill pass is stamped too."""
+    wd, _ = tiny
+    T = 12
+    ids = prompt_ids(0, Bn, T, TINY.vocab, seed=3).cuda()
+    stream = torch.cuda.Stream()
+    outs = {}
+    with torch.cuda.stream(stream):
+        for timing in (False, True):
+            sh = B.Shard(TINY, 0, 2, wd, max_slots=Bn, max_seq=T + 6, max_tokens=Bn * T, stream=stream)
+            sh.es_shard_set_step_timing(timing)
+            sh.es_shard_prefill(ids, None, Bn, T, list(range(Bn)))
+            if timing:
+                pre = sh.es_shard_step_timing()
+                assert {"embed", "qkv", "attention", "o", "gate_up", "down", "lm_head", "argmax", "set_ctx"} <= {e["category"] for e in pre}
+            n = sh.es_shard_handoff()[2]
+            rows = []
+            for _ in range(4):
+                sh.es_shard_decode_step(n, None, Bn, list(range(Bn)))
+                h, l, n = sh.es_shard_handoff()
+                rows.append((h.clone(), l.clone(), n.clone()))
+            if timing:
+                st = sh.es_shard_step_timing()
+                assert len(st) >= 2 * 5 + 4                      # 5 kernels per layer, embedding, head, argmax, counter
+                assert st[0]["category"] == "embed" and st[1]["category"] in ("rmsnorm", "qkv")
+                assert st[-1]["category"] == "set_ctx"
+                assert min(e["start_us"] for e in st) == 0.0
+                for e in st:
+                    assert 0.0 <= e["start_us"] <= e["end_us"] < 1e5, e
+                ends = [e["end_us"] for e in st]
+                # a kernel cannot finish before the one it depends on has finished
+                assert all(b >= a for a, b in zip(ends, ends[1:])), ends
+            sh.es_shard_device_status()
+            sh.close()
+            outs[timing] = rows
+    stream.synchronize()
+    for a, b in zip(outs[False], outs[True]):
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+
+
 def test_profile_feeds_the_partition_planners(B, tiny):
     """The per-layer profile is the planners' input: measured times for this GPU plus two synthetic slower
     devices (scaled times), activation and memory sizes from the profile."""

@@ -49,9 +49,40 @@ def test_static_scratch_matches_caller_scratch_on_consecutive_calls():
 def test_static_scratch_rejects_oversized_calls():
     from paper_2405_14371_b200 import binding as B
     q, k, v, table, ctx, max_ctx = _case(1, 8, 8, 128, 16, [16], seed=4)
-    # 64 sequences x 64 heads over a 6400-token context cut into 10 splits would need 21 MB of partials
-    Bn, Hq, Hkv, hd, P, pps = 64, 64, 1, 128, 16, 400
+    # 256 sequences x 64 heads need 8.5 MB of partials even with a single split
+    Bn, Hq, Hkv, hd, P, pps = 256, 64, 8, 128, 16, 4
     with pytest.raises(B.EsError) as e:
         B._check(B.lib.es_op_decode_attention_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), table.data_ptr(),
                                                      ctx.data_ptr(), q.data_ptr(), Bn, Hq, Hkv, hd, P, pps, P * pps, None))
     assert e.value.status == 6 and "8388608" in e.value.message
+    # a shape the kernels do not take is reported as such, before any capacity arithmetic
+    for bad in ((1, 8, 8, 96), (1, 8, 3, 128), (1, 64, 1, 128)):
+        with pytest.raises(B.EsError) as e:
+            B._check(B.lib.es_op_decode_attention_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), table.data_ptr(),
+                                                         ctx.data_ptr(), q.data_ptr(), bad[0], bad[1], bad[2], bad[3], 16, 1, 16, None))
+        assert e.value.status == 2, bad
+
+
+def test_static_scratch_takes_nothing_from_the_device_on_any_stream():
+    """After a first call (which looks up the array's address), further calls must leave the driver's count of
+    free device memory exactly where it was — a cudaMalloc inside the library would not show in torch's own
+    allocator statistics — on the default stream and on a stream of the caller's."""
+    from paper_2405_14371_b200 import binding as B
+    q, k, v, table, ctx, max_ctx = _case(4, 32, 8, 128, 64, [700, 513, 64, 1], seed=5)
+    want = B.es_op_decode_attention(q, k, v, table, ctx, max_ctx)
+    out = torch.empty_like(want)
+    side = torch.cuda.Stream()
+    B.es_op_decode_attention_static(q, k, v, table, ctx, max_ctx, out=out)          # warm-up: address look-up
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    n_before = torch.cuda.memory_stats().get("allocation.all.allocated", 0)
+    for i in range(6):
+        st = side if i % 2 else None
+        out.zero_()
+        if st is not None:
+            st.wait_stream(torch.cuda.current_stream())
+        got = B.es_op_decode_attention_static(q, k, v, table, ctx, max_ctx, out=out, stream=st)
+        torch.cuda.synchronize()                     # the calls share one array: never two in flight
+        assert torch.equal(got, want)
+    assert torch.cuda.mem_get_info()[0] == free_before
+    assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == n_before
