@@ -91,6 +91,59 @@ def test_split_point_equals_single_shard(B, tiny, k):
         s_.close()
 
 
+@pytest.mark.parametrize("d,Hq,Hkv,F,Bn", [(512, 8, 4, 1536, 5), (512, 8, 4, 1536, 12), (4096, 32, 32, 11008, 8), (4096, 32, 32, 11008, 16),
+                                            (8192, 64, 8, 4096, 16)])
+def test_decode_of_several_sequences_with_fused_norm_and_sliced_products(B, d, Hq, Hkv, F, Bn):
+    """Decode steps of 3..16 sequences on layer shapes where the tensor-core streaming kernels take every product:
+    the RMSNorm runs inside the QKV and gate / up kernels from sums of squares written by the O and down
+    epilogues, and products whose activations do not fit in shared memory are cut along K across CTAs and
+    finished by the last warp to deliver a unit.  Checked against the oracle at every step, for the split
+    [0,1) -> [1,3) == [0,3) bit for bit (a shard that receives its rows from another shard computes the sums of
+    squares with its own kernel), and for repeatability (the finishing order is fixed)."""
+    from workload import ModelShape, shard_weights
+    hd = 64 if d == 512 else 128
+    m = ModelShape("mid", 3, d, Hq, Hkv, hd, F, 512)
+    wd = shard_weights(11, m, 0, 3, device="cuda")
+    wh = {k: v.cpu() for k, v in wd.items() if k != "layers"}
+    wh["layers"] = [{k: v.cpu() for k, v in lw.items()} for lw in wd["layers"]]
+    T, S = 5, 4
+    ids = prompt_ids(11, Bn, T, m.vocab)
+    nxt = forced_decode_ids(11, Bn, S, m.vocab)
+    slots = list(range(Bn))
+    kw = dict(max_slots=Bn, max_seq=T + S, max_tokens=Bn * T)
+    full = B.Shard(m, 0, 3, wd, **kw)
+    a = B.Shard(m, 0, 1, slice_weights(wd, m, 0, 1), **kw)
+    b = B.Shard(m, 1, 3, slice_weights(wd, m, 1, 3), **kw)
+    runs = []
+    for rep in range(2):
+        full.es_shard_reset_slots(None)
+        full.es_shard_prefill(ids.cuda(), None, Bn, T, slots)
+        hs, ls = [], []
+        for s in range(S):
+            full.es_shard_decode_step(nxt[s].cuda(), None, Bn, slots)
+            h, l, _ = full.es_shard_handoff()
+            hs.append(h[:, 0].clone()); ls.append(l.clone())
+        runs.append((torch.stack(hs), torch.stack(ls)))
+    assert torch.equal(runs[0][0], runs[1][0]) and torch.equal(runs[0][1], runs[1][1])
+    a.es_shard_prefill(ids.cuda(), None, Bn, T, slots)
+    b.es_shard_prefill(None, a.es_shard_handoff()[0], Bn, T, slots)
+    for s in range(S):
+        a.es_shard_decode_step(nxt[s].cuda(), None, Bn, slots)
+        b.es_shard_decode_step(None, a.es_shard_handoff()[0], Bn, slots)
+        hb, lb, _ = b.es_shard_handoff()
+        assert torch.equal(hb[:, 0], runs[0][0][s]) and torch.equal(lb, runs[0][1][s]), s
+    for r in (0, Bn - 1):
+        seq = torch.cat([ids[r], nxt[:, r]])
+        want_h, _ = O.shard_forward_full(m, wh, 0, 3, ids=seq)
+        assert rel_err(runs[0][0][:, r], want_h[T:]) < TOL
+        for s in (0, S - 1):
+            _, want_l = O.shard_forward_full(m, wh, 0, 3, ids=seq[:T + s + 1])
+            assert rel_err(runs[0][1][s, r], want_l) < TOL
+    for sh in (full, a, b):
+        sh.es_shard_device_status()
+        sh.close()
+
+
 def test_batch_rows_independent_and_match_oracle(B, tiny):
     wd, wh = tiny
     T, S, Bn = 9, 4, 3
