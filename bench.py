@@ -163,6 +163,10 @@ def run_ours(args, name: str, steps: int, warmup: int, dist_ctx, with_clocks: bo
     wl = WORKLOADS[name]
     if args.layers:
         wl = dataclasses.replace(wl, layer_end=min(wl.layer_end, wl.layer_begin + args.layers * wl.n_shards))
+    if args.model_layers:
+        # a shallow model of the same layer shapes, so that a small capture case still ends with the output layer
+        wl = dataclasses.replace(wl, model=dataclasses.replace(wl.model, n_layers=args.model_layers), layer_begin=0,
+                                 layer_end=args.model_layers)
     m = wl.model
     Bn, T, S = (args.batch or wl.batch), (args.prompt_len or wl.prompt_len), (args.decode_steps or wl.decode_steps)
     if (Bn, T, S) != (wl.batch, wl.prompt_len, wl.decode_steps):
@@ -526,9 +530,11 @@ def main():
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length (profile runs only)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profile runs only)")
     ap.add_argument("--layers", type=int, default=0, help="keep only the first LAYERS layers of every shard (profile runs only)")
+    ap.add_argument("--model-layers", type=int, default=0,
+                    help="run a model of only this many layers of the workload's shapes, output layer included (profile runs only)")
     args = ap.parse_args()
-    if (args.prompt_len or args.batch or args.layers) and not args.profile:
-        ap.error("--prompt-len / --batch / --layers change the workload and are only accepted together with --profile")
+    if (args.prompt_len or args.batch or args.layers or args.model_layers) and not args.profile:
+        ap.error("--prompt-len / --batch / --layers / --model-layers change the workload and are only accepted together with --profile")
 
     from paper_2405_14371_b200 import replicas
     relaunch = replicas.launch_plan(args.gpus, os.environ, sys.argv)

@@ -183,6 +183,13 @@ ES_API es_status_t es_shard_set_graphs(es_shard_t *shard, int32_t enabled);
  * inside a kernel ran out since the last call. */
 ES_API es_status_t es_shard_device_status(es_shard_t *shard);
 
+/* Exercises the time-out path above without any kernel misbehaving: enqueues a one-CTA kernel built like the
+ * tensor-core kernels (barrier, TMEM allocation, bounded wait, common teardown) whose barrier is never arrived
+ * on.  Its wait gives up after limit_us microseconds (1 .. 100000), records its code in the status word, frees
+ * its TMEM and returns; the next es_shard_device_status reports ES_ERR_DEVICE_TIMEOUT and clears the word, and
+ * the shard stays usable.  For tests of a caller's error handling; the paper has no counterpart. */
+ES_API es_status_t es_shard_wait_probe(es_shard_t *shard, int32_t limit_us);
+
 /* Launch-by-launch timing of the linear-layer kernels (the weight-streaming and tensor-core
  * products that dominate a pass): while on, every such launch is bracketed by a CUDA event pair on
  * the shard's stream (every launch of a pass, by category) and decode steps are not replayed as graphs.  Switching it on or off clears
@@ -283,7 +290,11 @@ ES_API es_status_t es_op_linear(const void *A, const void *W, const float *R, fl
  * With 3 <= M <= 16 (a decode step of several sequences) the weight-streaming kernel is used instead:
  * every CTA keeps one K slice of the activations in shared memory and streams 16-row groups of W over
  * it; K must be a multiple of 256 and K / 32 divisible by k_splits, a slice of 8 (M <= 8) or 16 rows
- * must fit 100 KB.  M <= 2 is ES_ERR_UNSUPPORTED (such products never need slicing). */
+ * must fit 100 KB.  No second kernel runs in this form: the partial sums of a 16-column group go to the
+ * workspace, and the warp whose partial arrives last (one arrival counter per group, kept at the end of
+ * the workspace and cleared by this call) adds the slices in ascending order and the residual.  The
+ * workspace layout is private; size it with es_op_linear_splitk_workspace_bytes.
+ * M <= 2 is ES_ERR_UNSUPPORTED (such products never need slicing). */
 ES_API size_t es_op_linear_splitk_workspace_bytes(int32_t M, int32_t N, int32_t k_splits);
 ES_API es_status_t es_op_linear_splitk(const void *A, const void *W, const float *R, float *C, int32_t M, int32_t N,
                                        int32_t K, int32_t k_splits, void *workspace, size_t workspace_bytes,

@@ -80,6 +80,7 @@ def _load() -> C.CDLL:
         "es_shard_set_graphs": (i32, [vp, i32]),
         "es_shard_device_status": (i32, [vp]),
         "es_shard_launch_count": (C.c_int64, [vp]),
+        "es_shard_wait_probe": (i32, [vp, i32]),
         "es_shard_set_kernel_timing": (i32, [vp, i32]),
         "es_shard_kernel_timing": (i32, [vp, P(C.c_double), P(C.c_double), P(C.c_int64)]),
         "es_shard_kernel_timing_detail": (i32, [vp, P(C.c_double), P(C.c_double), P(C.c_int64)]),
@@ -110,7 +111,7 @@ def _load() -> C.CDLL:
 lib = _load()
 EXPORTS = ("es_shard_workspace_bytes es_shard_create es_shard_prefill es_shard_prefill_ragged es_shard_decode_step es_shard_handoff "
            "es_layer_profile es_shard_set_profiling es_shard_reset_slots es_shard_set_page_table es_shard_set_graphs "
-           "es_partition_latency es_partition_throughput es_shard_device_status es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_kernel_timing_detail es_shard_set_step_timing es_shard_step_timing es_shard_destroy es_last_error es_version es_op_rmsnorm "
+           "es_partition_latency es_partition_throughput es_shard_device_status es_shard_wait_probe es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_kernel_timing_detail es_shard_set_step_timing es_shard_step_timing es_shard_destroy es_last_error es_version es_op_rmsnorm "
            "es_op_linear es_op_linear_splitk_workspace_bytes es_op_linear_splitk es_op_prefill_attention es_op_decode_attention_scratch_bytes es_op_decode_attention "
            "es_op_decode_attention_static_capacity es_op_decode_attention_static").split()
 
@@ -257,6 +258,9 @@ class Shard:
 
     def es_shard_device_status(self) -> None:
         _check(lib.es_shard_device_status(self._handle))
+
+    def es_shard_wait_probe(self, limit_us: int) -> None:
+        _check(lib.es_shard_wait_probe(self._handle, int(limit_us)))
 
     def es_shard_launch_count(self) -> int:
         return int(lib.es_shard_launch_count(self._handle))

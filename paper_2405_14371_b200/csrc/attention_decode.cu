@@ -8,9 +8,10 @@
 //   * values: the head dimension is spread over the lanes (coalesced V rows), the 32
 //     probabilities are broadcast lane by lane with shuffles.
 // The warps of a CTA are merged through shared memory in warp order.  With a single split the
-// CTA writes the final output; otherwise it writes an unnormalised partial (o, max, sum) and a
-// second kernel merges the partials of a row in split order, so results never depend on
-// scheduling.
+// CTA writes the final output; otherwise it writes an unnormalised partial (o, max, sum) and bumps an
+// arrival counter of its (sequence, KV head): the CTA that arrives last merges the partials of the
+// group's rows in split order (no second launch, nobody waits, and the order of the merge is fixed,
+// so results never depend on scheduling).
 #include "es_internal.cuh"
 #include "launch.cuh"
 
@@ -32,6 +33,7 @@ __global__ void __launch_bounds__(DWARPS * 32, PRE ? 1 : 2) decode_attn_split_ke
   __shared__ float sm_o[DWARPS][G][HD];
   __shared__ float sm_m[DWARPS][G];
   __shared__ float sm_l[DWARPS][G];
+  __shared__ int s_last;
 
   const int split = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -48,8 +50,8 @@ __global__ void __launch_bounds__(DWARPS * 32, PRE ? 1 : 2) decode_attn_split_ke
   const int t_begin = split * tokens_per_split;
   if (t_begin >= ctx) {
     pdl_wait();
-    // an empty context with a single split has no merge kernel behind it: the output rows are zeros
-    if (p.n_splits == 1)
+    // an empty context: nobody will arrive to merge, the CTA of split 0 writes the zero rows
+    if (split == 0 && ctx <= 0)
       for (int i = threadIdx.x; i < G * HD; i += DWARPS * 32)
         p.out[((int64_t)b * p.Hq + (g * G + i / HD)) * HD + (i % HD)] = __float2half_rn(0.f);
     stamp_end(p.stamp);
@@ -209,29 +211,7 @@ __global__ void __launch_bounds__(DWARPS * 32, PRE ? 1 : 2) decode_attn_split_ke
       if (c == 0) { dst[HD] = mm; dst[HD + 1] = ll; }
     }
   }
-  stamp_end(p.stamp);
-}
-
-template <int HD>
-__global__ void __launch_bounds__(HD) decode_attn_merge_kernel(const DecodeAttnParams p) {
-  pdl_launch_dependents();
-  const int h = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
-  pdl_wait();
-  const int slot = p.kv.slots ? p.kv.slots[b] : b;
-  const int ctx = min(p.ctx_len[slot] + p.ctx_add, p.kv.pages_per_slot * p.kv.P);
-  const int tokens_per_split = p.pages_per_split * p.kv.P;
-  int active = (ctx + tokens_per_split - 1) / tokens_per_split;
-  active = active < p.n_splits ? active : p.n_splits;
-  const float* src = p.part + ((int64_t)b * p.Hq + h) * p.n_splits * (HD + 2);
-  float mm = -INFINITY;
-  for (int s = 0; s < active; ++s) mm = fmaxf(mm, src[(int64_t)s * (HD + 2) + HD]);
-  float o = 0.f, ll = 0.f;
-  for (int s = 0; s < active; ++s) {
-    const float f = __expf(src[(int64_t)s * (HD + 2) + HD] - mm);
-    o += src[(int64_t)s * (HD + 2) + c] * f;
-    ll += src[(int64_t)s * (HD + 2) + HD + 1] * f;
-  }
-  p.out[((int64_t)b * p.Hq + h) * HD + c] = __float2half_rn(active > 0 ? o / ll : 0.f);
+  if (p.n_splits > 1) merge_splits_if_last<HD, G>(p, b, g, ctx, &s_last);
   stamp_end(p.stamp);
 }
 
@@ -253,10 +233,6 @@ es_status_t launch_hd(const DecodeAttnParams& p, cudaStream_t s, bool pdl, int64
   if (many && tunables().attn_mma != 0 && decode_attention_mma_supported(p)) {
     ES_TRY(launch_decode_attention_mma(p, s, pdl));
     if (launches) ++*launches;
-    if (p.n_splits > 1) {
-      ES_CUDA_CHECK(launch_kernel(decode_attn_merge_kernel<HD>, dim3(p.Hq, p.B), dim3(HD), 0, s, pdl, p));
-      if (launches) ++*launches;
-    }
     return ES_OK;
   }
   switch (p.Hq / p.Hkv) {
@@ -268,17 +244,17 @@ es_status_t launch_hd(const DecodeAttnParams& p, cudaStream_t s, bool pdl, int64
   }
   ES_TRY(st);
   if (launches) ++*launches;
-  if (p.n_splits > 1) {
-    ES_CUDA_CHECK(launch_kernel(decode_attn_merge_kernel<HD>, dim3(p.Hq, p.B), dim3(HD), 0, s, pdl, p));
-    if (launches) ++*launches;
-  }
   return ES_OK;
 }
 
 }  // namespace
 
+size_t decode_attention_counter_offset(int B, int Hq, int hd, int n_splits) {
+  return ((size_t)B * Hq * n_splits * (hd + 2) * sizeof(float) + 255) / 256 * 256;
+}
+size_t decode_attention_counter_bytes(int B, int Hq) { return ((size_t)B * Hq * sizeof(int) + 255) / 256 * 256; }
 size_t decode_attention_scratch_bytes(int B, int Hq, int hd, int n_splits) {
-  return (size_t)B * Hq * n_splits * (hd + 2) * sizeof(float);
+  return decode_attention_counter_offset(B, Hq, hd, n_splits) + decode_attention_counter_bytes(B, Hq);
 }
 
 es_status_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t s, int64_t* launches, bool pdl) {

@@ -25,8 +25,9 @@
 // measured faster (config 4 shape 30.5 against 33.7 us; 8 sequences x 32 heads x 680 keys 27.1 -> 25.0 us
 // with two).  The four
 // warps of a CTA are merged through shared memory in warp order and the result is written as the
-// final row (one split) or as an unnormalised partial (o, max, sum) for the merge kernel, exactly
-// like the CUDA-core kernel, so results do not depend on scheduling.
+// final row (one split) or as an unnormalised partial (o, max, sum) that the last CTA to arrive for the
+// (sequence, KV head) merges in split order, exactly like the CUDA-core kernel, so results do not depend
+// on scheduling.
 #include "es_internal.cuh"
 #include "launch.cuh"
 
@@ -70,6 +71,7 @@ __global__ void __launch_bounds__(MW * 32, DB ? 2 : 3) decode_attn_mma_kernel(co
   __shared__ float sm_o[MW][G][HD];
   __shared__ float sm_m[MW][G];
   __shared__ float sm_l[MW][G];
+  __shared__ int s_last;
 
   const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -83,8 +85,8 @@ __global__ void __launch_bounds__(MW * 32, DB ? 2 : 3) decode_attn_mma_kernel(co
   const int t_begin = split * tokens_per_split;
   if (t_begin >= ctx) {
     pdl_wait();
-    // an empty context with a single split has no merge kernel behind it: the output rows are zeros
-    if (p.n_splits == 1)
+    // an empty context: nobody will arrive to merge, the CTA of split 0 writes the zero rows
+    if (split == 0 && ctx <= 0)
       for (int i = threadIdx.x; i < G * HD; i += MW * 32)
         p.out[((int64_t)b * p.Hq + ((int64_t)kvh * G + i / HD)) * HD + (i % HD)] = __float2half_rn(0.f);
     stamp_end(p.stamp);
@@ -235,6 +237,7 @@ __global__ void __launch_bounds__(MW * 32, DB ? 2 : 3) decode_attn_mma_kernel(co
       if (c == 0) { dst[HD] = mm; dst[HD + 1] = ll; }
     }
   }
+  if (p.n_splits > 1) merge_splits_if_last<HD, G>(p, b, kvh, ctx, &s_last);
   stamp_end(p.stamp);
 }
 
@@ -256,7 +259,7 @@ bool decode_attention_mma_supported(const DecodeAttnParams& p) {
   return true;
 }
 
-// The split kernel only; the caller launches the merge kernel when there is more than one split.
+// Like the CUDA-core kernel, the kernel merges its own splits (the last CTA to arrive for a (sequence, KV head)).
 es_status_t launch_decode_attention_mma(const DecodeAttnParams& p, cudaStream_t s, bool pdl) {
   if (!decode_attention_mma_supported(p)) return fail(ES_ERR_UNSUPPORTED, "tensor-core decode attention does not take this layout");
   switch (p.Hq / p.Hkv) {

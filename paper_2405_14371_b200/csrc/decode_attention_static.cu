@@ -70,8 +70,12 @@ es_status_t es_op_decode_attention_static(const void* q, const void* k_pages, co
                 "use es_op_decode_attention with a caller buffer", need, STATIC_SCRATCH_BYTES);
   void* scratch = nullptr;
   ES_TRY(scratch_address(&scratch, (cudaStream_t)stream));
-  // Nothing has to be cleared: every split that the merge step reads is written earlier in this same call.
+  // The partials need no clearing (every split that the merge reads is written earlier in this same call); the
+  // arrival counters that follow them must start at zero.  A fill is not an allocation.
   p.part = (float*)scratch;
+  if (p.n_splits > 1)
+    ES_CUDA_CHECK(cudaMemsetAsync((unsigned char*)scratch + decode_attention_counter_offset(B, Hq, hd, p.n_splits), 0,
+                                  decode_attention_counter_bytes(B, Hq), (cudaStream_t)stream));
   return launch_decode_attention(p, (cudaStream_t)stream, nullptr);
 }
 

@@ -36,6 +36,8 @@ struct Tunables {
   int pdl;           // ES_PDL: programmatic dependent launch in decode steps (1, default) or plain stream order (0)
   int attn_mma;      // ES_ATTN_MMA: tensor-core decode attention for launches with many items (1, default) or never (0)
   int split_k;       // ES_SPLIT_K: split-K for the O and down projections of short prefills (1, default) or never (0)
+  int decode_fused_norm;   // ES_DECODE_FUSED_NORM: decode steps of 3..16 rows normalise inside the QKV / gate-up kernels (1) or with a launch of their own (0)
+  int ks_min_slice;        // ES_KS_MIN_SLICE: smallest K slice of the K-sliced streaming kernel (elements)
 };
 const Tunables& tunables();
 
@@ -159,6 +161,10 @@ es_status_t launch_set_ctx(int* ctx_len, const int* slots, int B, int value, int
                            int64_t* launches, bool pdl = false, const int* values = nullptr,
                            unsigned long long* stamp = nullptr);
 
+// A one-CTA kernel whose only barrier is never arrived on: its bounded wait runs out after limit_ns and writes
+// its code to `status` (two ints), then the CTA leaves through the usual teardown.  Test support.
+es_status_t launch_wait_probe(int* status, unsigned long long limit_ns, cudaStream_t s, int64_t* launches);
+
 // ---- attention -------------------------------------------------------------------------------
 // K/V addressing shared by both attention kernels: token t of sequence b, kv head g lives at
 //   base + page * page_stride + g * head_stride + (t % P) * tok_stride,
@@ -202,12 +208,51 @@ struct DecodeAttnParams {
   KvView kv;
   const int* ctx_len;     // indexed by slot (or by b when kv.slots == nullptr)
   int ctx_add;            // keys visible = ctx_len[.] + ctx_add
-  float* part;            // scratch [B, Hq, n_splits, hd + 2]
+  float* part;            // scratch [B, Hq, n_splits, hd + 2], then (256-byte aligned) one arrival counter per
+                          // (sequence, KV head), zero before the launch and zero again after it
   int B, Hq, Hkv, hd;
   int n_splits, pages_per_split;
   unsigned long long* stamp;   // optional time stamps of the launch (split and merge kernels share them), nullptr = none
 };
 size_t decode_attention_scratch_bytes(int B, int Hq, int hd, int n_splits);
+// byte offset of the arrival counters inside the scratch, and their size
+size_t decode_attention_counter_offset(int B, int Hq, int hd, int n_splits);
+size_t decode_attention_counter_bytes(int B, int Hq);
+
+// The end of both split kernels when the context was cut into several splits: the CTA has written its
+// unnormalised partial (o, max, sum) of the G heads of (sequence b, KV head kvh); the CTA that arrives last
+// (a counter per (b, kvh); CTAs of splits beyond the context never arrive) merges the splits in ascending order,
+// writes the final rows and puts the counter back to zero.  Nobody waits.  All threads of the CTA call.
+template <int HD, int G>
+__device__ __forceinline__ void merge_splits_if_last(const DecodeAttnParams& p, int b, int kvh, int ctx, int* s_flag) {
+  int* cnt = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(p.part) +
+                                    (((size_t)p.B * p.Hq * p.n_splits * (HD + 2) * sizeof(float) + 255) / 256) * 256) +
+             (b * p.Hkv + kvh);
+  const int tokens_per_split = p.pages_per_split * p.kv.P;
+  int active = (ctx + tokens_per_split - 1) / tokens_per_split;
+  active = active < p.n_splits ? active : p.n_splits;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) *s_flag = (atomicAdd(cnt, 1) == active - 1) ? 1 : 0;
+  __syncthreads();
+  if (*s_flag == 0) return;
+  __threadfence();
+  for (int i = threadIdx.x; i < G * HD; i += blockDim.x) {
+    const int j = i / HD, c = i - j * HD;
+    const int64_t row = (int64_t)b * p.Hq + ((int64_t)kvh * G + j);
+    const float* src = p.part + row * p.n_splits * (HD + 2);
+    float mm = -INFINITY;
+    for (int s = 0; s < active; ++s) mm = fmaxf(mm, __ldcg(src + (int64_t)s * (HD + 2) + HD));
+    float o = 0.f, ll = 0.f;
+    for (int s = 0; s < active; ++s) {
+      const float f = __expf(__ldcg(src + (int64_t)s * (HD + 2) + HD) - mm);
+      o += __ldcg(src + (int64_t)s * (HD + 2) + c) * f;
+      ll += __ldcg(src + (int64_t)s * (HD + 2) + HD + 1) * f;
+    }
+    p.out[row * HD + c] = __float2half_rn(o / ll);
+  }
+  if (threadIdx.x == 0) *cnt = 0;
+}
 void choose_splits(int max_ctx, int P, int B, int Hkv, int group, int* n_splits, int* pages_per_split);
 es_status_t launch_decode_attention(const DecodeAttnParams& p, cudaStream_t s, int64_t* launches, bool pdl = false);
 // tensor-core (mma.sync) split kernel for head_dim 128; same partial layout, merged by the same merge kernel

@@ -600,7 +600,7 @@ int linear_stream_mma_splits(const LinearParams& p, int epi, size_t workspace_by
   for (int ks = 2; ks <= 64 && ks <= KS_GRID; ++ks) {
     if (steps % ks) continue;
     const int kslice = p.K / ks;
-    if (kslice < 512) break;
+    if (kslice < tunables().ks_min_slice) break;
     if ((size_t)nt * 8 * (kslice + 8) * sizeof(__half) > KS_SMEM_MAX) continue;
     if (linear_stream_mma_workspace_bytes(p.M, p.N, epi, ks) > workspace_bytes) continue;
     const int ncol = KS_GRID / ks;

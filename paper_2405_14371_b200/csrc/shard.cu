@@ -41,7 +41,7 @@ static int env_int(const char* name, int dflt) {
 }
 
 const Tunables& tunables() {
-  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_TC_PAIR_WIDE", 1), env_int("ES_SPLIT_PAIRS", 1), env_int("ES_PDL", 1), env_int("ES_ATTN_MMA", 1), env_int("ES_SPLIT_K", 1)};
+  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_TC_PAIR_WIDE", 1), env_int("ES_SPLIT_PAIRS", 1), env_int("ES_PDL", 1), env_int("ES_ATTN_MMA", 1), env_int("ES_SPLIT_K", 1), env_int("ES_DECODE_FUSED_NORM", 1), env_int("ES_KS_MIN_SLICE", 512)};
   return t;
 }
 
@@ -433,7 +433,7 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   // they stage their activations, from sums of squares that the O and down epilogues write (all layers have the
   // same shapes, so one check serves the pass).
   bool cn = false;
-  if (M > 2 && M <= 16 && !fuse_norm && s->splitk != nullptr && d.d_model % 16 == 0 && s->nl > 0) {
+  if (M > 2 && M <= 16 && !fuse_norm && s->splitk != nullptr && d.d_model % 16 == 0 && s->nl > 0 && tunables().decode_fused_norm != 0) {
     cn = true;
     for (int kind = 0; kind < 4 && cn; ++kind) {
       int epi = 0;
@@ -727,6 +727,8 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
     if (e == cudaSuccess) e = cudaMemsetAsync(s->ctx_len, 0, (size_t)desc->max_slots * 4, s->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->status, 0, 256, s->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->unit_cnt, 0, L.unit_cnt_bytes, s->stream);
+    if (e == cudaSuccess)       // arrival counters of the decode-attention splits (they follow the partials)
+      e = cudaMemsetAsync(s->part, 0, decode_attention_scratch_bytes((int)desc->max_batch, desc->n_heads, desc->head_dim, L.n_splits), s->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->kv, 0, L.kv_bytes, s->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s->stream);
     if (e != cudaSuccess) return bail(fail(ES_ERR_CUDA, "shard initialisation failed: %s", cudaGetErrorString(e)));
@@ -986,6 +988,12 @@ es_status_t es_shard_device_status(es_shard_t* s) {
   return ES_OK;
 }
 
+es_status_t es_shard_wait_probe(es_shard_t* s, int32_t limit_us) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  if (limit_us < 1 || limit_us > 100000) return fail(ES_ERR_RANGE, "limit_us must be in [1, 100000]");
+  return launch_wait_probe(s->status, (unsigned long long)limit_us * 1000ull, s->stream, &s->launches);
+}
+
 int64_t es_shard_launch_count(const es_shard_t* s) { return s ? s->launches : 0; }
 
 es_status_t es_shard_set_kernel_timing(es_shard_t* s, int32_t enabled) {
@@ -1202,6 +1210,9 @@ es_status_t es_op_decode_attention(const void* q, const void* k_pages, const voi
   if (scratch_bytes < decode_attention_scratch_bytes(B, Hq, hd, p.n_splits))
     return fail(ES_ERR_WORKSPACE, "scratch: %zu bytes given, %zu needed", scratch_bytes,
                 decode_attention_scratch_bytes(B, Hq, hd, p.n_splits));
+  if (p.n_splits > 1)         // the splits' arrival counters start at zero
+    ES_CUDA_CHECK(cudaMemsetAsync((unsigned char*)scratch + decode_attention_counter_offset(B, Hq, hd, p.n_splits), 0,
+                                  decode_attention_counter_bytes(B, Hq), (cudaStream_t)stream));
   return launch_decode_attention(p, (cudaStream_t)stream, nullptr);
 }
 

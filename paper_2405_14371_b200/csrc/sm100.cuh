@@ -33,9 +33,10 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 
-// Bounded wait: false if the CTA is aborting or the barrier did not flip within ~1 s.
+// Bounded wait: false if the CTA is aborting or the barrier did not flip within limit_ns (one second unless the
+// caller says otherwise).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code) {
+                                          int code, uint64_t limit_ns = 1000000000ull) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
@@ -43,7 +44,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 63u) == 0) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > 1000000000ull) {
+      if (global_timer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         if (status) { atomicCAS(status, 0, code); status[1] = (int)blockIdx.x; }
         return false;

@@ -246,12 +246,16 @@ def test_cfg4_gqa_shard_batch16(B):
         at_golden = got.abs().gather(1, where[:, None])[:, 0]
         assert float(((gmax.values - at_golden) / scale).max()) < TOL
 
-    # full depth, every column, on a prefix of the prompt against a live oracle run
+    # full depth, every column, on a prefix of the prompt against a live oracle run.  The stated metric divides by
+    # the largest magnitude of the compared handoff tensor (the sequence's whole prefill activation, known from the
+    # digest); the same error over the largest magnitude of the 96-position slice alone is reported beside it.
     P = 96
     xs, _ = oracle_streamed(m, wd, 0, wl.layer_end, [ids[r, :P].cpu() for r in (0, Bn - 1)])
-    for x, r in zip(xs, (0, Bn - 1)):
-        assert report_err(f"cfg4 layers 0-39 row {r} first {P} positions, all columns",
-                          rel_err(pre_full[r][:P], x)) < TOL
+    for i, (x, r) in enumerate(zip(xs, (0, Bn - 1))):
+        err = float((pre_full[r][:P].double().cpu() - x.double()).abs().max())
+        whole = float(torch.from_numpy(g["max_abs"][i])[:T].max())
+        report_err(f"cfg4 layers 0-39 row {r} first {P} positions, all columns, over the slice's own max", err / float(x.abs().max()))
+        assert report_err(f"cfg4 layers 0-39 row {r} first {P} positions, all columns", err / whole) < TOL
 
 
 @pytest.mark.parametrize("name,layers,Bn,T", [("cfg2_b1", 2, 2, 512), ("cfg4", 1, 2, 1024)])

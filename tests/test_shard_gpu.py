@@ -483,6 +483,35 @@ def test_profile_feeds_the_partition_planners(B, tiny):
     assert a2[0] == 0 and t2 <= max(sum(r) for r in zip(*t_comp))
 
 
+def test_a_device_wait_that_runs_out_is_reported_and_the_shard_stays_usable(B, tiny):
+    """The bounded waits of the tensor-core kernels end with a code in the shard's status word instead of
+    hanging.  A probe kernel with the same structure waits 2 ms on a barrier nobody arrives on: the status call
+    must report ES_ERR_DEVICE_TIMEOUT with the probe's code, clear the word, and the shard must go on computing
+    the same bits as before."""
+    import time
+    wd, _ = tiny
+    ids = prompt_ids(0, 1, 16, TINY.vocab, seed=1).cuda()
+    sh = B.Shard(TINY, 0, 2, wd, max_slots=1, max_seq=32, max_tokens=16)
+    sh.es_shard_prefill(ids, None, 1, 16, [0])
+    before = [t.clone() for t in sh.es_shard_handoff()]
+    sh.es_shard_device_status()                          # clean so far
+    t0 = time.perf_counter()
+    sh.es_shard_wait_probe(2000)
+    with pytest.raises(B.EsError) as e:
+        sh.es_shard_device_status()
+    assert time.perf_counter() - t0 < 5.0                # the wait ended by itself
+    assert e.value.status == 8 and "code 90" in e.value.message
+    sh.es_shard_device_status()                          # the word was cleared
+    sh.es_shard_reset_slots(None)
+    sh.es_shard_prefill(ids, None, 1, 16, [0])
+    after = sh.es_shard_handoff()
+    for x, y in zip(before, after):
+        assert torch.equal(x, y)
+    with pytest.raises(B.EsError):
+        sh.es_shard_wait_probe(0)
+    sh.close()
+
+
 def test_error_paths_launch_nothing(B, tiny):
     wd, _ = tiny
     ids = prompt_ids(0, 1, 8, TINY.vocab).cuda()

@@ -75,14 +75,14 @@ def test_static_scratch_takes_nothing_from_the_device_on_any_stream():
     B.es_op_decode_attention_static(q, k, v, table, ctx, max_ctx, out=out)          # warm-up: address look-up
     torch.cuda.synchronize()
     free_before = torch.cuda.mem_get_info()[0]
-    n_before = torch.cuda.memory_stats().get("allocation.all.allocated", 0)
     for i in range(6):
         st = side if i % 2 else None
         out.zero_()
         if st is not None:
             st.wait_stream(torch.cuda.current_stream())
+        n_before = torch.cuda.memory_stats().get("allocation.all.allocated", 0)
         got = B.es_op_decode_attention_static(q, k, v, table, ctx, max_ctx, out=out, stream=st)
+        assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == n_before   # nor from torch's allocator
         torch.cuda.synchronize()                     # the calls share one array: never two in flight
+        assert torch.cuda.mem_get_info()[0] == free_before
         assert torch.equal(got, want)
-    assert torch.cuda.mem_get_info()[0] == free_before
-    assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == n_before
