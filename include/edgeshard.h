@@ -290,11 +290,7 @@ ES_API es_status_t es_op_linear(const void *A, const void *W, const float *R, fl
  * With 3 <= M <= 16 (a decode step of several sequences) the weight-streaming kernel is used instead:
  * every CTA keeps one K slice of the activations in shared memory and streams 16-row groups of W over
  * it; K must be a multiple of 256 and K / 32 divisible by k_splits, a slice of 8 (M <= 8) or 16 rows
- * must fit 100 KB.  No second kernel runs in this form: the partial sums of a 16-column group go to the
- * workspace, and the warp whose partial arrives last (one arrival counter per group, kept at the end of
- * the workspace and cleared by this call) adds the slices in ascending order and the residual.  The
- * workspace layout is private; size it with es_op_linear_splitk_workspace_bytes.
- * M <= 2 is ES_ERR_UNSUPPORTED (such products never need slicing). */
+ * must fit 100 KB.  M <= 2 is ES_ERR_UNSUPPORTED (such products never need slicing). */
 ES_API size_t es_op_linear_splitk_workspace_bytes(int32_t M, int32_t N, int32_t k_splits);
 ES_API es_status_t es_op_linear_splitk(const void *A, const void *W, const float *R, float *C, int32_t M, int32_t N,
                                        int32_t K, int32_t k_splits, void *workspace, size_t workspace_bytes,

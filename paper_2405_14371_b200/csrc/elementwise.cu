@@ -1,4 +1,6 @@
 // Memory-bound helpers of the path: embedding gather, RMSNorm, greedy argmax, context counters.
+#include <cooperative_groups.h>
+
 #include "es_internal.cuh"
 #include "launch.cuh"
 
@@ -181,6 +183,177 @@ __global__ void __launch_bounds__(THREADS) splitk_reduce_kernel(const float* __r
   stamp_end(stamp);
 }
 
+// ---- up to 16 rows (decode steps of several sequences): a cluster of ROW_CTAS CTAs per row ------------------
+// With one CTA per row a 16-row launch runs on 16 SMs, and what one SM can pull in per microsecond bounds it: the
+// reduction of a product cut into 16 K slices reads 0.5 MB per row.  Here the columns of a row are cut into
+// ROW_CTAS contiguous parts, one per CTA of a thread-block cluster; each CTA adds up the squares of its part, the
+// parts' sums are exchanged through the cluster's shared memory and added in part order by every CTA, and each CTA
+// then normalises its own part.  Both kernels below use this one order of additions, so a row normalised in the
+// reduction and the same row normalised by the stand-alone kernel agree bit for bit.
+constexpr int ROW_CTAS = 8;
+constexpr int ROW_THREADS = 256;
+constexpr int ROW_REGS = 2;            // float4 columns per thread kept in registers (covers N <= 16384)
+
+// Sum of the ROW_CTAS per-CTA values, the same in every CTA of the cluster.  All threads of all CTAs call.
+__device__ __forceinline__ float cluster_row_total(float mine, float* parts /* [ROW_CTAS] shared */) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned rank = cluster.block_rank();
+  if (threadIdx.x < ROW_CTAS) *cluster.map_shared_rank(parts + rank, threadIdx.x) = mine;   // my value into everybody's slot
+  cluster.sync();
+  float total = 0.f;
+#pragma unroll
+  for (int r = 0; r < ROW_CTAS; ++r) total += parts[r];
+  return total;
+}
+
+// y[r, :] = rmsnorm(x[row r]) for M <= 16 rows; grid = M clusters of ROW_CTAS CTAs; N % (4 * ROW_CTAS) == 0.
+__global__ void __launch_bounds__(ROW_THREADS) rmsnorm_rows_kernel(const float* __restrict__ x, const __half* __restrict__ gain,
+                                                                   __half* __restrict__ y, int d, float eps, int64_t row_stride,
+                                                                   int64_t row_offset, const int* __restrict__ last_of,
+                                                                   unsigned long long* stamp) {
+  __shared__ float red[32];
+  __shared__ float parts[ROW_CTAS];
+  pdl_launch_dependents();
+  stamp_begin(stamp);
+  pdl_wait();
+  const int r = blockIdx.x / ROW_CTAS, part = blockIdx.x % ROW_CTAS;
+  const int64_t off = last_of ? (int64_t)last_of[r] - 1 : row_offset;
+  const int n4 = d / 4 / ROW_CTAS, lo = part * n4;                  // this CTA's float4 columns [lo, lo + n4)
+  const float4* src = reinterpret_cast<const float4*>(x + ((int64_t)r * row_stride + off) * d) + lo;
+  float4 v[ROW_REGS];
+  float ss = 0.f;
+#pragma unroll
+  for (int i = 0; i < ROW_REGS; ++i) {
+    const int c = threadIdx.x + i * ROW_THREADS;
+    if (c < n4) {
+      v[i] = src[c];
+      ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+    }
+  }
+  for (int c = threadIdx.x + ROW_REGS * ROW_THREADS; c < n4; c += ROW_THREADS) {
+    const float4 t = src[c];
+    ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+  }
+  const float total = cluster_row_total(block_sum(ss, red), parts);
+  const float inv = 1.0f / sqrtf(total / (float)d + eps);
+  __half2* dst = reinterpret_cast<__half2*>(y + (int64_t)r * d) + 2 * lo;
+  const __half2* g2 = reinterpret_cast<const __half2*>(gain) + 2 * lo;
+#pragma unroll
+  for (int i = 0; i < ROW_REGS; ++i) {
+    const int c = threadIdx.x + i * ROW_THREADS;
+    if (c < n4) {
+      const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
+      dst[2 * c] = __floats2half2_rn(v[i].x * inv * ga.x, v[i].y * inv * ga.y);
+      dst[2 * c + 1] = __floats2half2_rn(v[i].z * inv * gb.x, v[i].w * inv * gb.y);
+    }
+  }
+  for (int c = threadIdx.x + ROW_REGS * ROW_THREADS; c < n4; c += ROW_THREADS) {
+    const float4 t = src[c];
+    const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
+    dst[2 * c] = __floats2half2_rn(t.x * inv * ga.x, t.y * inv * ga.y);
+    dst[2 * c + 1] = __floats2half2_rn(t.z * inv * gb.x, t.w * inv * gb.y);
+  }
+  stamp_end(stamp);
+}
+
+// The split-K reduction for M <= 16 rows, same cluster shape: out[r, :] = res[r, :] + slices in ascending order,
+// then (with gain) y[r, :] = rmsnorm(out[r, :]).
+__global__ void __launch_bounds__(ROW_THREADS) splitk_reduce_rows_kernel(const float* __restrict__ part, int k_splits, const float* res,
+                                                                         float* out, int M, int N, int64_t ldo,
+                                                                         const __half* __restrict__ gain, __half* __restrict__ y,
+                                                                         float eps, unsigned long long* stamp) {
+  __shared__ float red[32];
+  __shared__ float parts[ROW_CTAS];
+  pdl_launch_dependents();
+  stamp_begin(stamp);
+  pdl_wait();
+  const int r = blockIdx.x / ROW_CTAS, pt = blockIdx.x % ROW_CTAS;
+  const int n4 = N / 4 / ROW_CTAS, lo = pt * n4;
+  const int64_t slice4 = (int64_t)M * N / 4;
+  const float4* src = reinterpret_cast<const float4*>(part + (int64_t)r * N) + lo;
+  const float4* rs = res ? reinterpret_cast<const float4*>(res + (int64_t)r * ldo) + lo : nullptr;
+  float4* dst = reinterpret_cast<float4*>(out + (int64_t)r * ldo) + lo;
+  auto finish = [&](int c, float4 a) {
+    for (int s0 = 0; s0 < k_splits; s0 += 8) {
+      float4 v[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        v[j] = (s0 + j < k_splits) ? __ldcs(src + (s0 + j) * slice4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (s0 + j < k_splits) { a.x += v[j].x; a.y += v[j].y; a.z += v[j].z; a.w += v[j].w; }
+    }
+    dst[c] = a;
+    return a;
+  };
+  float4 v[ROW_REGS];
+  float ss = 0.f;
+  // the residual may alias the output: all of a thread's residual elements are requested before it stores anything
+#pragma unroll
+  for (int i = 0; i < ROW_REGS; ++i) {
+    const int c = threadIdx.x + i * ROW_THREADS;
+    v[i] = (rs && c < n4) ? rs[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+#pragma unroll
+  for (int i = 0; i < ROW_REGS; ++i) {
+    const int c = threadIdx.x + i * ROW_THREADS;
+    if (c < n4) {
+      v[i] = finish(c, v[i]);
+      ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+    }
+  }
+  for (int c = threadIdx.x + ROW_REGS * ROW_THREADS; c < n4; c += ROW_THREADS) {
+    const float4 t = finish(c, rs ? rs[c] : make_float4(0.f, 0.f, 0.f, 0.f));
+    ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+  }
+  if (gain == nullptr) { stamp_end(stamp); return; }   // uniform over the cluster
+  const float total = cluster_row_total(block_sum(ss, red), parts);
+  const float inv = 1.0f / sqrtf(total / (float)N + eps);
+  __half2* yd = reinterpret_cast<__half2*>(y + (int64_t)r * N) + 2 * lo;
+  const __half2* g2 = reinterpret_cast<const __half2*>(gain) + 2 * lo;
+#pragma unroll
+  for (int i = 0; i < ROW_REGS; ++i) {
+    const int c = threadIdx.x + i * ROW_THREADS;
+    if (c < n4) {
+      const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
+      yd[2 * c] = __floats2half2_rn(v[i].x * inv * ga.x, v[i].y * inv * ga.y);
+      yd[2 * c + 1] = __floats2half2_rn(v[i].z * inv * gb.x, v[i].w * inv * gb.y);
+    }
+  }
+  for (int c = threadIdx.x + ROW_REGS * ROW_THREADS; c < n4; c += ROW_THREADS) {
+    const float4 t = dst[c];                         // written by this thread above
+    const float2 ga = __half22float2(g2[2 * c]), gb = __half22float2(g2[2 * c + 1]);
+    yd[2 * c] = __floats2half2_rn(t.x * inv * ga.x, t.y * inv * ga.y);
+    yd[2 * c + 1] = __floats2half2_rn(t.z * inv * gb.x, t.w * inv * gb.y);
+  }
+  stamp_end(stamp);
+}
+
+// Launch of the cluster kernels: M clusters of ROW_CTAS CTAs.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_row_clusters(void (*kernel)(KArgs...), int M, cudaStream_t stream, bool pdl, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(M * ROW_CTAS);
+  cfg.blockDim = dim3(ROW_THREADS);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = ROW_CTAS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// rows for which the cluster kernels are used: few enough that one CTA per row would leave most SMs idle
+constexpr int ROW_CLUSTER_MAX_ROWS = 16;
+inline bool use_row_clusters(int M, int N) { return M <= ROW_CLUSTER_MAX_ROWS && N % (4 * ROW_CTAS) == 0; }
+
 // Greedy token: index of the largest logit, the lowest index on ties.  One CTA per sequence.
 __global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ logits, int* __restrict__ out, int V,
                                                       unsigned long long* stamp) {
@@ -248,7 +421,9 @@ es_status_t launch_rmsnorm(const float* x, const __half* gain, __half* y, int M,
                            int64_t row_stride, int64_t row_offset, cudaStream_t s, int64_t* launches, bool pdl,
                            const int* last_of, unsigned long long* stamp) {
   if (M <= 0) return ES_OK;
-  if (M <= WIDE_ROWS_MAX)
+  if (use_row_clusters(M, d))
+    ES_CUDA_CHECK(launch_row_clusters(rmsnorm_rows_kernel, M, s, pdl, x, gain, y, d, eps, row_stride, row_offset, last_of, stamp));
+  else if (M <= WIDE_ROWS_MAX)
     ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset, last_of, stamp));
   else
     ES_CUDA_CHECK(launch_kernel(rmsnorm_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, x, gain, y, d, eps, row_stride, row_offset, last_of, stamp));
@@ -269,7 +444,9 @@ es_status_t launch_splitk_reduce(const float* part, int k_splits, const float* r
                                  unsigned long long* stamp) {
   if (M <= 0 || N <= 0) return ES_OK;
   if (N % 4 != 0 || ldo % 4 != 0) return fail(ES_ERR_SHAPE, "split-K reduction needs N and the row stride to be multiples of 4");
-  if (M <= WIDE_ROWS_MAX)
+  if (use_row_clusters(M, N))
+    ES_CUDA_CHECK(launch_row_clusters(splitk_reduce_rows_kernel, M, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps, stamp));
+  else if (M <= WIDE_ROWS_MAX)
     ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel<1024, 2>, dim3(M), dim3(1024), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps, stamp));
   else
     ES_CUDA_CHECK(launch_kernel(splitk_reduce_kernel<RMS_THREADS, RMS_REGS>, dim3(M), dim3(RMS_THREADS), 0, s, pdl, part, k_splits, res, out, M, N, ldo, gain, y, eps, stamp));

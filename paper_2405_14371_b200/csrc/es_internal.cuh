@@ -36,8 +36,7 @@ struct Tunables {
   int pdl;           // ES_PDL: programmatic dependent launch in decode steps (1, default) or plain stream order (0)
   int attn_mma;      // ES_ATTN_MMA: tensor-core decode attention for launches with many items (1, default) or never (0)
   int split_k;       // ES_SPLIT_K: split-K for the O and down projections of short prefills (1, default) or never (0)
-  int decode_fused_norm;   // ES_DECODE_FUSED_NORM: decode steps of 3..16 rows normalise inside the QKV / gate-up kernels (1) or with a launch of their own (0)
-  int ks_min_slice;        // ES_KS_MIN_SLICE: smallest K slice of the K-sliced streaming kernel (elements)
+  int ks_min_slice;        // ES_KS_MIN_SLICE: smallest K slice of the K-sliced streaming kernel (elements, default 512)
 };
 const Tunables& tunables();
 
@@ -60,17 +59,11 @@ struct LinearParams {
   const TcMaps* tc_maps;   // host pointer to pre-encoded maps (rows of A >= M), or nullptr: encode per launch
   const __half* A;
   int64_t lda;
-  // optional fused RMSNorm (weight-streaming kernels, M <= 16): A = rmsnorm(norm_x rows; norm_gain)
+  // optional fused RMSNorm (weight-streaming kernel, M <= 2): A = rmsnorm(norm_x rows; norm_gain)
   const float* norm_x;     // fp32 [M, K], row stride norm_ldx; nullptr = read A
   int64_t norm_ldx;
   const __half* norm_gain;
   float norm_eps;
-  // 3 <= M <= 16: the rows' sums of squares, one value per 16 columns [M, K / 16], written by the producer of
-  // norm_x (a plain epilogue with ssq_out, or launch_row_ssq); M <= 2: unused, the kernel sums the rows itself
-  const float* norm_ssq;
-  // plain epilogue of the tensor-core streaming kernels: also write the finished rows' sums of squares per 16
-  // columns [M, N / 16] (N % 16 == 0), or nullptr
-  float* ssq_out;
   const __half* w[3];
   int seg_rows[3];
   int M, N, K;
@@ -91,13 +84,10 @@ struct LinearParams {
   int T;                   // rows per sequence: row m belongs to sequence m / T at prompt offset m % T
   int is_decode;           // position = ctx_len[slot] instead of m % T
   int Hq, Hkv, hd, P, pages_per_slot, max_seq;
-  // split-K.  Tensor-core kernel with EPI_F32: > 1 = raw partial sums go to part[k_splits, M, N] and
-  // launch_splitk_reduce finishes the product.  K-sliced streaming kernel (any epilogue): partial sums go to
-  // part (linear_stream_mma_workspace_bytes) and the kernel finishes every 16-row unit itself through the
-  // arrival counters unit_cnt (one int per unit, zero before the launch and zero again after it)
+  // split-K (tensor-core kernel with EPI_F32; K-sliced streaming kernel with any epilogue): > 1 = raw partial
+  // sums go to part[k_splits, M, columns] and a second kernel finishes the product
   int k_splits;
   float* part;
-  int* unit_cnt;
   // CTA-pair tensor-core kernel: accumulators per tile, 1 = 256 x 256 tiles, 2 = 256 x 512 tiles, 0 = chosen per shape
   int pair_nacc;
   // k_splits > 1 on the tensor-core path: the CTA-pair kernel computes the slices (else the single-CTA kernel)
@@ -114,15 +104,10 @@ bool linear_stream_can_fuse_norm(int M);
 bool linear_stream_mma_supported(const LinearParams& p, int epi);
 es_status_t launch_linear_stream_mma(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl = false);
 // K slices across CTAs for this product (1 = the activations fit in shared memory whole); with p.k_splits > 1
-// the kernel needs p.part (linear_stream_mma_workspace_bytes) and p.unit_cnt and finishes the product itself
+// the kernel writes partial sums to p.part ([k_splits, M, N], SwiGLU: [k_splits, M, 2N] gate | up) and the
+// product is finished by launch_splitk_reduce (plain epilogue) or launch_splitk_finish (SwiGLU, QKV)
 int linear_stream_mma_splits(const LinearParams& p, int epi, size_t workspace_bytes);
-size_t linear_stream_mma_workspace_bytes(int M, int N, int epi, int k_splits);
-// true if the kernel chosen for p keeps the activations in shared memory (whole or as K slices), which is what
-// the fused RMSNorm (p.norm_x) needs
-bool linear_stream_mma_stages_activations(const LinearParams& p, int epi, size_t workspace_bytes);
-// ssq[m, c] = sum of squares of x[m, 16c .. 16c+15] for M <= 16 rows (the tree the plain epilogue uses)
-es_status_t launch_row_ssq(const float* x, int64_t ldx, float* ssq, int M, int d, cudaStream_t s, int64_t* launches,
-                           bool pdl = false, unsigned long long* stamp = nullptr);
+es_status_t launch_splitk_finish(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl = false);
 es_status_t launch_linear_tc(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, int* status_word, bool pdl = false);
 bool linear_tc_supported(const LinearParams& p, int epi);
 // number of K slices the tensor-core kernel should use for this product (1 = do not split), and the

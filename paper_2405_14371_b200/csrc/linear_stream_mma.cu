@@ -16,14 +16,8 @@
 //    shared memory and its warps stream different 16-row groups over that slice, so activations are
 //    read once per CTA rather than once per row group (on this machine what the SMs can take in
 //    is about what HBM delivers, so re-read activations cost as much as weights).  The slices' partial
-//    sums of a 16-row unit go to a workspace; the warp whose partial arrives last (an arrival counter per
-//    unit, nobody waits) adds the slices in slice order and applies the epilogue at once, while the other
-//    warps keep streaming: no finishing launch, and the order of additions is fixed;
-//  * the RMSNorm in front of the QKV and gate / up products is folded into the staging of the
-//    activations: the kernel reads the fp32 residual rows and multiplies by the gains and by the rows'
-//    1 / rms.  The sums of squares come, as one value per 16 columns, from the kernel that produced the
-//    rows (the plain epilogue below writes them) and are added up in a fixed order, so a row normalised
-//    here and a row normalised from sums written by another kernel agree bit for bit.
+//    sums go to a workspace [slices, M, columns] and a finishing kernel adds them in slice order and
+//    applies the epilogue.
 #include "epilogue.cuh"
 #include "launch.cuh"
 
@@ -53,90 +47,6 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// ---- sums of squares of residual rows, one value per 16 columns --------------------------------------------
-// The value for columns 16c .. 16c+15 of a row is a fixed tree: t_j = x[2j]^2 + x[2j+1]^2 (one multiply, one
-// fused multiply-add), then ((t0 + t1) + (t2 + t3)) + ((t4 + t5) + (t6 + t7)).  Eight adjacent lanes (an aligned
-// group) hold the pairs j = 0..7; every lane gets the value.  All 32 lanes must call.
-__device__ __forceinline__ float ssq16_of_pairs(float x0, float x1) {
-  float t = fmaf(x1, x1, x0 * x0);
-  t += __shfl_xor_sync(0xffffffffu, t, 1);
-  t += __shfl_xor_sync(0xffffffffu, t, 2);
-  t += __shfl_xor_sync(0xffffffffu, t, 4);
-  return t;
-}
-
-// 1 / rms of a row from its per-16-column sums (n_chunks of them), by one warp: lane l adds chunks l, l + 32, ...
-// in ascending order, then the lanes are combined by the xor butterfly.  Every lane returns the same value.
-__device__ __forceinline__ float row_inv_rms(const float* ssq_row, int n_chunks, int d, float eps, int lane) {
-  float t = 0.f;
-  for (int c = lane; c < n_chunks; c += 32) t += ssq_row[c];
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-  return 1.0f / sqrtf(t / (float)d + eps);
-}
-
-// Stages rows [0, rows) x columns [k_lo, k_lo + kslice) of the activations into shared memory (row stride
-// a_stride halves), rows >= p.M as zeros.  With p.norm_x the source is the fp32 residual stream and the rows are
-// normalised on the way (see above); otherwise it is the fp16 matrix p.A.
-__device__ __forceinline__ void stage_activations(const LinearParams& p, __half* a_s, int a_stride, int rows, int k_lo,
-                                                  int kslice, float* inv_s, int nthreads) {
-  const int chunks = kslice / 8;
-  if (p.norm_x != nullptr) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int m = warp; m < rows; m += nthreads / 32) {
-      const float inv = (m < p.M) ? row_inv_rms(p.norm_ssq + (int64_t)m * (p.K / 16), p.K / 16, p.K, p.norm_eps, lane) : 0.f;
-      if (lane == 0) inv_s[m] = inv;
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < rows * chunks; i += nthreads) {
-      const int m = i / chunks, c = i - m * chunks;
-      uint4 o = make_uint4(0, 0, 0, 0);
-      if (m < p.M) {
-        const float4* xr = reinterpret_cast<const float4*>(p.norm_x + (int64_t)m * p.norm_ldx + k_lo + c * 8);
-        const float4 xa = xr[0], xb = xr[1];
-        const uint4 gv = __ldg(reinterpret_cast<const uint4*>(p.norm_gain + k_lo + c * 8));
-        const __half2* g2 = reinterpret_cast<const __half2*>(&gv);
-        const float inv = inv_s[m];
-        const float2 g0 = __half22float2(g2[0]), g1 = __half22float2(g2[1]), g2f = __half22float2(g2[2]), g3 = __half22float2(g2[3]);
-        *reinterpret_cast<__half2*>(&o.x) = __floats2half2_rn(xa.x * inv * g0.x, xa.y * inv * g0.y);
-        *reinterpret_cast<__half2*>(&o.y) = __floats2half2_rn(xa.z * inv * g1.x, xa.w * inv * g1.y);
-        *reinterpret_cast<__half2*>(&o.z) = __floats2half2_rn(xb.x * inv * g2f.x, xb.y * inv * g2f.y);
-        *reinterpret_cast<__half2*>(&o.w) = __floats2half2_rn(xb.z * inv * g3.x, xb.w * inv * g3.y);
-      }
-      *reinterpret_cast<uint4*>(a_s + (int64_t)m * a_stride + c * 8) = o;
-    }
-  } else {
-    for (int i = threadIdx.x; i < rows * chunks; i += nthreads) {
-      const int m = i / chunks, c = i - m * chunks;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (m < p.M) v = *reinterpret_cast<const uint4*>(p.A + (int64_t)m * p.lda + k_lo + c * 8);
-      *reinterpret_cast<uint4*>(a_s + (int64_t)m * a_stride + c * 8) = v;
-    }
-  }
-  __syncthreads();
-}
-
-// Plain epilogue of columns (n, n + 1) of row m that also reports the sum of squares of the 16-column chunk the
-// pair belongs to: the eight lanes of an aligned group hold the chunk's eight pairs of one row.  All 32 lanes call
-// (rows >= M and columns >= N contribute nothing and store nothing); lane (n / 2) % 8 == 0 writes the chunk's value.
-__device__ __forceinline__ void epi_f32_pair_ssq(const LinearParams& p, int m, int n, float v0, float v1) {
-  const bool in = m < p.M && n < p.N;
-  const bool two = n + 1 < p.N;
-  if (in) {
-    const int64_t o = (int64_t)m * p.ldo + n;
-    if (p.res != nullptr) {
-      v0 += p.res[o];
-      if (two) v1 += p.res[o + 1];
-    }
-    p.out_f32[o] = v0;
-    if (two) p.out_f32[o + 1] = v1;
-  }
-  if (p.ssq_out != nullptr) {                      // uniform over the warp
-    const float t = ssq16_of_pairs(in ? v0 : 0.f, (in && two) ? v1 : 0.f);
-    if (in && ((n >> 1) & 7) == 0) p.ssq_out[(int64_t)m * (p.N / 16) + (n >> 4)] = t;
-  }
-}
-
 // NT: groups of 8 activation rows (1 or 2).  RG: 16-row groups of weights a warp carries at once (1 or
 // 2); with two, every activation fragment is used twice, which halves the activation traffic when
 // the activations do not fit in shared memory and come through L1 / L2.
@@ -147,7 +57,6 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __half* a_s = reinterpret_cast<__half*>(smem_raw);                 // [NT*8][a_stride], padded rows
   __shared__ float red[2][MW][RG][NT][32][4];
-  __shared__ float inv_s[NT * 8];
 
   const int K = p.K;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -212,7 +121,16 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
 
   pdl_wait();
 
-  if (A_SMEM) stage_activations(p, a_s, a_stride, NT * 8, 0, K, inv_s, MTHREADS);
+  if (A_SMEM) {
+    const int chunks = K / 8;
+    for (int i = threadIdx.x; i < NT * 8 * chunks; i += MTHREADS) {
+      const int m = i / chunks, c = i - m * chunks;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (m < p.M) v = *reinterpret_cast<const uint4*>(p.A + (int64_t)m * p.lda + c * 8);
+      *reinterpret_cast<uint4*>(a_s + (int64_t)m * a_stride + c * 8) = v;
+    }
+    __syncthreads();
+  }
 
   // In the unit epilogue below thread i always finishes activation row (i / 8) % (NT * 8) (the loop over idx runs
   // at most once: RG * 8 * NT * 8 <= MTHREADS): its slot, position and KV page are looked up once.
@@ -280,8 +198,7 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
         }
         const int u = u0 + cur_i;
         const int n = (EPI == EPI_SWIGLU) ? u * COLS + rg * 8 + pr : u * COLS + rg * 16 + 2 * pr;
-        if (EPI == EPI_F32) epi_f32_pair_ssq(p, m, n, v0, v1);   // whole warps run this loop: the chunk's 8 pairs sit in 8 adjacent lanes
-        else epi_pair_row<EPI>(p, qrow, m, n, v0, v1);  // idx == threadIdx.x: the row is the one looked up before the loop
+        epi_pair_row<EPI>(p, qrow, m, n, v0, v1);       // idx == threadIdx.x: the row is the one looked up before the loop
       }
       cur_cc = 0;
       ++cur_i;
@@ -302,74 +219,14 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_kernel(const Li
 // ---- K sliced across CTAs (activations too large for shared memory) ---------------------------------
 // CTA blockIdx.x works on K slice blockIdx.x / n_col_ctas and on the (blockIdx.x % n_col_ctas)-th balanced
 // range of 16-row units; warp w takes units w, w + 8, ... of that range over the CTA's whole slice.
-// The raw accumulators of a unit go to part[unit][slice][activation row][weight row of the unit] (with
-// SwiGLU weight rows 0..7 are gate rows and 8..15 the up rows of the same columns).  After its stores a warp
-// bumps the unit's arrival counter; the warp that finds every other slice already there adds the slices in
-// slice order, applies the epilogue and puts the counter back to zero for the next launch.
-template <int NT, int EPI>
-__device__ __forceinline__ void finish_unit(const LinearParams& p, const float* upart, int u, int lane) {
-  constexpr int ROWS = NT * 8;
-  const int pr = lane & 7, mrow = lane >> 3;
-  const int64_t slice = ROWS * 16;
-#pragma unroll 1
-  for (int it = 0; it < ROWS / 4; ++it) {
-    const int m = it * 4 + mrow;
-    const float* src = upart + m * 16;
-    float v0 = 0.f, v1 = 0.f;
-    // plain form: the residual pair is requested with the slices (same lane reads and writes it)
-    float r0 = 0.f, r1 = 0.f;
-    const int n = (EPI == EPI_SWIGLU) ? u * 8 + pr : u * 16 + 2 * pr;
-    const bool in = m < p.M && n < p.N;
-    if (EPI == EPI_F32 && p.res != nullptr && in) {
-      const int64_t o = (int64_t)m * p.ldo + n;
-      r0 = p.res[o];
-      if (n + 1 < p.N) r1 = p.res[o + 1];
-    }
-    for (int s0 = 0; s0 < p.k_splits; s0 += 8) {      // eight slices are requested at a time, added in slice order
-      float a[8], b[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const bool have = s0 + j < p.k_splits;
-        if (EPI == EPI_SWIGLU) {
-          a[j] = have ? __ldcg(src + (s0 + j) * slice + pr) : 0.f;
-          b[j] = have ? __ldcg(src + (s0 + j) * slice + 8 + pr) : 0.f;
-        } else {
-          const float2 t = have ? __ldcg(reinterpret_cast<const float2*>(src + (s0 + j) * slice + 2 * pr)) : make_float2(0.f, 0.f);
-          a[j] = t.x;
-          b[j] = t.y;
-        }
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j)
-        if (s0 + j < p.k_splits) { v0 += a[j]; v1 += b[j]; }
-    }
-    if (EPI == EPI_F32) {
-      const bool two = n + 1 < p.N;
-      if (in) {
-        const int64_t o = (int64_t)m * p.ldo + n;
-        if (p.res != nullptr) { v0 += r0; if (two) v1 += r1; }
-        p.out_f32[o] = v0;
-        if (two) p.out_f32[o + 1] = v1;
-      }
-      if (p.ssq_out != nullptr) {
-        const float t = ssq16_of_pairs(in ? v0 : 0.f, (in && two) ? v1 : 0.f);
-        if (in && pr == 0) p.ssq_out[(int64_t)m * (p.N / 16) + u] = t;
-      }
-    } else if (EPI == EPI_QKV) {
-      if (in) epi_qkv_pair_row(p, qkv_row(p, m), n, v0, v1);
-    } else {
-      epi_swiglu(p, m, n, v0, v1);
-    }
-  }
-}
-
+// Raw accumulators are stored to part[slice][m][column]; with SwiGLU the gate rows land in columns
+// [0, N) and the up rows in [N, 2N).
 template <int NT, int EPI>
 __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_ks_kernel(const LinearParams p, int a_stride, int n_col_ctas) {
   pdl_launch_dependents();
   stamp_begin(p.stamp);
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __half* a_s = reinterpret_cast<__half*>(smem_raw);                 // [NT*8][a_stride]: this CTA's K slice of the activations
-  __shared__ float inv_s[NT * 8];
 
   const int K = p.K;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -377,7 +234,6 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_ks_kernel(const
   constexpr int COLS = (EPI == EPI_SWIGLU) ? 8 : 16;
   constexpr int UM = UM_TOTAL;
   constexpr int CHUNK_K = KSTEP * UM;
-  constexpr int ROWS = NT * 8;
   const int ks = blockIdx.x / n_col_ctas, nc = blockIdx.x - ks * n_col_ctas;
   const int kslice = K / p.k_splits;                                  // multiple of KSTEP (host)
   const int k_lo = ks * kslice, k_hi = k_lo + kslice;
@@ -428,7 +284,16 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_ks_kernel(const
 
   pdl_wait();
 
-  stage_activations(p, a_s, a_stride, ROWS, k_lo, kslice, inv_s, MTHREADS);
+  {
+    const int chunks = kslice / 8;
+    for (int i = threadIdx.x; i < NT * 8 * chunks; i += MTHREADS) {
+      const int m = i / chunks, c = i - m * chunks;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (m < p.M) v = *reinterpret_cast<const uint4*>(p.A + (int64_t)m * p.lda + k_lo + c * 8);
+      *reinterpret_cast<uint4*>(a_s + (int64_t)m * a_stride + c * 8) = v;
+    }
+    __syncthreads();
+  }
 
   float acc[NT][4];
 #pragma unroll
@@ -436,7 +301,8 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_ks_kernel(const
 #pragma unroll
     for (int i = 0; i < 4; ++i) acc[t][i] = 0.f;
   int cur_i = 0, cur_cc = 0;
-  const int64_t unit_stride = (int64_t)p.k_splits * ROWS * 16;
+  const int64_t part_cols = (EPI == EPI_SWIGLU) ? 2 * (int64_t)p.N : p.N;
+  float* part = p.part + (int64_t)ks * p.M * part_cols;
 
   auto consume = [&](const uint4 (&w0)[UM], const uint4 (&w1)[UM]) {
     const int kb = cur_cc * CHUNK_K + q * 8;                          // offset inside the slice
@@ -456,29 +322,23 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_ks_kernel(const
       // accumulator element (weight row r, activation row m) of group t: lane (r % 8) * 4 + (m % 8) / 2,
       // register (r / 8) * 2 + (m % 2)
       const int u = u0 + warp + cur_i * MW;
-      float* upart = p.part + (int64_t)u * unit_stride;
-      float* mine = upart + (int64_t)ks * ROWS * 16;
+      const int na = u * COLS + g;                                     // rows 0..7 of the unit
+      const int64_t ca = na;
+      const int64_t cb = (EPI == EPI_SWIGLU) ? (int64_t)p.N + na : (int64_t)na + 8;
+      const bool va = na < p.N, vb = (EPI == EPI_SWIGLU) ? va : (na + 8 < p.N);
 #pragma unroll
       for (int t = 0; t < NT; ++t) {
         const int m0 = t * 8 + 2 * q;
-        __stcg(mine + m0 * 16 + g, acc[t][0]);
-        __stcg(mine + (m0 + 1) * 16 + g, acc[t][1]);
-        __stcg(mine + m0 * 16 + g + 8, acc[t][2]);
-        __stcg(mine + (m0 + 1) * 16 + g + 8, acc[t][3]);
+        if (m0 < p.M) {
+          if (va) part[(int64_t)m0 * part_cols + ca] = acc[t][0];
+          if (vb) part[(int64_t)m0 * part_cols + cb] = acc[t][2];
+        }
+        if (m0 + 1 < p.M) {
+          if (va) part[(int64_t)(m0 + 1) * part_cols + ca] = acc[t][1];
+          if (vb) part[(int64_t)(m0 + 1) * part_cols + cb] = acc[t][3];
+        }
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[t][i] = 0.f;
-      }
-      // arrival: the stores above are made visible before the counter moves; whoever sees k_splits - 1 earlier
-      // arrivals owns the unit
-      __threadfence();
-      __syncwarp();
-      int prev = 0;
-      if (lane == 0) prev = atomicAdd(p.unit_cnt + u, 1);
-      prev = __shfl_sync(0xffffffffu, prev, 0);
-      if (prev == p.k_splits - 1) {
-        __threadfence();
-        finish_unit<NT, EPI>(p, upart, u, lane);
-        if (lane == 0) p.unit_cnt[u] = 0;
       }
       cur_cc = 0;
       ++cur_i;
@@ -496,21 +356,51 @@ __global__ void __launch_bounds__(MTHREADS, 2) linear_stream_mma_ks_kernel(const
   stamp_end(p.stamp);
 }
 
-// Sums of squares per 16 columns of M <= 16 fp32 rows (the same tree as the plain epilogue writes): for rows that
-// no product of this library produced (embedding rows, an activation handed over by another shard).
-__global__ void __launch_bounds__(256) row_ssq_kernel(const float* __restrict__ x, int64_t ldx, float* __restrict__ ssq, int M,
-                                                      int d, unsigned long long* stamp) {
+// Adds the K slices of one output pair in slice order and applies the epilogue (SwiGLU / QKV forms;
+// the plain form is finished by the reduction kernel that also fuses the following RMSNorm).
+template <int EPI>
+__global__ void __launch_bounds__(256) splitk_finish_kernel(const LinearParams p) {
   pdl_launch_dependents();
-  stamp_begin(stamp);
+  stamp_begin(p.stamp);
   pdl_wait();
-  const int pairs = d / 2;                                            // d % 16 == 0: whole warps stay together
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < (int64_t)M * pairs; i += (int64_t)gridDim.x * blockDim.x) {
-    const int m = (int)(i / pairs), j = (int)(i - (int64_t)m * pairs);
-    const float2 v = *reinterpret_cast<const float2*>(x + (int64_t)m * ldx + 2 * j);
-    const float t = ssq16_of_pairs(v.x, v.y);
-    if ((j & 7) == 0) ssq[(int64_t)m * (d / 16) + (j >> 3)] = t;
+  const int pairs = (EPI == EPI_SWIGLU) ? p.N : (p.N + 1) / 2;
+  const int64_t part_cols = (EPI == EPI_SWIGLU) ? 2 * (int64_t)p.N : p.N;
+  const int64_t slice = (int64_t)p.M * part_cols;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < (int64_t)p.M * pairs; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int m = (int)(idx / pairs), pr = (int)(idx - (int64_t)m * pairs);
+    const int n = (EPI == EPI_SWIGLU) ? pr : 2 * pr;
+    const int64_t c0 = n, c1 = (EPI == EPI_SWIGLU) ? (int64_t)p.N + n : (int64_t)n + 1;
+    const bool has1 = (EPI == EPI_SWIGLU) || (n + 1 < p.N);
+    const float* src = p.part + (int64_t)m * part_cols;
+    // the row's slot, position and KV page do not depend on the sums: looked up while the slices are on their way
+    QkvRow row;
+    if (EPI == EPI_QKV) row = qkv_row(p, m);
+    float v0 = 0.f, v1 = 0.f;
+    // eight slices are requested at a time and then added in slice order; adjacent columns (n even, N even) come
+    // as one 8-byte load
+    const bool pair8 = (EPI != EPI_SWIGLU) && has1 && ((part_cols & 1) == 0);
+    for (int s0 = 0; s0 < p.k_splits; s0 += 8) {
+      float a[8], b[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const bool in = s0 + j < p.k_splits;
+        if (pair8) {
+          const float2 t = in ? __ldcs(reinterpret_cast<const float2*>(src + (s0 + j) * slice + c0)) : make_float2(0.f, 0.f);
+          a[j] = t.x;
+          b[j] = t.y;
+        } else {
+          a[j] = in ? __ldcs(src + (s0 + j) * slice + c0) : 0.f;
+          b[j] = (in && has1) ? __ldcs(src + (s0 + j) * slice + c1) : 0.f;
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (s0 + j < p.k_splits) { v0 += a[j]; v1 += b[j]; }
+    }
+    if (EPI == EPI_QKV) epi_qkv_pair_row(p, row, n, v0, v1);
+    else epi_pair<EPI>(p, m, n, v0, v1);
   }
-  stamp_end(stamp);
+  stamp_end(p.stamp);
 }
 
 template <int NT, int EPI>
@@ -575,13 +465,9 @@ es_status_t launch_epi(const LinearParams& p, cudaStream_t s, bool pdl) {
 }  // namespace
 
 bool linear_stream_mma_supported(const LinearParams& p, int epi) {
-  if (p.M < 1 || p.M > 16 || p.N <= 0) return false;
+  if (p.M < 1 || p.M > 16 || p.N <= 0 || p.norm_x != nullptr) return false;
   if (p.K % (MW * KSTEP) != 0) return false;            // every warp gets a whole number of 32-element steps
-  if (p.norm_x == nullptr && (p.lda % 8 != 0 || ((uintptr_t)p.A % 16))) return false;
-  if (p.norm_x != nullptr && (p.norm_ssq == nullptr || p.norm_gain == nullptr || p.norm_ldx % 4 != 0 ||
-                              (((uintptr_t)p.norm_x | (uintptr_t)p.norm_gain) % 16)))
-    return false;
-  if (p.ssq_out != nullptr && (epi != EPI_F32 || p.N % 16 != 0)) return false;
+  if (p.lda % 8 != 0 || ((uintptr_t)p.A % 16)) return false;
   for (int i = 0; i < 3; ++i)
     if (p.w[i] && ((uintptr_t)p.w[i] % 16)) return false;
   if (epi == EPI_QKV && (p.N % 2)) return false;
@@ -595,6 +481,7 @@ int linear_stream_mma_splits(const LinearParams& p, int epi, size_t workspace_by
   const int steps = p.K / KSTEP;
   const int cols = (epi == EPI_SWIGLU) ? 8 : 16;
   const int n_units = (p.N + cols - 1) / cols;
+  const size_t part_cols = (epi == EPI_SWIGLU) ? 2 * (size_t)p.N : (size_t)p.N;
   int best = 1;
   long long best_cost = 0;
   for (int ks = 2; ks <= 64 && ks <= KS_GRID; ++ks) {
@@ -602,7 +489,7 @@ int linear_stream_mma_splits(const LinearParams& p, int epi, size_t workspace_by
     const int kslice = p.K / ks;
     if (kslice < tunables().ks_min_slice) break;
     if ((size_t)nt * 8 * (kslice + 8) * sizeof(__half) > KS_SMEM_MAX) continue;
-    if (linear_stream_mma_workspace_bytes(p.M, p.N, epi, ks) > workspace_bytes) continue;
+    if ((size_t)ks * p.M * part_cols * sizeof(float) > workspace_bytes) continue;
     const int ncol = KS_GRID / ks;
     const int units_per_cta = (n_units + ncol - 1) / ncol;
     const long long cost = (long long)((units_per_cta + MW - 1) / MW) * kslice;   // K elements the busiest warp walks
@@ -611,28 +498,17 @@ int linear_stream_mma_splits(const LinearParams& p, int epi, size_t workspace_by
   return best;
 }
 
-size_t linear_stream_mma_workspace_bytes(int M, int N, int epi, int k_splits) {
-  const int cols = (epi == EPI_SWIGLU) ? 8 : 16;
-  const size_t n_units = (size_t)(N + cols - 1) / cols;
-  const size_t rows = M <= 8 ? 8 : 16;
-  return n_units * k_splits * rows * 16 * sizeof(float);
-}
-
-bool linear_stream_mma_stages_activations(const LinearParams& p, int epi, size_t workspace_bytes) {
-  if (!linear_stream_mma_supported(p, epi)) return false;
-  const int nt = p.M <= 8 ? 1 : 2;
-  if ((size_t)nt * 8 * (p.K + 8) * sizeof(__half) <= KS_SMEM_MAX) return true;
-  return linear_stream_mma_splits(p, epi, workspace_bytes) > 1;
-}
-
-es_status_t launch_row_ssq(const float* x, int64_t ldx, float* ssq, int M, int d, cudaStream_t s, int64_t* launches, bool pdl,
-                           unsigned long long* stamp) {
-  if (M <= 0) return ES_OK;
-  if (d % 16 != 0 || ldx % 2 != 0) return fail(ES_ERR_SHAPE, "row sums of squares need d to be a multiple of 16");
-  const long long work = (long long)M * (d / 2);
+es_status_t launch_splitk_finish(const LinearParams& p, int epi, cudaStream_t s, int64_t* launches, bool pdl) {
+  if (p.k_splits < 2 || p.part == nullptr) return fail(ES_ERR_INVALID_ARG, "nothing to finish");
+  const int pairs = (epi == EPI_SWIGLU) ? p.N : (p.N + 1) / 2;
+  const long long work = (long long)p.M * pairs;
   int grid = (int)((work + 255) / 256);
-  if (grid > 296) grid = 296;
-  ES_CUDA_CHECK(launch_kernel(row_ssq_kernel, dim3(grid), dim3(256), 0, s, pdl, x, ldx, ssq, M, d, stamp));
+  if (grid > 4 * 148) grid = 4 * 148;
+  switch (epi) {
+    case EPI_SWIGLU: ES_CUDA_CHECK(launch_kernel(splitk_finish_kernel<EPI_SWIGLU>, dim3(grid), dim3(256), 0, s, pdl, p)); break;
+    case EPI_QKV: ES_CUDA_CHECK(launch_kernel(splitk_finish_kernel<EPI_QKV>, dim3(grid), dim3(256), 0, s, pdl, p)); break;
+    default: return fail(ES_ERR_INVALID_ARG, "the plain epilogue is finished by the reduction kernel");
+  }
   if (launches) ++*launches;
   return ES_OK;
 }
@@ -641,12 +517,10 @@ es_status_t launch_linear_stream_mma(const LinearParams& p, int epi, cudaStream_
   if (!linear_stream_mma_supported(p, epi)) return fail(ES_ERR_UNSUPPORTED, "tensor-core streaming kernel does not take this shape");
   if (p.k_splits > 1) {
     const int nt = p.M <= 8 ? 1 : 2;
-    if (p.part == nullptr || p.unit_cnt == nullptr || (p.K / KSTEP) % p.k_splits != 0 || p.k_splits > KS_GRID ||
+    if (p.part == nullptr || (p.K / KSTEP) % p.k_splits != 0 || p.k_splits > KS_GRID ||
         (size_t)nt * 8 * (p.K / p.k_splits + 8) * sizeof(__half) > KS_SMEM_MAX)
       return fail(ES_ERR_INVALID_ARG, "K-sliced streaming kernel: %d slices do not fit K = %d", p.k_splits, p.K);
   }
-  if (p.norm_x != nullptr && p.k_splits <= 1 && (size_t)(p.M <= 8 ? 8 : 16) * (p.K + 8) * sizeof(__half) > KS_SMEM_MAX)
-    return fail(ES_ERR_UNSUPPORTED, "the fused RMSNorm needs the activations staged in shared memory");
   es_status_t st;
   switch (epi) {
     case EPI_F32: st = launch_epi<EPI_F32>(p, s, pdl); break;

@@ -41,7 +41,7 @@ static int env_int(const char* name, int dflt) {
 }
 
 const Tunables& tunables() {
-  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_TC_PAIR_WIDE", 1), env_int("ES_SPLIT_PAIRS", 1), env_int("ES_PDL", 1), env_int("ES_ATTN_MMA", 1), env_int("ES_SPLIT_K", 1), env_int("ES_DECODE_FUSED_NORM", 1), env_int("ES_KS_MIN_SLICE", 512)};
+  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_TC_PAIR_WIDE", 1), env_int("ES_SPLIT_PAIRS", 1), env_int("ES_PDL", 1), env_int("ES_ATTN_MMA", 1), env_int("ES_SPLIT_K", 1), env_int("ES_KS_MIN_SLICE", 512)};
   return t;
 }
 
@@ -72,8 +72,7 @@ struct Layout {
   size_t page_elems;   // halves in one page of one of K / V
   size_t kv_bytes;
   size_t off_x, off_h, off_q, off_ao, off_act, off_logits, off_next, off_hlast, off_part, off_cos, off_sin,
-      off_table, off_ctx, off_slots, off_status, off_splitk, off_stamps, off_ssq, off_unitcnt;
-  size_t unit_cnt_bytes;
+      off_table, off_ctx, off_slots, off_status, off_splitk, off_stamps;
   size_t scratch_bytes;
 };
 
@@ -127,17 +126,6 @@ Layout make_layout(const es_model_desc_t& d, int begin, int end) {
   L.off_slots = take(2 * B * 4);       // slots, then the prompt lengths of a ragged prefill
   L.off_status = take(256);
   L.off_splitk = take(d.max_tokens > 2 ? linear_tc_split_workspace_bytes() : 0);   // split-K partial sums of short prefills
-  // decode steps of 3..16 sequences: the rows' sums of squares per 16 columns, and one arrival counter per
-  // 16-row unit of the widest product (QKV: 16 columns per unit, gate / up: 8)
-  L.off_ssq = take((size_t)16 * (d.d_model / 16 + 1) * 4);
-  {
-    const size_t nqkv = (size_t)(d.n_heads + 2 * d.n_kv_heads) * d.head_dim;
-    size_t units = nqkv / 16 + 1;
-    if ((size_t)d.d_ffn / 8 + 1 > units) units = (size_t)d.d_ffn / 8 + 1;
-    if ((size_t)d.d_model / 16 + 1 > units) units = (size_t)d.d_model / 16 + 1;
-    L.off_unitcnt = take(units * 4);
-    L.unit_cnt_bytes = units * 4;
-  }
   L.off_stamps = take((size_t)2 * STAMP_SLOTS * sizeof(unsigned long long));
   L.scratch_bytes = o;
   return L;
@@ -188,8 +176,6 @@ struct es_shard {
   float *logits, *part, *rope_cos, *rope_sin;
   int *next_ids, *block_table, *ctx_len, *slots_dev, *lens_dev, *status;
   float* splitk = nullptr;      // split-K workspace (nullptr when the shard never runs more than 2 rows)
-  float* ssq = nullptr;         // [16, d_model / 16] sums of squares of the residual rows of a decode step
-  int* unit_cnt = nullptr;      // arrival counters of the K-sliced streaming kernel (zero between launches)
   std::vector<int> ctx;         // host mirror of ctx_len, -1 = never prefilled
   std::vector<int> slots_host;  // slots currently uploaded to slots_dev
   std::vector<int> lens_host;   // prompt lengths of the last ragged prefill (source of the upload)
@@ -343,16 +329,17 @@ int split_k_for(const es_shard* s, LinearParams& p, int epi) {
   return linear_tc_splits(p, epi);
 }
 
-// A product of a decode step (at most 16 rows): with 3 or more rows its K range may be sliced across CTAs, and
-// the kernel then finishes the product itself (no second launch).
-es_status_t run_linear_decode(es_shard* s, LinearParams& p, int epi) {
+// A product whose K range may be sliced (QKV and gate / up forms): the kernel, then the finishing kernel.
+es_status_t run_linear_sliced(es_shard* s, LinearParams& p, int epi, bool pdl) {
   const int splits = split_k_for(s, p, epi);
-  if (splits > 1) {
-    p.k_splits = splits;
-    p.part = s->splitk;
-    p.unit_cnt = s->unit_cnt;
-  }
-  return run_linear(s, p, epi);
+  if (splits <= 1 || p.M > 16) return run_linear(s, p, epi);
+  p.k_splits = splits;
+  p.part = s->splitk;
+  ES_TRY(run_linear(s, p, epi));
+  p.stamp = next_stamp(s, ES_KT_FINISH, 0.0);
+  ES_TRY(kt_begin(s));
+  ES_TRY(launch_splitk_finish(p, epi, s->stream, &s->launches, pdl));
+  return kt_end(s, ES_KT_FINISH, 0.0);
 }
 
 // Parameters of the four linear layers of decoder layer li (kind: 0 qkv, 1 o, 2 gate/up, 3 down).
@@ -429,36 +416,11 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
   } else {
     xin = hidden_in;
   }
-  // Decode steps of 3..16 sequences: the RMSNorm in front of QKV and gate / up is done by those kernels while
-  // they stage their activations, from sums of squares that the O and down epilogues write (all layers have the
-  // same shapes, so one check serves the pass).
-  bool cn = false;
-  if (M > 2 && M <= 16 && !fuse_norm && s->splitk != nullptr && d.d_model % 16 == 0 && s->nl > 0 && tunables().decode_fused_norm != 0) {
-    cn = true;
-    for (int kind = 0; kind < 4 && cn; ++kind) {
-      int epi = 0;
-      LinearParams p = layer_linear(s, 0, kind, M, T, decode, xin, &epi);
-      if (kind == 0 || kind == 2) {
-        p.norm_x = s->x; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)s->lw[0].attn_norm; p.norm_eps = d.rms_eps; p.norm_ssq = s->ssq;
-        cn = linear_stream_mma_stages_activations(p, epi, linear_tc_split_workspace_bytes());
-      } else {
-        p.ssq_out = s->ssq;
-        cn = linear_stream_mma_supported(p, epi);
-      }
-    }
-  }
-  if (cn) {
-    const bool pdl_first = s->has_emb ? pdl : false;                  // first kernel of the pass: full dependency
-    ES_TRY(kt_begin(s));
-    ES_TRY(launch_row_ssq(xin, d.d_model, s->ssq, M, d.d_model, s->stream, &s->launches, pdl_first,
-                          next_stamp(s, ES_KT_RMSNORM, (double)M * d.d_model * 4.0)));
-    ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)M * d.d_model * 4.0));
-  }
   for (int li = 0; li < s->nl; ++li, ++pi) {
     const es_layer_weights_t& w = s->lw[li];
     prof_mark(s, pi, 0);
-    const bool pdl0 = (li == 0 && !s->has_emb && !cn) ? false : pdl;     // first kernel of the pass: full dependency
-    if (!fuse_norm && !h_ready && !cn) {
+    const bool pdl0 = (li == 0 && !s->has_emb) ? false : pdl;     // first kernel of the pass: full dependency
+    if (!fuse_norm && !h_ready) {
       ES_TRY(kt_begin(s));
       ES_TRY(launch_rmsnorm(xin, (const __half*)w.attn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl0,
                             nullptr, next_stamp(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0)));
@@ -468,12 +430,10 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     int epi = 0;
     {
       LinearParams p = layer_linear(s, li, 0, M, T, decode, xin, &epi);
-      if (fuse_norm || cn) { p.norm_x = xin; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.attn_norm; p.norm_eps = d.rms_eps; }
-      if (cn) p.norm_ssq = s->ssq;
+      if (fuse_norm) { p.norm_x = xin; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.attn_norm; p.norm_eps = d.rms_eps; }
       s->kt_next_cat = ES_KT_QKV;
       s->pdl_now = fuse_norm ? pdl0 : pdl;
-      if (M <= 16) ES_TRY(run_linear_decode(s, p, epi));
-      else ES_TRY(run_linear(s, p, epi));
+      ES_TRY(run_linear_sliced(s, p, epi, pdl));
       s->pdl_now = pdl;
     }
     KvView kvv{};
@@ -503,28 +463,23 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     {
       LinearParams p = layer_linear(s, li, 1, M, T, decode, xin, &epi);
       s->kt_next_cat = ES_KT_O;
-      if (M <= 16) {
-        if (cn) p.ssq_out = s->ssq;
-        ES_TRY(run_linear_decode(s, p, epi));
+      const int splits = split_k_for(s, p, epi);
+      if (splits > 1) {
+        // short prompt: K slices into the workspace, then residual + RMSNorm for gate / up in the reduction
+        p.k_splits = splits; p.part = s->splitk;
+        ES_TRY(run_linear(s, p, epi));
+        ES_TRY(kt_begin(s));
+        ES_TRY(launch_splitk_reduce(s->splitk, splits, p.res, p.out_f32, M, p.N, p.ldo, (const __half*)w.ffn_norm, s->h,
+                                    d.rms_eps, s->stream, &s->launches, pdl,
+                                    next_stamp(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + 2.0))));
+        ES_TRY(kt_end(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + 2.0)));
+        o_split = true;
       } else {
-        const int splits = split_k_for(s, p, epi);
-        if (splits > 1) {
-          // short prompt: K slices into the workspace, then residual + RMSNorm for gate / up in the reduction
-          p.k_splits = splits; p.part = s->splitk;
-          ES_TRY(run_linear(s, p, epi));
-          ES_TRY(kt_begin(s));
-          ES_TRY(launch_splitk_reduce(s->splitk, splits, p.res, p.out_f32, M, p.N, p.ldo, (const __half*)w.ffn_norm, s->h,
-                                      d.rms_eps, s->stream, &s->launches, pdl,
-                                      next_stamp(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + 2.0))));
-          ES_TRY(kt_end(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + 2.0)));
-          o_split = true;
-        } else {
-          ES_TRY(run_linear(s, p, epi));
-        }
+        ES_TRY(run_linear(s, p, epi));
       }
     }
     xin = s->x;
-    if (!fuse_norm && !o_split && !cn) {
+    if (!fuse_norm && !o_split) {
       ES_TRY(kt_begin(s));
       ES_TRY(launch_rmsnorm(s->x, (const __half*)w.ffn_norm, s->h, M, d.d_model, d.rms_eps, 1, 0, s->stream, &s->launches, pdl,
                             nullptr, next_stamp(s, ES_KT_RMSNORM, (double)M * d.d_model * 6.0)));
@@ -532,35 +487,28 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     }
     {
       LinearParams p = layer_linear(s, li, 2, M, T, decode, xin, &epi);
-      if (fuse_norm || cn) { p.norm_x = s->x; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.ffn_norm; p.norm_eps = d.rms_eps; }
-      if (cn) p.norm_ssq = s->ssq;
+      if (fuse_norm) { p.norm_x = s->x; p.norm_ldx = d.d_model; p.norm_gain = (const __half*)w.ffn_norm; p.norm_eps = d.rms_eps; }
       s->kt_next_cat = ES_KT_GATE_UP;
-      if (M <= 16) ES_TRY(run_linear_decode(s, p, epi));
-      else ES_TRY(run_linear(s, p, epi));
+      ES_TRY(run_linear_sliced(s, p, epi, pdl));
     }
     {
       LinearParams p = layer_linear(s, li, 3, M, T, decode, xin, &epi);
       s->kt_next_cat = ES_KT_DOWN;
-      if (M <= 16) {
-        if (cn) p.ssq_out = s->ssq;
-        ES_TRY(run_linear_decode(s, p, epi));
+      const int splits = split_k_for(s, p, epi);
+      if (splits > 1) {
+        // the reduction also normalises the finished rows for the next layer's QKV projection
+        p.k_splits = splits; p.part = s->splitk;
+        ES_TRY(run_linear(s, p, epi));
+        const bool more = li + 1 < s->nl;
+        ES_TRY(kt_begin(s));
+        ES_TRY(launch_splitk_reduce(s->splitk, splits, p.res, p.out_f32, M, p.N, p.ldo,
+                                    more ? (const __half*)s->lw[li + 1].attn_norm : nullptr, s->h, d.rms_eps, s->stream,
+                                    &s->launches, pdl,
+                                    next_stamp(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + (more ? 2.0 : 0.0)))));
+        ES_TRY(kt_end(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + (more ? 2.0 : 0.0))));
+        h_ready = more;
       } else {
-        const int splits = split_k_for(s, p, epi);
-        if (splits > 1) {
-          // the reduction also normalises the finished rows for the next layer's QKV projection
-          p.k_splits = splits; p.part = s->splitk;
-          ES_TRY(run_linear(s, p, epi));
-          const bool more = li + 1 < s->nl;
-          ES_TRY(kt_begin(s));
-          ES_TRY(launch_splitk_reduce(s->splitk, splits, p.res, p.out_f32, M, p.N, p.ldo,
-                                      more ? (const __half*)s->lw[li + 1].attn_norm : nullptr, s->h, d.rms_eps, s->stream,
-                                      &s->launches, pdl,
-                                      next_stamp(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + (more ? 2.0 : 0.0)))));
-          ES_TRY(kt_end(s, ES_KT_REDUCE, (double)M * d.d_model * (8.0 + 4.0 * splits + (more ? 2.0 : 0.0))));
-          h_ready = more;
-        } else {
-          ES_TRY(run_linear(s, p, epi));
-        }
+        ES_TRY(run_linear(s, p, epi));
       }
     }
     prof_mark(s, pi, 1);
@@ -703,8 +651,6 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
   s->status = (int*)(sb + L.off_status);
   s->splitk = desc->max_tokens > 2 ? (float*)(sb + L.off_splitk) : nullptr;
   s->stamps = (unsigned long long*)(sb + L.off_stamps);
-  s->ssq = (float*)(sb + L.off_ssq);
-  s->unit_cnt = (int*)(sb + L.off_unitcnt);
   s->ctx.assign(desc->max_slots, -1);
 
   auto bail = [&](es_status_t st) { delete s; return st; };
@@ -726,7 +672,6 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
     if (e == cudaSuccess) e = cudaMemcpyAsync(s->block_table, table.data(), table.size() * 4, cudaMemcpyHostToDevice, s->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->ctx_len, 0, (size_t)desc->max_slots * 4, s->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->status, 0, 256, s->stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(s->unit_cnt, 0, L.unit_cnt_bytes, s->stream);
     if (e == cudaSuccess)       // arrival counters of the decode-attention splits (they follow the partials)
       e = cudaMemsetAsync(s->part, 0, decode_attention_scratch_bytes((int)desc->max_batch, desc->n_heads, desc->head_dim, L.n_splits), s->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->kv, 0, L.kv_bytes, s->stream);
@@ -1116,14 +1061,8 @@ es_status_t es_op_linear(const void* A, const void* W, const float* R, float* C,
   }
 }
 
-// K-sliced streaming kernel (3..16 rows): partial sums per 16-row unit, then one arrival counter per unit
-static size_t skinny_counter_offset(int32_t M, int32_t N, int32_t k_splits) {
-  return align_up(linear_stream_mma_workspace_bytes(M, N, EPI_F32, k_splits));
-}
-
 size_t es_op_linear_splitk_workspace_bytes(int32_t M, int32_t N, int32_t k_splits) {
   if (M <= 0 || N <= 0 || k_splits <= 0) return 0;
-  if (M <= 16) return skinny_counter_offset(M, N, k_splits) + align_up((size_t)((N + 15) / 16) * sizeof(int));
   return (size_t)k_splits * M * N * sizeof(float);
 }
 
@@ -1139,11 +1078,7 @@ es_status_t es_op_linear_splitk(const void* A, const void* W, const float* R, fl
   if (skinny) {
     if (M < 3 || !linear_stream_mma_supported(p, EPI_F32))
       return fail(ES_ERR_UNSUPPORTED, "K-sliced streaming kernel takes 3..16 rows and K a multiple of 256");
-    if (k_splits == 0) {
-      // the most slices whose partial sums and counters fit the given workspace
-      const size_t counters = align_up((size_t)((N + 15) / 16) * sizeof(int)) + ALIGN;
-      k_splits = linear_stream_mma_splits(p, EPI_F32, (workspace && workspace_bytes > counters) ? workspace_bytes - counters : 0);
-    }
+    if (k_splits == 0) k_splits = linear_stream_mma_splits(p, EPI_F32, workspace ? workspace_bytes : 0);
   } else {
     if (!linear_tc_supported(p, EPI_F32)) return fail(ES_ERR_UNSUPPORTED, "tensor-core kernel does not take this shape");
     p.split_on_pairs = (M >= 256 && tunables().tc_pair && tunables().split_pairs) ? 1 : 0;   // 256 or more rows: slices on CTA pairs
@@ -1161,10 +1096,8 @@ es_status_t es_op_linear_splitk(const void* A, const void* W, const float* R, fl
   if ((uintptr_t)workspace % 16) return fail(ES_ERR_INVALID_ARG, "workspace must be 16-byte aligned");
   p.k_splits = k_splits; p.part = (float*)workspace;
   if (skinny) {
-    // the kernel adds the slices itself: the last warp to deliver a unit's partial sums finishes the unit
-    p.unit_cnt = (int*)((unsigned char*)workspace + skinny_counter_offset(M, N, k_splits));
-    ES_CUDA_CHECK(cudaMemsetAsync(p.unit_cnt, 0, (size_t)((N + 15) / 16) * sizeof(int), st));
-    return launch_linear_stream_mma(p, EPI_F32, st, nullptr);
+    ES_TRY(launch_linear_stream_mma(p, EPI_F32, st, nullptr));
+    return launch_splitk_reduce(p.part, k_splits, R, C, M, N, N, nullptr, nullptr, 0.f, st, nullptr);
   }
   p.k_splits = k_splits; p.part = (float*)workspace;
   if (p.split_on_pairs) ES_TRY(launch_linear_tc2(p, EPI_F32, st, nullptr, nullptr));

@@ -93,13 +93,13 @@ def test_split_point_equals_single_shard(B, tiny, k):
 
 @pytest.mark.parametrize("d,Hq,Hkv,F,Bn", [(512, 8, 4, 1536, 5), (512, 8, 4, 1536, 12), (4096, 32, 32, 11008, 8), (4096, 32, 32, 11008, 16),
                                             (8192, 64, 8, 4096, 16)])
-def test_decode_of_several_sequences_with_fused_norm_and_sliced_products(B, d, Hq, Hkv, F, Bn):
+def test_decode_of_several_sequences_on_tensor_core_streaming_shapes(B, d, Hq, Hkv, F, Bn):
     """Decode steps of 3..16 sequences on layer shapes where the tensor-core streaming kernels take every product:
-    the RMSNorm runs inside the QKV and gate / up kernels from sums of squares written by the O and down
-    epilogues, and products whose activations do not fit in shared memory are cut along K across CTAs and
-    finished by the last warp to deliver a unit.  Checked against the oracle at every step, for the split
-    [0,1) -> [1,3) == [0,3) bit for bit (a shard that receives its rows from another shard computes the sums of
-    squares with its own kernel), and for repeatability (the finishing order is fixed)."""
+    whole-K products with the activations in shared memory, and products whose activations do not fit, which are
+    cut along K across CTAs and finished by a second kernel (slices added in slice order, RMSNorm for the next
+    product fused into the reduction).  Checked against the oracle at every step, for the split
+    [0,1) -> [1,3) == [0,3) bit for bit (a shard that receives its rows from another shard normalises them with
+    the stand-alone kernel), and for repeatability."""
     from workload import ModelShape, shard_weights
     hd = 64 if d == 512 else 128
     m = ModelShape("mid", 3, d, Hq, Hkv, hd, F, 512)
