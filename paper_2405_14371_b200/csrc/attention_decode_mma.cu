@@ -237,7 +237,7 @@ __global__ void __launch_bounds__(MW * 32, DB ? 2 : 3) decode_attn_mma_kernel(co
       if (c == 0) { dst[HD] = mm; dst[HD + 1] = ll; }
     }
   }
-  if (p.n_splits > 1) merge_splits_if_last<HD, G>(p, b, kvh, ctx, &s_last);
+  if (p.n_splits > 1 && p.merge_in_kernel) merge_splits_if_last<HD, G>(p, b, kvh, ctx, &s_last);
   stamp_end(p.stamp);
 }
 
@@ -259,7 +259,8 @@ bool decode_attention_mma_supported(const DecodeAttnParams& p) {
   return true;
 }
 
-// Like the CUDA-core kernel, the kernel merges its own splits (the last CTA to arrive for a (sequence, KV head)).
+// The split kernel only; with p.merge_in_kernel the last CTA to arrive for a (sequence, KV head) merges the splits,
+// otherwise the caller launches the merge kernel.
 es_status_t launch_decode_attention_mma(const DecodeAttnParams& p, cudaStream_t s, bool pdl) {
   if (!decode_attention_mma_supported(p)) return fail(ES_ERR_UNSUPPORTED, "tensor-core decode attention does not take this layout");
   switch (p.Hq / p.Hkv) {

@@ -37,6 +37,10 @@ struct Tunables {
   int attn_mma;      // ES_ATTN_MMA: tensor-core decode attention for launches with many items (1, default) or never (0)
   int split_k;       // ES_SPLIT_K: split-K for the O and down projections of short prefills (1, default) or never (0)
   int ks_min_slice;        // ES_KS_MIN_SLICE: smallest K slice of the K-sliced streaming kernel (elements, default 512)
+  int ks_splits;           // ES_KS_SPLITS: K slices of the K-sliced streaming kernel (0 = chosen per shape; a value that does not fit is ignored)
+  int ks_cols;             // ES_KS_COLS: column ranges per K slice of that kernel (0 = chosen per shape)
+  int attn_split_tokens;   // ES_ATTN_SPLIT_TOKENS: smallest split of a decode-attention context (tokens; 0 = 256, or 384 for groups of 4-8 query heads)
+  int even_grid;           // ES_EVEN_GRID: weight-streaming kernels shrink their grid so that every CTA (warp) gets the same number of units (1) or fill the machine (0)
 };
 const Tunables& tunables();
 
@@ -197,6 +201,7 @@ struct DecodeAttnParams {
                           // (sequence, KV head), zero before the launch and zero again after it
   int B, Hq, Hkv, hd;
   int n_splits, pages_per_split;
+  int merge_in_kernel;    // set by launch_decode_attention: the last split CTA to arrive merges (else a merge launch)
   unsigned long long* stamp;   // optional time stamps of the launch (split and merge kernels share them), nullptr = none
 };
 size_t decode_attention_scratch_bytes(int B, int Hq, int hd, int n_splits);

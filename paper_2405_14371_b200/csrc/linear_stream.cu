@@ -300,6 +300,10 @@ es_status_t launch_inst(const LinearParams& p, cudaStream_t s, bool pdl) {
   int grid = sms * per_sm;
   const int max_useful = (n_units + WARPS - 1) / WARPS;
   if (grid > max_useful) grid = max_useful;
+  if (tunables().even_grid) {
+    const int per_warp = (n_units + grid * WARPS - 1) / (grid * WARPS);   // the same number of units for every warp
+    grid = (n_units + per_warp * WARPS - 1) / (per_warp * WARPS);
+  }
   ES_CUDA_CHECK(launch_kernel(kern, dim3(grid), dim3(THREADS), smem, s, pdl, p));
   return ES_OK;
 }

@@ -403,6 +403,8 @@ __global__ void __launch_bounds__(256) splitk_finish_kernel(const LinearParams p
   stamp_end(p.stamp);
 }
 
+int ks_col_ctas(int ks);   // defined with the host-side planning below
+
 template <int NT, int EPI>
 es_status_t launch_ks(const LinearParams& p, cudaStream_t s, bool pdl) {
   auto kern = linear_stream_mma_ks_kernel<NT, EPI>;
@@ -414,7 +416,7 @@ es_status_t launch_ks(const LinearParams& p, cudaStream_t s, bool pdl) {
     ES_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured = smem;
   }
-  const int n_col_ctas = KS_GRID / p.k_splits;
+  const int n_col_ctas = ks_col_ctas(p.k_splits);
   ES_CUDA_CHECK(launch_kernel(kern, dim3(n_col_ctas * p.k_splits), dim3(MTHREADS), smem, s, pdl, p, a_stride, n_col_ctas));
   return ES_OK;
 }
@@ -442,6 +444,10 @@ es_status_t launch_inst(const LinearParams& p, cudaStream_t s, bool pdl) {
   const int n_units = (p.N + COLS - 1) / COLS;
   int grid = sms * per_sm;
   if (grid > n_units) grid = n_units;
+  if (tunables().even_grid) {
+    const int per_cta = (n_units + grid - 1) / grid;       // the same number of units for every CTA
+    grid = (n_units + per_cta - 1) / per_cta;
+  }
   ES_CUDA_CHECK(launch_kernel(kern, dim3(grid), dim3(MTHREADS), smem, s, pdl, p, a_stride));
   return ES_OK;
 }
@@ -474,6 +480,17 @@ bool linear_stream_mma_supported(const LinearParams& p, int epi) {
   return true;
 }
 
+namespace {
+
+// Column ranges per K slice: as many as fill the machine (two CTAs per SM).  Fewer, evenly loaded CTAs were
+// measured and lost at every shape of the 70B layer (e.g. gate / up 163 -> 175 us with 64 instead of 74 ranges).
+int ks_col_ctas(int ks) {
+  const int hi = KS_GRID / ks;
+  return (tunables().ks_cols > 0 && tunables().ks_cols <= hi) ? tunables().ks_cols : hi;
+}
+
+}  // namespace
+
 int linear_stream_mma_splits(const LinearParams& p, int epi, size_t workspace_bytes) {
   if (!linear_stream_mma_supported(p, epi) || p.M < 3) return 1;
   const int nt = p.M <= 8 ? 1 : 2;
@@ -482,6 +499,8 @@ int linear_stream_mma_splits(const LinearParams& p, int epi, size_t workspace_by
   const int cols = (epi == EPI_SWIGLU) ? 8 : 16;
   const int n_units = (p.N + cols - 1) / cols;
   const size_t part_cols = (epi == EPI_SWIGLU) ? 2 * (size_t)p.N : (size_t)p.N;
+  // The slice count that minimises the K elements the busiest warp walks.  Measured on the 70B layer at 16 rows
+  // (in-step, normalised): QKV 16 slices 32 us, 8 slices 35, 4 slices 40; down 16 slices 83 us, 14 slices 86.
   int best = 1;
   long long best_cost = 0;
   for (int ks = 2; ks <= 64 && ks <= KS_GRID; ++ks) {
@@ -490,6 +509,7 @@ int linear_stream_mma_splits(const LinearParams& p, int epi, size_t workspace_by
     if (kslice < tunables().ks_min_slice) break;
     if ((size_t)nt * 8 * (kslice + 8) * sizeof(__half) > KS_SMEM_MAX) continue;
     if ((size_t)ks * p.M * part_cols * sizeof(float) > workspace_bytes) continue;
+    if (tunables().ks_splits == ks) return ks;
     const int ncol = KS_GRID / ks;
     const int units_per_cta = (n_units + ncol - 1) / ncol;
     const long long cost = (long long)((units_per_cta + MW - 1) / MW) * kslice;   // K elements the busiest warp walks

@@ -41,7 +41,22 @@ static int env_int(const char* name, int dflt) {
 }
 
 const Tunables& tunables() {
-  static const Tunables t = {env_int("ES_STREAM_DEEP", 1), env_int("ES_TC_PAIR", 1), env_int("ES_TC_PAIR_WIDE", 1), env_int("ES_SPLIT_PAIRS", 1), env_int("ES_PDL", 1), env_int("ES_ATTN_MMA", 1), env_int("ES_SPLIT_K", 1), env_int("ES_KS_MIN_SLICE", 512)};
+  static const Tunables t = [] {
+    Tunables v;
+    v.stream_deep = env_int("ES_STREAM_DEEP", 1);
+    v.tc_pair = env_int("ES_TC_PAIR", 1);
+    v.tc_pair_wide = env_int("ES_TC_PAIR_WIDE", 1);
+    v.split_pairs = env_int("ES_SPLIT_PAIRS", 1);
+    v.pdl = env_int("ES_PDL", 1);
+    v.attn_mma = env_int("ES_ATTN_MMA", 1);
+    v.split_k = env_int("ES_SPLIT_K", 1);
+    v.ks_min_slice = env_int("ES_KS_MIN_SLICE", 512);
+    v.ks_splits = env_int("ES_KS_SPLITS", 0);
+    v.ks_cols = env_int("ES_KS_COLS", 0);
+    v.attn_split_tokens = env_int("ES_ATTN_SPLIT_TOKENS", 0);
+    v.even_grid = env_int("ES_EVEN_GRID", 0);
+    return v;
+  }();
   return t;
 }
 
@@ -54,7 +69,7 @@ void choose_splits(int max_ctx, int P, int B, int Hkv, int group, int* n_splits,
   const int ctas = (group >= 4 ? 4 : 1) * 148;
   long long pps = (long long)pages * B * Hkv / ctas;
   // at least 256 tokens per split (384 for large groups, whose CTAs carry more fixed work per split)
-  const int min_tokens = group >= 4 ? 384 : 256;
+  const int min_tokens = tunables().attn_split_tokens > 0 ? tunables().attn_split_tokens : (group >= 4 ? 384 : 256);
   const int min_pps = min_tokens / P > 1 ? min_tokens / P : 1;
   if (pps < min_pps) pps = min_pps;
   if (pps > pages) pps = pages;
