@@ -180,7 +180,14 @@ ES_API es_status_t es_shard_set_page_table(es_shard_t *shard, const int32_t *tab
 ES_API es_status_t es_shard_set_graphs(es_shard_t *shard, int32_t enabled);
 
 /* Reads the device status word (synchronises): ES_OK, or ES_ERR_DEVICE_TIMEOUT if a bounded wait
- * inside a kernel ran out since the last call. */
+ * inside a kernel ran out since the last call.
+ * Checking mode: with ES_DEBUG=1 in the environment of the process (read once), the call also verifies
+ * that the 256 guard bytes the library keeps behind every region it carves out of the scratch buffer are
+ * intact (a kernel that wrote past its region lands there first) and that the tables the kernels index
+ * with hold values inside their ranges (page numbers, context lengths against the host's own count, the
+ * uploaded slot list); a violation is ES_ERR_STATE with the region or entry named in es_last_error.  In
+ * this mode every prefill / decode call first synchronises and runs the same checks on what the previous
+ * pass left behind (so it is for testing, not for timing). */
 ES_API es_status_t es_shard_device_status(es_shard_t *shard);
 
 /* Exercises the time-out path above without any kernel misbehaving: enqueues a one-CTA kernel built like the

@@ -350,9 +350,14 @@ cudaError_t launch_row_clusters(void (*kernel)(KArgs...), int M, cudaStream_t st
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// rows for which the cluster kernels are used: few enough that one CTA per row would leave most SMs idle
+// Where the cluster kernels are used: few rows (one CTA per row would leave most SMs idle) that are long (the
+// slices of a wide product are what one SM cannot pull in fast enough).  Measured per layer, in a replayed step:
+// 16 rows of 8192 columns, 16 slices: 17.3 -> 12.8 us for the two reductions; 8 rows of 4096 columns: 7.1 -> 8.5 us
+// (the cluster launch costs more than it saves), hence the width threshold.  The rule depends on the shape only,
+// never on the slice count, so the reduction and the stand-alone kernel always agree on it.
 constexpr int ROW_CLUSTER_MAX_ROWS = 16;
-inline bool use_row_clusters(int M, int N) { return M <= ROW_CLUSTER_MAX_ROWS && N % (4 * ROW_CTAS) == 0; }
+constexpr int ROW_CLUSTER_MIN_COLS = 8192;
+inline bool use_row_clusters(int M, int N) { return M <= ROW_CLUSTER_MAX_ROWS && N >= ROW_CLUSTER_MIN_COLS && N % (4 * ROW_CTAS) == 0; }
 
 // Greedy token: index of the largest logit, the lowest index on ties.  One CTA per sequence.
 __global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ logits, int* __restrict__ out, int V,

@@ -40,6 +40,7 @@ struct Tunables {
   int ks_splits;           // ES_KS_SPLITS: K slices of the K-sliced streaming kernel (0 = chosen per shape; a value that does not fit is ignored)
   int ks_cols;             // ES_KS_COLS: column ranges per K slice of that kernel (0 = chosen per shape)
   int attn_split_tokens;   // ES_ATTN_SPLIT_TOKENS: smallest split of a decode-attention context (tokens; 0 = 256, or 384 for groups of 4-8 query heads)
+  int debug_checks;        // ES_DEBUG: es_shard_device_status also verifies the guard bytes behind every scratch region and the ranges of the page table, context lengths and slot list (1) or not (0, default)
   int even_grid;           // ES_EVEN_GRID: weight-streaming kernels shrink their grid so that every CTA (warp) gets the same number of units (1) or fill the machine (0)
 };
 const Tunables& tunables();

@@ -55,6 +55,7 @@ const Tunables& tunables() {
     v.ks_cols = env_int("ES_KS_COLS", 0);
     v.attn_split_tokens = env_int("ES_ATTN_SPLIT_TOKENS", 0);
     v.even_grid = env_int("ES_EVEN_GRID", 0);
+    v.debug_checks = env_int("ES_DEBUG", 0);
     return v;
   }();
   return t;
@@ -80,6 +81,8 @@ void choose_splits(int max_ctx, int P, int B, int Hkv, int group, int* n_splits,
 namespace {
 
 constexpr size_t ALIGN = 256;
+constexpr size_t CANARY_BYTES = 256;
+constexpr unsigned char CANARY = 0xC5;
 inline size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
@@ -89,6 +92,8 @@ struct Layout {
   size_t off_x, off_h, off_q, off_ao, off_act, off_logits, off_next, off_hlast, off_part, off_cos, off_sin,
       off_table, off_ctx, off_slots, off_status, off_splitk, off_stamps;
   size_t scratch_bytes;
+  // every carved region is followed by CANARY_BYTES that no kernel may touch: (offset of the guard, region name)
+  std::vector<std::pair<size_t, const char*>> guards;
 };
 
 es_status_t validate_desc(const es_model_desc_t* d, int begin, int end) {
@@ -124,24 +129,30 @@ Layout make_layout(const es_model_desc_t& d, int begin, int end) {
   const size_t M = d.max_tokens, B = d.max_batch, nq = (size_t)d.n_heads * d.head_dim;
   const bool head = end == d.n_layers_total;
   size_t o = 0;
-  auto take = [&](size_t bytes) { size_t at = o; o += align_up(bytes); return at; };
-  L.off_x = take(M * d.d_model * 4);
-  L.off_h = take(M * d.d_model * 2);
-  L.off_q = take(M * nq * 2);
-  L.off_ao = take(M * nq * 2);
-  L.off_act = take(M * (size_t)d.d_ffn * 2);
-  L.off_logits = take(head ? B * (size_t)d.vocab * 4 : 0);
-  L.off_next = take(B * 4);
-  L.off_hlast = take(B * (size_t)d.d_model * 2);
-  L.off_part = take(decode_attention_scratch_bytes((int)B, d.n_heads, d.head_dim, L.n_splits));
-  L.off_cos = take((size_t)d.max_seq * (d.head_dim / 2) * 4);
-  L.off_sin = take((size_t)d.max_seq * (d.head_dim / 2) * 4);
-  L.off_table = take((size_t)L.n_pages * 4);
-  L.off_ctx = take((size_t)d.max_slots * 4);
-  L.off_slots = take(2 * B * 4);       // slots, then the prompt lengths of a ragged prefill
-  L.off_status = take(256);
-  L.off_splitk = take(d.max_tokens > 2 ? linear_tc_split_workspace_bytes() : 0);   // split-K partial sums of short prefills
-  L.off_stamps = take((size_t)2 * STAMP_SLOTS * sizeof(unsigned long long));
+  auto take = [&](size_t bytes, const char* name) {
+    size_t at = o;
+    o += align_up(bytes);
+    L.guards.emplace_back(o, name);
+    o += CANARY_BYTES;
+    return at;
+  };
+  L.off_x = take(M * d.d_model * 4, "residual stream");
+  L.off_h = take(M * d.d_model * 2, "normalised activations");
+  L.off_q = take(M * nq * 2, "q");
+  L.off_ao = take(M * nq * 2, "attention output");
+  L.off_act = take(M * (size_t)d.d_ffn * 2, "ffn activations");
+  L.off_logits = take(head ? B * (size_t)d.vocab * 4 : 0, "logits");
+  L.off_next = take(B * 4, "next ids");
+  L.off_hlast = take(B * (size_t)d.d_model * 2, "last-row norm");
+  L.off_part = take(decode_attention_scratch_bytes((int)B, d.n_heads, d.head_dim, L.n_splits), "attention partials");
+  L.off_cos = take((size_t)d.max_seq * (d.head_dim / 2) * 4, "rope cos");
+  L.off_sin = take((size_t)d.max_seq * (d.head_dim / 2) * 4, "rope sin");
+  L.off_table = take((size_t)L.n_pages * 4, "page table");
+  L.off_ctx = take((size_t)d.max_slots * 4, "context lengths");
+  L.off_slots = take(2 * B * 4, "slots");       // slots, then the prompt lengths of a ragged prefill
+  L.off_status = take(256, "status words");
+  L.off_splitk = take(d.max_tokens > 2 ? linear_tc_split_workspace_bytes() : 0, "split-K workspace");   // split-K partial sums of short prefills
+  L.off_stamps = take((size_t)2 * STAMP_SLOTS * sizeof(unsigned long long), "time stamps");
   L.scratch_bytes = o;
   return L;
 }
@@ -589,6 +600,40 @@ es_status_t check_inputs(const es_shard* s, const int32_t* ids, const es_tensor_
   return ES_OK;
 }
 
+// The checking mode (ES_DEBUG=1): the guard bytes behind every carved region of the scratch buffer must be intact
+// (a kernel that wrote past its region lands there first), and the tables the kernels index with must hold values
+// inside their ranges: page numbers, context lengths, the uploaded slot list.  Reads device memory; synchronises.
+es_status_t debug_checks(es_shard* s) {
+  std::vector<unsigned char> g(CANARY_BYTES);
+  for (const auto& gd : s->lay.guards) {
+    ES_CUDA_CHECK(cudaMemcpy(g.data(), s->scratch + gd.first, CANARY_BYTES, cudaMemcpyDeviceToHost));
+    for (size_t i = 0; i < CANARY_BYTES; ++i)
+      if (g[i] != CANARY) return fail(ES_ERR_STATE, "debug check: the guard behind '%s' was overwritten at byte %zu", gd.second, i);
+  }
+  std::vector<int> table(s->lay.n_pages), ctx(s->d.max_slots);
+  ES_CUDA_CHECK(cudaMemcpy(table.data(), s->block_table, table.size() * 4, cudaMemcpyDeviceToHost));
+  ES_CUDA_CHECK(cudaMemcpy(ctx.data(), s->ctx_len, ctx.size() * 4, cudaMemcpyDeviceToHost));
+  for (int i = 0; i < s->lay.n_pages; ++i)
+    if (table[i] < 0 || table[i] >= s->lay.n_pages) return fail(ES_ERR_STATE, "debug check: page table entry %d = %d", i, table[i]);
+  for (int i = 0; i < s->d.max_slots; ++i) {
+    if (ctx[i] < 0 || ctx[i] > s->d.max_seq) return fail(ES_ERR_STATE, "debug check: context length of slot %d = %d", i, ctx[i]);
+    if (s->ctx[i] >= 0 && ctx[i] != s->ctx[i])
+      return fail(ES_ERR_STATE, "debug check: slot %d holds %d positions on the device, %d on the host", i, ctx[i], s->ctx[i]);
+  }
+  if (!s->slots_host.empty()) {
+    std::vector<int> sl(s->slots_host.size());
+    ES_CUDA_CHECK(cudaMemcpy(sl.data(), s->slots_dev, sl.size() * 4, cudaMemcpyDeviceToHost));
+    for (size_t i = 0; i < sl.size(); ++i)
+      if (sl[i] != s->slots_host[i]) return fail(ES_ERR_STATE, "debug check: uploaded slot %zu = %d, expected %d", i, sl[i], s->slots_host[i]);
+  }
+  return ES_OK;
+}
+
+es_status_t debug_checks_now(es_shard* s) {
+  ES_CUDA_CHECK(cudaStreamSynchronize(s->stream));
+  return debug_checks(s);
+}
+
 }  // namespace
 }  // namespace es
 
@@ -687,6 +732,8 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
     if (e == cudaSuccess) e = cudaMemcpyAsync(s->block_table, table.data(), table.size() * 4, cudaMemcpyHostToDevice, s->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->ctx_len, 0, (size_t)desc->max_slots * 4, s->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->status, 0, 256, s->stream);
+    for (const auto& g : L.guards)
+      if (e == cudaSuccess) e = cudaMemsetAsync(sb + g.first, CANARY, CANARY_BYTES, s->stream);
     if (e == cudaSuccess)       // arrival counters of the decode-attention splits (they follow the partials)
       e = cudaMemsetAsync(s->part, 0, decode_attention_scratch_bytes((int)desc->max_batch, desc->n_heads, desc->head_dim, L.n_splits), s->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->kv, 0, L.kv_bytes, s->stream);
@@ -757,6 +804,7 @@ es_status_t es_shard_prefill(es_shard_t* s, const int32_t* ids, const es_tensor_
   const float* hin;
   ES_TRY(check_inputs(s, ids, hidden_in, (int64_t)B * T, &hin));
   if (s->profiling) ES_TRY(harvest_profile(s));
+  if (tunables().debug_checks) ES_TRY(debug_checks_now(s));    // checking mode: what the previous pass left behind
   ES_TRY(upload_slots(s, slots, B));
   s->last_valid = false;
   ES_TRY(enqueue_pass(s, ids, hin, B, T, false));
@@ -780,6 +828,7 @@ es_status_t es_shard_prefill_ragged(es_shard_t* s, const int32_t* ids, const es_
   const float* hin;
   ES_TRY(check_inputs(s, ids, hidden_in, (int64_t)B * T, &hin));
   if (s->profiling) ES_TRY(harvest_profile(s));
+  if (tunables().debug_checks) ES_TRY(debug_checks_now(s));    // checking mode: what the previous pass left behind
   ES_TRY(upload_slots(s, slots, B));
   s->lens_host.assign(lens, lens + B);
   ES_CUDA_CHECK(cudaMemcpyAsync(s->lens_dev, s->lens_host.data(), B * sizeof(int), cudaMemcpyHostToDevice, s->stream));
@@ -805,6 +854,7 @@ es_status_t es_shard_decode_step(es_shard_t* s, const int32_t* ids, const es_ten
   const float* hin;
   ES_TRY(check_inputs(s, ids, hidden_in, B, &hin));
   if (s->profiling) ES_TRY(harvest_profile(s));
+  if (tunables().debug_checks) ES_TRY(debug_checks_now(s));    // checking mode: what the previous pass left behind
   ES_TRY(upload_slots(s, slots, B));
   s->last_valid = false;
 
@@ -945,6 +995,7 @@ es_status_t es_shard_device_status(es_shard_t* s) {
     cudaMemset(s->status, 0, 256);
     return fail(ES_ERR_DEVICE_TIMEOUT, "a device-side wait ran out (code %d, detail %d)", host[0], host[1]);
   }
+  if (tunables().debug_checks) ES_TRY(debug_checks(s));
   return ES_OK;
 }
 

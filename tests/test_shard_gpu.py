@@ -512,6 +512,22 @@ def test_a_device_wait_that_runs_out_is_reported_and_the_shard_stays_usable(B, t
     sh.close()
 
 
+def test_checking_mode_passes_over_the_tiny_configuration():
+    """ES_DEBUG=1 (read once per process, hence a child process): after every pass of the tiny-configuration
+    tests the status call also verifies the guard bytes behind each scratch region and the ranges of the page
+    table, context lengths and slot list.  All of those tests must still pass, i.e. no kernel writes outside its
+    region and the device-side counters follow the host's."""
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, ES_DEBUG="1")
+    sel = "cfg0_greedy or split_point or batch_rows or page_map or edge_shapes or ragged or micro_batch"
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_shard_gpu.py"), "-m", "gpu", "-q", "-x",
+                        "-k", sel, "-p", "no:cacheprovider"], cwd=root, env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
+    assert " passed" in r.stdout
+
+
 def test_error_paths_launch_nothing(B, tiny):
     wd, _ = tiny
     ids = prompt_ids(0, 1, 8, TINY.vocab).cuda()
