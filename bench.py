@@ -41,7 +41,11 @@ DEFAULT_ALSO = "cfg1,cfg2_b1,cfg2_b8,cfg3"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant decode kernel (average over the four
 # products of a layer), from the ncu captures summarised under profiles/; an entry is None when that kernel
 # has changed since its counters were taken.
-TRAFFIC_PER_LAUNCH = {"cfg1": 105.0e6}
+TRAFFIC_PER_LAUNCH = {
+    "cfg1": 103.7e6,      # profiles/linear_stream_kernel_cfg1_decode.md (same workload)
+    "cfg4": 434.2e6,      # profiles/decode_kernels_cfg4_shapes_batch16_2layers.md: the four products of a layer, whose
+                          # launches are the same in the 2-layer capture case and in the 40-layer workload
+}
 
 
 def _peaks() -> dict:
@@ -325,9 +329,12 @@ def run_ours(args, name: str, steps: int, warmup: int, dist_ctx, with_clocks: bo
             pre_stamps = in_step_breakdown(sh.es_shard_step_timing())
             src = sh.es_shard_handoff()[2] if (wl.has_head and n_sh == 1) else cur_ids[0]
             dec_breaks = []
-            for i in range(min(6, S)):
+            n_probe = min(40, S)
+            for i in range(n_probe):
                 sh.es_shard_decode_step(src, None, Bn, slots[0])
-                if i >= 2:                      # the first steps capture and upload the graph
+                # the first steps capture and upload the graph, and steps right behind a long prefill run at the low
+                # clock the prefill left: the last few of a run of steps are read
+                if i >= max(2, n_probe - 6):
                     dec_breaks.append(in_step_breakdown(sh.es_shard_step_timing()))
             sh.es_shard_set_step_timing(False)
         for x in shards:
@@ -441,9 +448,9 @@ def cpu_oracle_sample(wl, threads=None, layers=None, decode_steps=2):
         torch.set_num_threads(threads)
     nl_all = wl.layer_end - wl.layer_begin
     if layers is None:
-        # about 0.2 TFLOP of matrix-form prefill per sample keeps one sample to a few seconds of host time
+        # about 10 TFLOP of matrix-form prefill per sample: ten to twenty seconds of host time with the decode steps
         per_layer = 2.0 * wl.prompt_len * m.layer_params()
-        layers = max(1, min(nl_all, int(0.4e12 / per_layer)))
+        layers = max(1, min(nl_all, int(1.0e13 / per_layer)))
     gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
     host = {"layers": [{k: v.cpu() for k, v in layer_weights(wl.cfg, m, wl.layer_begin + i, gen_dev).items()} for i in range(layers)]}
     if wl.has_embedding:
