@@ -243,7 +243,7 @@ __global__ void __launch_bounds__(HD) decode_attn_merge_kernel(const DecodeAttnP
 
 template <int HD, int G>
 es_status_t launch_g(const DecodeAttnParams& p, cudaStream_t s, bool pdl) {
-  const bool small = (long long)p.n_splits * p.Hkv * p.B <= 2 * 148;
+  const bool small = (long long)p.n_splits * p.Hkv * p.B <= 2 * sm_count();
   if (small)
     ES_CUDA_CHECK(launch_kernel(decode_attn_split_kernel<HD, G, true>, dim3(p.n_splits, p.Hkv, p.B), dim3(DWARPS * 32), 0, s, pdl, p));
   else
@@ -299,7 +299,7 @@ es_status_t launch_decode_attention(const DecodeAttnParams& p0, cudaStream_t s, 
   // 512..768 keys).  A large launch merges faster with a kernel of its own, one CTA per head (16 sequences x 8 KV
   // heads x 3 splits: 30 us against 40 us per layer with the merge in the split kernel's tail).
   DecodeAttnParams p = p0;
-  p.merge_in_kernel = (long long)p.n_splits * p.Hkv * p.B <= 2 * 148 ? 1 : 0;
+  p.merge_in_kernel = (long long)p.n_splits * p.Hkv * p.B <= 2 * sm_count() ? 1 : 0;
   if (p.hd == 128) return launch_hd<128>(p, s, pdl, launches);
   if (p.hd == 64) return launch_hd<64>(p, s, pdl, launches);
   return fail(ES_ERR_SHAPE, "head_dim must be 64 or 128, got %d", p.hd);

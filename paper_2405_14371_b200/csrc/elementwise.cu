@@ -148,11 +148,30 @@ __global__ void __launch_bounds__(THREADS) splitk_reduce_kernel(const float* __r
     const int c = threadIdx.x + i * THREADS;
     v[i] = (rs && c < n4) ? rs[c] : make_float4(0.f, 0.f, 0.f, 0.f);
   }
+  // The slices of ALL of a thread's register-resident columns are requested four slices at a time before anything
+  // is added or stored (one memory round trip per four slices instead of one per column); every element is still
+  // residual + slice 0 + slice 1 + ... in that order.
+  constexpr int SB = 4;
+  for (int s0 = 0; s0 < k_splits; s0 += SB) {
+    float4 t[REGS][SB];
+#pragma unroll
+    for (int i = 0; i < REGS; ++i) {
+      const int c = threadIdx.x + i * THREADS;
+#pragma unroll
+      for (int j = 0; j < SB; ++j)
+        t[i][j] = (c < n4 && s0 + j < k_splits) ? __ldcs(src + (s0 + j) * slice4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int i = 0; i < REGS; ++i)
+#pragma unroll
+      for (int j = 0; j < SB; ++j)
+        if (s0 + j < k_splits) { v[i].x += t[i][j].x; v[i].y += t[i][j].y; v[i].z += t[i][j].z; v[i].w += t[i][j].w; }
+  }
 #pragma unroll
   for (int i = 0; i < REGS; ++i) {
     const int c = threadIdx.x + i * THREADS;
     if (c < n4) {
-      v[i] = finish(c, v[i]);
+      dst[c] = v[i];
       ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
     }
   }

@@ -45,6 +45,10 @@ struct Tunables {
 };
 const Tunables& tunables();
 
+// Number of SMs of the current device (148 on a B200; 0 if the query fails, which callers treat as 1).  Every
+// grid size, wave count and split rule below is written in terms of it.
+int sm_count();
+
 // ---- the linear layer family ----------------------------------------------------------------
 // C[m, n] = sum_k A[m, k] * W[n, k], A fp16 [M, K] row-major (row stride lda), W fp16 row-major
 // [*, K].  The N output columns are a concatenation of up to three weight matrices ("segments",

@@ -29,7 +29,7 @@ constexpr int MW = 8;                 // warps per CTA
 constexpr int MTHREADS = MW * 32;
 constexpr int KSTEP = 32;             // K elements per lane-load step
 constexpr int UM_TOTAL = 4;           // lane-load steps per chunk over all row groups of a warp
-constexpr int KS_GRID = 296;          // CTAs of the K-sliced kernel: two per SM
+inline int ks_grid() { return 2 * sm_count(); }   // CTAs of the K-sliced kernel: two per SM
 constexpr size_t KS_SMEM_MAX = 100 * 1024;   // activation slice per CTA (two CTAs per SM)
 
 __device__ __forceinline__ uint4 ld_stream16(const void* ptr) {
@@ -485,7 +485,7 @@ namespace {
 // Column ranges per K slice: as many as fill the machine (two CTAs per SM).  Fewer, evenly loaded CTAs were
 // measured and lost at every shape of the 70B layer (e.g. gate / up 163 -> 175 us with 64 instead of 74 ranges).
 int ks_col_ctas(int ks) {
-  const int hi = KS_GRID / ks;
+  const int hi = ks_grid() / ks;
   return (tunables().ks_cols > 0 && tunables().ks_cols <= hi) ? tunables().ks_cols : hi;
 }
 
@@ -503,14 +503,15 @@ int linear_stream_mma_splits(const LinearParams& p, int epi, size_t workspace_by
   // (in-step, normalised): QKV 16 slices 32 us, 8 slices 35, 4 slices 40; down 16 slices 83 us, 14 slices 86.
   int best = 1;
   long long best_cost = 0;
-  for (int ks = 2; ks <= 64 && ks <= KS_GRID; ++ks) {
+  const int grid_max = ks_grid();
+  for (int ks = 2; ks <= 64 && ks <= grid_max; ++ks) {
     if (steps % ks) continue;
     const int kslice = p.K / ks;
     if (kslice < tunables().ks_min_slice) break;
     if ((size_t)nt * 8 * (kslice + 8) * sizeof(__half) > KS_SMEM_MAX) continue;
     if ((size_t)ks * p.M * part_cols * sizeof(float) > workspace_bytes) continue;
     if (tunables().ks_splits == ks) return ks;
-    const int ncol = KS_GRID / ks;
+    const int ncol = grid_max / ks;
     const int units_per_cta = (n_units + ncol - 1) / ncol;
     const long long cost = (long long)((units_per_cta + MW - 1) / MW) * kslice;   // K elements the busiest warp walks
     if (best == 1 || cost < best_cost) { best = ks; best_cost = cost; }
@@ -523,7 +524,7 @@ es_status_t launch_splitk_finish(const LinearParams& p, int epi, cudaStream_t s,
   const int pairs = (epi == EPI_SWIGLU) ? p.N : (p.N + 1) / 2;
   const long long work = (long long)p.M * pairs;
   int grid = (int)((work + 255) / 256);
-  if (grid > 4 * 148) grid = 4 * 148;
+  if (grid > 4 * sm_count()) grid = 4 * sm_count();
   switch (epi) {
     case EPI_SWIGLU: ES_CUDA_CHECK(launch_kernel(splitk_finish_kernel<EPI_SWIGLU>, dim3(grid), dim3(256), 0, s, pdl, p)); break;
     case EPI_QKV: ES_CUDA_CHECK(launch_kernel(splitk_finish_kernel<EPI_QKV>, dim3(grid), dim3(256), 0, s, pdl, p)); break;
@@ -537,7 +538,7 @@ es_status_t launch_linear_stream_mma(const LinearParams& p, int epi, cudaStream_
   if (!linear_stream_mma_supported(p, epi)) return fail(ES_ERR_UNSUPPORTED, "tensor-core streaming kernel does not take this shape");
   if (p.k_splits > 1) {
     const int nt = p.M <= 8 ? 1 : 2;
-    if (p.part == nullptr || (p.K / KSTEP) % p.k_splits != 0 || p.k_splits > KS_GRID ||
+    if (p.part == nullptr || (p.K / KSTEP) % p.k_splits != 0 || p.k_splits > ks_grid() ||
         (size_t)nt * 8 * (p.K / p.k_splits + 8) * sizeof(__half) > KS_SMEM_MAX)
       return fail(ES_ERR_INVALID_ARG, "K-sliced streaming kernel: %d slices do not fit K = %d", p.k_splits, p.K);
   }

@@ -278,6 +278,7 @@ int pick_bn(const LinearParams& p, int epi) {
   // that minimises it (the wider one on ties); QKV segments must be whole tiles.
   const int m_tiles = (p.M + BM - 1) / BM;
   const int cands[8] = {256, 224, 192, 160, 128, 96, 64, 32};
+  const int sms = sm_count();
   int best = 0;
   long long best_cost = 0;
   for (int bn : cands) {
@@ -287,7 +288,7 @@ int pick_bn(const LinearParams& p, int epi) {
       for (int s = 0; s < 3; ++s) if (p.seg_rows[s] % out) fits = false;
     if (!fits) continue;
     const long long tiles = (long long)m_tiles * ((p.N + out - 1) / out);
-    const long long waves = (tiles + 147) / 148;
+    const long long waves = (tiles + sms - 1) / sms;
     const long long cost = waves * (BM + bn);
     if (best == 0 || cost < best_cost) { best = bn; best_cost = cost; }
   }
@@ -359,7 +360,7 @@ int linear_tc_splits(const LinearParams& p, int epi) {
   if (epi != EPI_F32 || p.M <= 16 || p.N % 4 != 0) return 1;
   const int tiles = ((p.M + BM - 1) / BM) * ((p.N + 255) / 256);
   const int num_kb = (p.K + BK - 1) / BK;
-  int s = 148 / tiles;
+  int s = sm_count() / tiles;
   if (s > 8) s = 8;
   if (s > num_kb / 4) s = num_kb / 4;
   if (s < 2) return 1;
@@ -367,7 +368,7 @@ int linear_tc_splits(const LinearParams& p, int epi) {
   return (num_kb + kb_per - 1) / kb_per;       // no empty slice
 }
 
-size_t linear_tc_split_workspace_bytes() { return (size_t)148 * BM * 256 * sizeof(float); }
+size_t linear_tc_split_workspace_bytes() { return (size_t)sm_count() * BM * 256 * sizeof(float); }
 
 bool linear_tc_supported(const LinearParams& p, int epi) {
   if (p.M <= 0 || p.N <= 0 || p.K <= 0) return false;

@@ -332,7 +332,8 @@ int pair_nacc(const LinearParams& p, int epi) {
   const int out = (epi == EPI_SWIGLU) ? BN2 / 2 : BN2;
   const long long mt = (p.M + 2 * BM2 - 1) / (2 * BM2);
   const long long t1 = mt * ((p.N + out - 1) / out), t2 = mt * ((p.N + 2 * out - 1) / (2 * out));
-  const long long w1 = (t1 + 73) / 74, w2 = 2 * ((t2 + 73) / 74);
+  const long long pairs = sm_count() / 2 > 0 ? sm_count() / 2 : 1;
+  const long long w1 = (t1 + pairs - 1) / pairs, w2 = 2 * ((t2 + pairs - 1) / pairs);
   return (w2 * 92 < w1 * 100) ? 2 : 1;
 }
 
@@ -363,9 +364,10 @@ bool linear_tc2_supported(const LinearParams& p, int epi) {
 int linear_tc2_splits(const LinearParams& p, int epi) {
   if (epi != EPI_F32 || p.M < 2 * BM2 || p.N % 4 != 0 || !linear_tc_supported(p, epi)) return 1;
   const int tiles = ((p.M + 2 * BM2 - 1) / (2 * BM2)) * ((p.N + BN2 - 1) / BN2);
-  if (tiles >= 74) return 1;
+  const int pairs = sm_count() / 2;
+  if (tiles >= pairs) return 1;
   const int num_kb = (p.K + BK2 - 1) / BK2;
-  int s = 74 / tiles;
+  int s = pairs / tiles;
   if (s > 8) s = 8;
   if (s > num_kb / 4) s = num_kb / 4;
   while (s > 1 && (size_t)s * p.M * p.N * sizeof(float) > linear_tc_split_workspace_bytes()) --s;

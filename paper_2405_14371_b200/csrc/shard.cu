@@ -61,13 +61,19 @@ const Tunables& tunables() {
   return t;
 }
 
+int sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 1;
+  return n;
+}
+
 // How the context of a decode-attention call is cut into splits: enough CTAs to fill the machine,
 // never less than one KV page per split.
 void choose_splits(int max_ctx, int P, int B, int Hkv, int group, int* n_splits, int* pages_per_split) {
   const int pages = (max_ctx + P - 1) / P;
   // about one CTA per SM when every KV head serves one or two query heads (the kernel then lives on
   // bytes in flight); four times as many for larger groups, whose CTAs are arithmetic heavy
-  const int ctas = (group >= 4 ? 4 : 1) * 148;
+  const int ctas = (group >= 4 ? 4 : 1) * sm_count();
   long long pps = (long long)pages * B * Hkv / ctas;
   // at least 256 tokens per split (384 for large groups, whose CTAs carry more fixed work per split)
   // ... except for one or two sequences with a context beyond 256 tokens: those launches are latency bound, their
