@@ -12,6 +12,13 @@ start on the next micro-batch while the previous one is still on the wire: with 
 work concurrently without any global step (the paper's "no bubbles" schedule falls out of the data dependencies;
 its "bubbles" variant adds a barrier per iteration).
 
+Ordering without tags.  NCCL matches point-to-point messages of a pair of ranks in issue order and runs a
+communicator's operations one after the other, so two rules keep the flow free of deadlock there as well as over
+gloo: both ends of every link walk the micro-batches in the same order, and the return hop (tokens, last rank ->
+rank 0) has a communicator of its own.  With a single communicator rank 0 would queue the activations of all
+micro-batches before its first token receive while the last rank queues each token send before its next
+activation receive: each side's queue would wait for an operation the other side has not reached.
+
 This module only moves tensors and orders calls: every step of a pass runs in the shard library's kernels.  The
 `shard` argument is any object with the binding's `es_shard_prefill / es_shard_decode_step / es_shard_handoff`
 methods.  Over NCCL the tensors live on the rank's GPU; over gloo on the CPU (the multi-process tests run there,
@@ -42,18 +49,26 @@ class PipelineStage:
         self.device, self.schedule, self.group = device, schedule, group
         self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
         self.first, self.last = self.rank == 0, self.rank == self.world - 1
+        # the return hop's own communicator (a collective call: every rank of the group constructs its stage)
+        self.group_back = None
+        if self.world > 1:
+            ranks = list(range(dist.get_world_size())) if group is None else dist.get_process_group_ranks(group)
+            self.group_back = dist.new_group(ranks=ranks)
         self._pending: List = []              # send requests in flight (their tensors are kept alive with them)
         self._tok_in = [torch.empty(batch, dtype=torch.int32, device=device) for _ in range(micro_batches)]
         self._row_in = [torch.empty(batch, 1, d_model, dtype=torch.float32, device=device) for _ in range(micro_batches)]
         self._act_in: List[Optional[torch.Tensor]] = [None] * micro_batches     # prefill activations, sized on first use
 
     # -- plumbing ----------------------------------------------------------------------------------
+    def _link(self, tag: int):
+        return self.group_back if tag == TAG_TOK else self.group
+
     def _send(self, t: torch.Tensor, dst: int, tag: int, mb: int) -> None:
         t = t.contiguous().clone()            # the handoff view is overwritten by this shard's next pass
-        self._pending.append((dist.isend(t, dst, group=self.group, tag=tag * 4096 + mb), t))
+        self._pending.append((dist.isend(t, dst, group=self._link(tag), tag=tag * 4096 + mb), t))
 
     def _recv(self, buf: torch.Tensor, src: int, tag: int, mb: int) -> torch.Tensor:
-        dist.recv(buf, src, group=self.group, tag=tag * 4096 + mb)
+        dist.recv(buf, src, group=self._link(tag), tag=tag * 4096 + mb)
         return buf
 
     def _reap(self) -> None:
