@@ -73,9 +73,9 @@ es_status_t es_op_decode_attention_static(const void* q, const void* k_pages, co
   // The partials need no clearing (every split that the merge reads is written earlier in this same call); the
   // arrival counters that follow them must start at zero.  A fill is not an allocation.
   p.part = (float*)scratch;
+  p.split_cnt = (int*)((unsigned char*)scratch + decode_attention_counter_offset(B, Hq, hd, p.n_splits));
   if (p.n_splits > 1)
-    ES_CUDA_CHECK(cudaMemsetAsync((unsigned char*)scratch + decode_attention_counter_offset(B, Hq, hd, p.n_splits), 0,
-                                  decode_attention_counter_bytes(B, Hq), (cudaStream_t)stream));
+    ES_CUDA_CHECK(cudaMemsetAsync(p.split_cnt, 0, decode_attention_counter_bytes(B, Hq), (cudaStream_t)stream));
   return launch_decode_attention(p, (cudaStream_t)stream, nullptr);
 }
 

@@ -202,8 +202,9 @@ struct DecodeAttnParams {
   KvView kv;
   const int* ctx_len;     // indexed by slot (or by b when kv.slots == nullptr)
   int ctx_add;            // keys visible = ctx_len[.] + ctx_add
-  float* part;            // scratch [B, Hq, n_splits, hd + 2], then (256-byte aligned) one arrival counter per
-                          // (sequence, KV head), zero before the launch and zero again after it
+  float* part;            // scratch [B, Hq, n_splits, hd + 2]
+  int* split_cnt;         // one arrival counter per (sequence, KV head), zero before the launch and zero again after
+                          // it (needed when n_splits > 1 and the launch is small enough to merge in the kernel)
   int B, Hq, Hkv, hd;
   int n_splits, pages_per_split;
   int merge_in_kernel;    // set by launch_decode_attention: the last split CTA to arrive merges (else a merge launch)
@@ -220,9 +221,7 @@ size_t decode_attention_counter_bytes(int B, int Hq);
 // writes the final rows and puts the counter back to zero.  Nobody waits.  All threads of the CTA call.
 template <int HD, int G>
 __device__ __forceinline__ void merge_splits_if_last(const DecodeAttnParams& p, int b, int kvh, int ctx, int* s_flag) {
-  int* cnt = reinterpret_cast<int*>(reinterpret_cast<unsigned char*>(p.part) +
-                                    (((size_t)p.B * p.Hq * p.n_splits * (HD + 2) * sizeof(float) + 255) / 256) * 256) +
-             (b * p.Hkv + kvh);
+  int* cnt = p.split_cnt + (b * p.Hkv + kvh);
   const int tokens_per_split = p.pages_per_split * p.kv.P;
   int active = (ctx + tokens_per_split - 1) / tokens_per_split;
   active = active < p.n_splits ? active : p.n_splits;

@@ -481,6 +481,8 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     if (decode) {
       DecodeAttnParams a{};
       a.q = s->q; a.out = s->ao; a.kv = kvv; a.ctx_len = s->ctx_len; a.ctx_add = 1; a.part = s->part;
+      // the counters sit behind the partials of the LARGEST batch, so that no batch's partials ever cover them
+      a.split_cnt = (int*)((unsigned char*)s->part + decode_attention_counter_offset(d.max_batch, d.n_heads, d.head_dim, s->lay.n_splits));
       a.B = B; a.Hq = d.n_heads; a.Hkv = d.n_kv_heads; a.hd = d.head_dim;
       a.n_splits = s->lay.n_splits; a.pages_per_split = s->lay.pages_per_split;
       a.stamp = next_stamp(s, ES_KT_ATTENTION, 0.0);
@@ -1219,9 +1221,9 @@ es_status_t es_op_decode_attention(const void* q, const void* k_pages, const voi
   if (scratch_bytes < decode_attention_scratch_bytes(B, Hq, hd, p.n_splits))
     return fail(ES_ERR_WORKSPACE, "scratch: %zu bytes given, %zu needed", scratch_bytes,
                 decode_attention_scratch_bytes(B, Hq, hd, p.n_splits));
+  p.split_cnt = (int*)((unsigned char*)scratch + decode_attention_counter_offset(B, Hq, hd, p.n_splits));
   if (p.n_splits > 1)         // the splits' arrival counters start at zero
-    ES_CUDA_CHECK(cudaMemsetAsync((unsigned char*)scratch + decode_attention_counter_offset(B, Hq, hd, p.n_splits), 0,
-                                  decode_attention_counter_bytes(B, Hq), (cudaStream_t)stream));
+    ES_CUDA_CHECK(cudaMemsetAsync(p.split_cnt, 0, decode_attention_counter_bytes(B, Hq), (cudaStream_t)stream));
   return launch_decode_attention(p, (cudaStream_t)stream, nullptr);
 }
 

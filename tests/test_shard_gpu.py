@@ -175,6 +175,31 @@ def test_batch_rows_independent_and_match_oracle(B, tiny):
     sh.close()
 
 
+def test_batch_size_changes_between_steps_with_split_contexts(B, tiny):
+    """Contexts long enough to be cut into several splits (merged inside the kernel for so few sequences), decoded with a
+    batch that shrinks and grows again between steps: what one batch size leaves in the scratch buffer (partials,
+    arrival counters) must not disturb the next.  Every step is compared with the oracle, sequence by sequence."""
+    wd, wh = tiny
+    T, Bn = 300, 3
+    ids = prompt_ids(0, Bn, T, TINY.vocab, seed=21)
+    forced = forced_decode_ids(0, Bn, 6, TINY.vocab, seed=21)
+    sh = B.Shard(TINY, 0, 2, wd, max_slots=Bn, max_seq=T + 8, max_tokens=Bn * T)
+    sh.es_shard_prefill(ids.cuda(), None, Bn, T, [0, 1, 2])
+    seqs = [ids[b].tolist() for b in range(Bn)]
+    plan = [[0, 1, 2], [1], [0, 1, 2], [2, 0], [0, 1, 2], [1]]
+    for step, rows in enumerate(plan):
+        tok = torch.tensor([int(forced[step, b]) for b in rows], dtype=torch.int32)
+        sh.es_shard_decode_step(tok.cuda(), None, len(rows), rows)
+        h, l, _ = sh.es_shard_handoff()
+        for i, b in enumerate(rows):
+            seqs[b].append(int(tok[i]))
+            want_h, want_l = O.shard_forward_full(TINY, wh, 0, 2, ids=torch.tensor(seqs[b]))
+            assert rel_err(h[i, 0], want_h[-1]) < TOL, (step, b)
+            assert rel_err(l[i], want_l) < TOL, (step, b)
+    sh.es_shard_device_status()
+    sh.close()
+
+
 def test_page_map_and_graphs_do_not_change_results(B, tiny):
     wd, _ = tiny
     ids = prompt_ids(0, 2, 20, TINY.vocab, seed=9).cuda()
