@@ -142,6 +142,20 @@ ES_API es_status_t es_shard_prefill(es_shard_t *shard, const int32_t *ids, const
 ES_API es_status_t es_shard_prefill_ragged(es_shard_t *shard, const int32_t *ids, const es_tensor_t *hidden_in,
                                     int32_t B, int32_t T, const int32_t *slots, const int32_t *lens);
 
+/* The same prompts without the padding (Sec. "Generative LLM Inference" pads a batch to one length; this form
+ * computes only the real tokens): the B prompts are PACKED one after the other,
+ *   ids        dev int32 [sum(lens)]            (shard with the embedding), or
+ *   hidden_in  dev fp32 [sum(lens), d_model]    (other shards: the previous shard's packed handoff),
+ *   lens       host int32 [B], 1 <= lens[b] <= max_seq; sum(lens) <= max_tokens.
+ * Sequence b owns rows sum(lens[0..b-1]) .. + lens[b] - 1; every product runs over sum(lens) rows, attention runs
+ * per sequence over its own rows, K/V go to the sequence's slot, and slot b then holds lens[b] positions exactly
+ * as after es_shard_prefill_ragged.  With the output layer, logits and greedy tokens are [B, ...], those of each
+ * sequence's last token.  es_shard_handoff() gives hidden as [1, sum(lens), d_model] (packed the same way): the
+ * next shard takes it with the same lens.  Results equal the padded form's up to fp32 summation order (the
+ * products see a different number of rows).  ES_ERR_RANGE / ES_ERR_KV_FULL as for the other prefill calls. */
+ES_API es_status_t es_shard_prefill_packed(es_shard_t *shard, const int32_t *ids, const es_tensor_t *hidden_in,
+                                           int32_t B, const int32_t *slots, const int32_t *lens);
+
 /* One autoregressive step for B sequences: each consumes one token (ids dev int32 [B]) or one
  * activation row (hidden_in fp32 [B, d_model]) at its slot's next position and attends to the
  * slot's cached keys/values.  ES_ERR_STATE if a slot has no prefilled context, ES_ERR_KV_FULL if

@@ -71,6 +71,7 @@ def _load() -> C.CDLL:
         "es_shard_create": (i32, [P(es_model_desc_t), i32, i32, P(es_weights_t), vp, sz, vp, sz, vp, P(vp)]),
         "es_shard_prefill": (i32, [vp, vp, P(es_tensor_t), i32, i32, P(i32)]),
         "es_shard_prefill_ragged": (i32, [vp, vp, P(es_tensor_t), i32, i32, P(i32), P(i32)]),
+        "es_shard_prefill_packed": (i32, [vp, vp, P(es_tensor_t), i32, P(i32), P(i32)]),
         "es_shard_decode_step": (i32, [vp, vp, P(es_tensor_t), i32, P(i32)]),
         "es_shard_handoff": (i32, [vp, P(es_tensor_t), P(es_tensor_t), P(es_tensor_t)]),
         "es_layer_profile": (i32, [vp, P(es_layer_profile_t), i32, P(i32)]),
@@ -109,7 +110,7 @@ def _load() -> C.CDLL:
 
 
 lib = _load()
-EXPORTS = ("es_shard_workspace_bytes es_shard_create es_shard_prefill es_shard_prefill_ragged es_shard_decode_step es_shard_handoff "
+EXPORTS = ("es_shard_workspace_bytes es_shard_create es_shard_prefill es_shard_prefill_ragged es_shard_prefill_packed es_shard_decode_step es_shard_handoff "
            "es_layer_profile es_shard_set_profiling es_shard_reset_slots es_shard_set_page_table es_shard_set_graphs "
            "es_partition_latency es_partition_throughput es_shard_device_status es_shard_wait_probe es_shard_launch_count es_shard_set_kernel_timing es_shard_kernel_timing es_shard_kernel_timing_detail es_shard_set_step_timing es_shard_step_timing es_shard_destroy es_last_error es_version es_op_rmsnorm "
            "es_op_linear es_op_linear_splitk_workspace_bytes es_op_linear_splitk es_op_prefill_attention es_op_decode_attention_scratch_bytes es_op_decode_attention "
@@ -218,6 +219,16 @@ class Shard:
         if len(lens) != B:
             raise EsError(1, "lens must have one entry per sequence")
         _check(lib.es_shard_prefill_ragged(self._handle, _ptr(ids), hin, B, T, _i32_array(slots), _i32_array(lens)))
+
+    def es_shard_prefill_packed(self, ids: Optional[torch.Tensor], hidden_in: Optional[torch.Tensor], B: int,
+                                slots: Sequence[int], lens: Sequence[int]) -> None:
+        """Prompts of different lengths packed one after the other: ids [sum(lens)] or hidden_in [sum(lens), d]."""
+        hin = C.byref(_as_tensor_struct(hidden_in)) if hidden_in is not None else None
+        if ids is not None and not (ids.is_cuda and ids.dtype == torch.int32 and ids.is_contiguous()):
+            raise EsError(1, "ids must be a contiguous int32 CUDA tensor")
+        if len(lens) != B:
+            raise EsError(1, "lens must have one entry per sequence")
+        _check(lib.es_shard_prefill_packed(self._handle, _ptr(ids), hin, B, _i32_array(slots), _i32_array(lens)))
 
     def es_shard_decode_step(self, ids: Optional[torch.Tensor], hidden_in: Optional[torch.Tensor], B: int,
                              slots: Sequence[int]) -> None:

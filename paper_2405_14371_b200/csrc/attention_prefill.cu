@@ -22,11 +22,14 @@ __global__ void __launch_bounds__(PWARPS * 32) prefill_attn_simt_kernel(const Pr
   const int h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.Hq / p.Hkv);
   const int slot = p.kv.slots ? p.kv.slots[b] : b;
-  const bool active = t < p.T;
+  // packed prompts: the sequence's first row and length come from the first-row table (p.T = the longest prompt)
+  const int row0 = p.cu_rows ? p.cu_rows[b] : b * p.T;
+  const int Tb = p.cu_rows ? p.cu_rows[b + 1] - row0 : p.T;
+  const bool active = t < Tb;
   const float scale = rsqrtf((float)HD);
   stamp_begin(p.stamp);
   if (active) {
-    const __half* qrow = p.q + (((int64_t)b * p.T + t) * p.Hq + h) * HD;
+    const __half* qrow = p.q + (((int64_t)row0 + t) * p.Hq + h) * HD;
 #pragma unroll
     for (int e = 0; e < E; ++e) q_s[warp][lane * E + e] = __half2float(qrow[lane * E + e]) * scale;
   }
@@ -86,7 +89,7 @@ __global__ void __launch_bounds__(PWARPS * 32) prefill_attn_simt_kernel(const Pr
       }
     }
   }
-  __half* orow = p.out + (((int64_t)b * p.T + t) * p.Hq + h) * HD + lane * E;
+  __half* orow = p.out + (((int64_t)row0 + t) * p.Hq + h) * HD + lane * E;
   const float inv = 1.0f / l;
 #pragma unroll
   for (int e = 0; e < E; ++e) orow[e] = __float2half_rn(acc[e] * inv);

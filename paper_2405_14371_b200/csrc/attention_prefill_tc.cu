@@ -50,6 +50,7 @@ struct AttnArgs {
   int* status;
   int B, T, Hq, Hkv;
   int paged, P, pages_per_slot;
+  const int* cu_rows;        // packed prompts: first query row of every sequence [B + 1], or nullptr (row b * T)
   float scale_log2e;         // log2(e) / sqrt(hd)
   unsigned long long* stamp; // optional time stamps of the launch, nullptr = none
 };
@@ -95,7 +96,15 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = blockIdx.x * QT, h = blockIdx.y, b = blockIdx.z;
   const int g = h / (a.Hq / a.Hkv);
-  const int q_hi = min(a.T, q0 + QT);                    // one past the last query row of this tile
+  // rows of this sequence in the q / output matrices and its prompt length (packed prompts: from the first-row
+  // table, which the host uploaded before the pass began; a.T is then the longest prompt and sizes the grid)
+  const int row0 = a.cu_rows ? a.cu_rows[b] : b * a.T;
+  const int Tb = a.cu_rows ? a.cu_rows[b + 1] - row0 : a.T;
+  if (q0 >= Tb) {                                        // a tile past the end of a shorter prompt: nothing set up yet
+    stamp_end(a.stamp);
+    return;
+  }
+  const int q_hi = min(Tb, q0 + QT);                     // one past the last query row of this tile
   const int n_kv = (q_hi + KT - 1) / KT;                 // causal: keys 0 .. q_hi-1
 
   if (threadIdx.x == 0) {
@@ -131,7 +140,7 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
       mbar_expect_tx(qb, L::Q_BYTES);
 #pragma unroll
       for (int hf = 0; hf < HALVES; ++hf)
-        tma_load_2d(smem_u32(q_s + hf * (QT * 128)), &maps.q, h * HD + hf * 64, b * a.T + q0, qb);
+        tma_load_2d(smem_u32(q_s + hf * (QT * 128)), &maps.q, h * HD + hf * 64, row0 + q0, qb);
       const int slot = a.paged ? (a.slots ? a.slots[b] : b) : 0;
       for (int j = 0; j < n_kv; ++j) {
         const int s = j & 1;
@@ -144,7 +153,7 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
           row = (page * a.Hkv + g) * a.P + (t0 % a.P);
           col = 0;
         } else {
-          row = b * a.T + j * KT;
+          row = row0 + j * KT;
           col = g * HD;
         }
         const uint32_t fb = smem_u32(&kv_full[s]);
@@ -294,12 +303,12 @@ prefill_attn_tc_kernel(const __grid_constant__ AttnMaps maps, const AttnArgs a) 
     if (ok) {
       tc_fence_after();
       const float inv = (l_run > 0.f) ? 1.0f / l_run : 0.f;
-      __half* orow = a.out + ((int64_t)b * a.T + qi) * ((int64_t)a.Hq * HD) + (int64_t)h * HD;
+      __half* orow = a.out + ((int64_t)row0 + qi) * ((int64_t)a.Hq * HD) + (int64_t)h * HD;
 #pragma unroll 1
       for (int c = 0; c < HD; c += 32) {
         float o[32];
         tmem_ld32(tmem_o + lane_off + c, o);
-        if (qi < a.T) {
+        if (qi < Tb) {
 #pragma unroll
           for (int q8 = 0; q8 < 4; ++q8) {
             uint4 val;
@@ -344,6 +353,7 @@ es_status_t launch_hd(const AttnMaps& maps, const PrefillAttnParams& p, cudaStre
   a.slots = p.kv.slots;
   a.status = p.status;
   a.B = p.B; a.T = p.T; a.Hq = p.Hq; a.Hkv = p.Hkv;
+  a.cu_rows = p.cu_rows;
   a.paged = is_paged(p) ? 1 : 0;
   a.P = p.kv.P;
   a.pages_per_slot = p.kv.pages_per_slot;

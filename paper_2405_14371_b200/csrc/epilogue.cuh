@@ -12,6 +12,23 @@ namespace es {
 // z below about -87, gives 0 where the exact value is below 1e-36 in magnitude).  Every kernel path uses this one.
 __device__ __forceinline__ float silu_f(float z) { return __fdividef(z, 1.0f + __expf(-z)); }
 
+// Sequence and prompt offset of row m of a prefill: m / T and m % T, or with packed prompts the sequence whose row
+// range holds m (binary search over the first-row table) and the offset inside it.
+__device__ __forceinline__ void row_to_seq(const LinearParams& p, int m, int& b, int& off) {
+  if (p.cu_rows == nullptr) {
+    b = m / p.T;
+    off = m - b * p.T;
+    return;
+  }
+  int lo = 0, hi = p.n_seq;                  // invariant: cu_rows[lo] <= m < cu_rows[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (p.cu_rows[mid] <= m) lo = mid; else hi = mid;
+  }
+  b = lo;
+  off = m - p.cu_rows[lo];
+}
+
 // Residual / plain store of columns n and n+1 of row m.
 __device__ __forceinline__ void epi_f32_pair(const LinearParams& p, int m, int n, float v0, float v1) {
   if (m >= p.M || n >= p.N) return;
@@ -36,9 +53,10 @@ __device__ __forceinline__ void epi_swiglu(const LinearParams& p, int m, int n, 
 // fp16 once; k and v go straight to the slot's KV page.
 __device__ __forceinline__ void epi_qkv_pair(const LinearParams& p, int m, int n, float v0, float v1) {
   if (m >= p.M || n >= p.N) return;
-  const int b = m / p.T;
+  int b, row_off;
+  row_to_seq(p, m, b, row_off);
   const int slot = p.slots[b];
-  const int pos = p.is_decode ? p.ctx_len[slot] : (m - b * p.T);
+  const int pos = p.is_decode ? p.ctx_len[slot] : row_off;
   if (pos < 0 || pos >= p.max_seq) return;   // host validates; never index outside the tables
   const int nq = p.Hq * p.hd, nkv = p.Hkv * p.hd;
   int c;          // column inside its head
@@ -156,9 +174,10 @@ __device__ __forceinline__ QkvRow qkv_row(const LinearParams& p, int m) {
   r.valid = false;
   r.rope_off = 0; r.q_off = 0; r.kv_off = 0;
   if (m >= p.M) return r;
-  const int b = m / p.T;
+  int b, off;
+  row_to_seq(p, m, b, off);
   const int slot = p.slots[b];
-  const int pos = p.is_decode ? p.ctx_len[slot] : (m - b * p.T);
+  const int pos = p.is_decode ? p.ctx_len[slot] : off;
   if (pos < 0 || pos >= p.max_seq) return r;
   const int page = p.block_table[(int64_t)slot * p.pages_per_slot + pos / p.P];
   r.valid = true;

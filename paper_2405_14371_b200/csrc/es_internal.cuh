@@ -92,6 +92,8 @@ struct LinearParams {
   const float* rope_sin;
   int T;                   // rows per sequence: row m belongs to sequence m / T at prompt offset m % T
   int is_decode;           // position = ctx_len[slot] instead of m % T
+  const int* cu_rows;      // packed prompts: [n_seq + 1] first row of every sequence (device); row m then belongs to the
+  int n_seq;               // sequence b with cu_rows[b] <= m < cu_rows[b + 1], at offset m - cu_rows[b].  nullptr = m / T
   int Hq, Hkv, hd, P, pages_per_slot, max_seq;
   // split-K (tensor-core kernel with EPI_F32; K-sliced streaming kernel with any epilogue): > 1 = raw partial
   // sums go to part[k_splits, M, columns] and a second kernel finishes the product
@@ -185,6 +187,7 @@ struct PrefillAttnParams {
   KvView kv;
   int B, T, Hq, Hkv, hd;
   int64_t kv_rows;          // rows of the K / V matrices as 2-D [rows, row width] views (tensor-core kernel)
+  const int* cu_rows;       // packed prompts: [B + 1] first query row of every sequence (T = the longest prompt), or nullptr
   const TcMaps* tc_maps;    // pre-encoded maps {q, k, v} or nullptr: encode per launch
   int* status;
   unsigned long long* stamp;   // optional time stamps of this launch, nullptr = none

@@ -159,7 +159,7 @@ Layout make_layout(const es_model_desc_t& d, int begin, int end) {
   L.off_sin = take((size_t)d.max_seq * (d.head_dim / 2) * 4, "rope sin");
   L.off_table = take((size_t)L.n_pages * 4, "page table");
   L.off_ctx = take((size_t)d.max_slots * 4, "context lengths");
-  L.off_slots = take(2 * B * 4, "slots");       // slots, then the prompt lengths of a ragged prefill
+  L.off_slots = take((3 * B + 1) * 4, "slots");  // slots, the prompt lengths of a ragged prefill, the first rows of packed prompts
   L.off_status = take(256, "status words");
   L.off_splitk = take(d.max_tokens > 2 ? linear_tc_split_workspace_bytes() : 0, "split-K workspace");   // split-K partial sums of short prefills
   L.off_stamps = take((size_t)2 * STAMP_SLOTS * sizeof(unsigned long long), "time stamps");
@@ -210,12 +210,14 @@ struct es_shard {
   float* x;
   __half *h, *q, *ao, *act, *h_last;
   float *logits, *part, *rope_cos, *rope_sin;
-  int *next_ids, *block_table, *ctx_len, *slots_dev, *lens_dev, *status;
+  int *next_ids, *block_table, *ctx_len, *slots_dev, *lens_dev, *cu_dev, *status;
   float* splitk = nullptr;      // split-K workspace (nullptr when the shard never runs more than 2 rows)
   std::vector<int> ctx;         // host mirror of ctx_len, -1 = never prefilled
   std::vector<int> slots_host;  // slots currently uploaded to slots_dev
   std::vector<int> lens_host;   // prompt lengths of the last ragged prefill (source of the upload)
+  std::vector<int> cu_host;     // first rows of the last packed prefill (source of the upload)
   int last_B = 0, last_T = 0;
+  int last_head_rows = 0;      // rows of logits / next ids of the last pass (sequences, also when the hidden rows are packed)
   bool last_valid = false;
   int64_t launches = 0;
   bool profiling = false;
@@ -223,6 +225,8 @@ struct es_shard {
   std::vector<ProfileEntry> prof;
   bool graphs = true;
   bool pdl_now = false;   // the pass being enqueued uses programmatic dependent launch (decode steps)
+  const int* pass_cu = nullptr;   // the pass being enqueued is a prefill of packed prompts: their first-row table (device)
+  int pass_n_seq = 0;
   std::map<GraphKey, GraphEntry> graph_cache;
   // tensor maps of the prefill GEMMs, encoded once: [layer][qkv, o, gate/up, down]
   std::vector<TcMaps> tmaps;
@@ -349,6 +353,8 @@ LinearParams base_params(const es_shard* s, int M, int T, bool decode) {
   p.P = s->d.kv_page_tokens;
   p.pages_per_slot = s->lay.pages_per_slot;
   p.max_seq = s->d.max_seq;
+  p.cu_rows = s->pass_cu;
+  p.n_seq = s->pass_n_seq;
   return p;
 }
 
@@ -422,10 +428,14 @@ inline void prof_mark(es_shard* s, int idx, int which) {
 // The launch sequence of one pass (prefill: T tokens per sequence; decode: T == 1 at each slot's
 // next position).  Everything is enqueued on s->stream.
 // lens (device, [B]) != nullptr: a prefill of right-padded prompts; sequence b has lens[b] <= T real tokens
+// cu (device, [B + 1]) != nullptr: a prefill of PACKED prompts; sequence b owns rows cu[b] .. cu[b + 1] - 1 of the
+// total_rows rows, T is the longest prompt, lens its lengths
 es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in, int B, int T, bool decode,
-                         const int* lens = nullptr) {
+                         const int* lens = nullptr, const int* cu = nullptr, int total_rows = 0) {
   const es_model_desc_t& d = s->d;
-  const int M = B * T;
+  const int M = cu ? total_rows : B * T;
+  s->pass_cu = cu;
+  s->pass_n_seq = cu ? B : 0;
   int pi = 0;
   const float* xin = s->x;
   const bool pdl = tunables().pdl != 0;
@@ -493,6 +503,7 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
       a.kv_rows = (int64_t)s->lay.n_pages * d.n_kv_heads * d.kv_page_tokens;
       a.status = s->status;
       a.tc_maps = s->attn_maps_valid ? &s->attn_maps[li] : nullptr;
+      a.cu_rows = cu;
       a.stamp = next_stamp(s, ES_KT_ATTENTION, 0.0);
       ES_TRY(launch_prefill_attention(a, s->stream, &s->launches, 0, pdl));
     }
@@ -557,7 +568,9 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
     const bool fuse_head = lens == nullptr && linear_stream_can_fuse_norm(B);
     if (!fuse_head) {
       ES_TRY(kt_begin(s));
-      ES_TRY(launch_rmsnorm(s->x, s->fnorm, s->h_last, B, d.d_model, d.rms_eps, T, T - 1, s->stream, &s->launches, pdl, lens,
+      // last row of every sequence: row b * T + lens[b] - 1, or with packed prompts row cu[b + 1] - 1
+      ES_TRY(launch_rmsnorm(s->x, s->fnorm, s->h_last, B, d.d_model, d.rms_eps, cu ? 0 : T, T - 1, s->stream, &s->launches, pdl,
+                            cu ? cu + 1 : lens,
                             next_stamp(s, ES_KT_RMSNORM, (double)B * d.d_model * 6.0)));
       ES_TRY(kt_end(s, ES_KT_RMSNORM, (double)B * d.d_model * 6.0));
     }
@@ -585,6 +598,8 @@ es_status_t enqueue_pass(es_shard* s, const int32_t* ids, const float* hidden_in
                         next_stamp(s, ES_KT_SET_CTX, 0.0)));
   ES_TRY(kt_end(s, ES_KT_SET_CTX, 0.0));
   s->pdl_now = false;
+  s->pass_cu = nullptr;
+  s->pass_n_seq = 0;
   return ES_OK;
 }
 
@@ -720,6 +735,7 @@ es_status_t es_shard_create(const es_model_desc_t* desc, int32_t layer_begin, in
   s->ctx_len = (int*)(sb + L.off_ctx);
   s->slots_dev = (int*)(sb + L.off_slots);
   s->lens_dev = s->slots_dev + desc->max_batch;
+  s->cu_dev = s->lens_dev + desc->max_batch;
   s->status = (int*)(sb + L.off_status);
   s->splitk = desc->max_tokens > 2 ? (float*)(sb + L.off_splitk) : nullptr;
   s->stamps = (unsigned long long*)(sb + L.off_stamps);
@@ -821,7 +837,7 @@ es_status_t es_shard_prefill(es_shard_t* s, const int32_t* ids, const es_tensor_
   s->last_valid = false;
   ES_TRY(enqueue_pass(s, ids, hin, B, T, false));
   for (int b = 0; b < B; ++b) s->ctx[slots[b]] = T;
-  s->last_B = B; s->last_T = T; s->last_valid = true;
+  s->last_B = B; s->last_T = T; s->last_head_rows = B; s->last_valid = true;
   if (s->profiling) { s->pending = true; s->pending_prefill = true; }
   return ES_OK;
 }
@@ -847,7 +863,42 @@ es_status_t es_shard_prefill_ragged(es_shard_t* s, const int32_t* ids, const es_
   s->last_valid = false;
   ES_TRY(enqueue_pass(s, ids, hin, B, T, false, s->lens_dev));
   for (int b = 0; b < B; ++b) s->ctx[slots[b]] = lens[b];
-  s->last_B = B; s->last_T = T; s->last_valid = true;
+  s->last_B = B; s->last_T = T; s->last_head_rows = B; s->last_valid = true;
+  if (s->profiling) { s->pending = true; s->pending_prefill = true; }
+  return ES_OK;
+}
+
+es_status_t es_shard_prefill_packed(es_shard_t* s, const int32_t* ids, const es_tensor_t* hidden_in, int32_t B,
+                                    const int32_t* slots, const int32_t* lens) {
+  if (!s) return fail(ES_ERR_INVALID_ARG, "shard is null");
+  if (!lens) return fail(ES_ERR_INVALID_ARG, "lens is null");
+  if (B <= 0) return fail(ES_ERR_INVALID_ARG, "B must be positive");
+  if (B > s->d.max_batch) return fail(ES_ERR_RANGE, "B = %d exceeds max_batch = %d", B, s->d.max_batch);
+  int64_t total = 0;
+  int longest = 0;
+  for (int b = 0; b < B; ++b) {
+    if (lens[b] < 1) return fail(ES_ERR_RANGE, "lens[%d] = %d must be at least 1", b, lens[b]);
+    if (lens[b] > s->d.max_seq) return fail(ES_ERR_KV_FULL, "prompt %d of %d tokens exceeds max_seq = %d", b, lens[b], s->d.max_seq);
+    total += lens[b];
+    if (lens[b] > longest) longest = lens[b];
+  }
+  if (total > s->d.max_tokens) return fail(ES_ERR_RANGE, "%lld packed rows exceed max_tokens = %d", (long long)total, s->d.max_tokens);
+  ES_TRY(check_slots(s, slots, B));
+  const float* hin;
+  ES_TRY(check_inputs(s, ids, hidden_in, total, &hin));
+  if (s->profiling) ES_TRY(harvest_profile(s));
+  if (tunables().debug_checks) ES_TRY(debug_checks_now(s));    // checking mode: what the previous pass left behind
+  ES_TRY(upload_slots(s, slots, B));
+  s->lens_host.assign(lens, lens + B);
+  s->cu_host.assign(B + 1, 0);
+  for (int b = 0; b < B; ++b) s->cu_host[b + 1] = s->cu_host[b] + lens[b];
+  ES_CUDA_CHECK(cudaMemcpyAsync(s->lens_dev, s->lens_host.data(), B * sizeof(int), cudaMemcpyHostToDevice, s->stream));
+  ES_CUDA_CHECK(cudaMemcpyAsync(s->cu_dev, s->cu_host.data(), (B + 1) * sizeof(int), cudaMemcpyHostToDevice, s->stream));
+  s->last_valid = false;
+  ES_TRY(enqueue_pass(s, ids, hin, B, longest, false, s->lens_dev, s->cu_dev, (int)total));
+  for (int b = 0; b < B; ++b) s->ctx[slots[b]] = lens[b];
+  s->last_B = 1; s->last_T = (int)total; s->last_valid = true;     // the handoff is the packed [1, total rows, d_model]
+  s->last_head_rows = B;
   if (s->profiling) { s->pending = true; s->pending_prefill = true; }
   return ES_OK;
 }
@@ -905,7 +956,7 @@ es_status_t es_shard_decode_step(es_shard_t* s, const int32_t* ids, const es_ten
     s->launches += it->second.nodes;
   }
   for (int b = 0; b < B; ++b) s->ctx[slots[b]] += 1;
-  s->last_B = B; s->last_T = 1; s->last_valid = true;
+  s->last_B = B; s->last_T = 1; s->last_head_rows = B; s->last_valid = true;
   if (s->profiling) { s->pending = true; s->pending_prefill = false; }
   return ES_OK;
 }
@@ -919,11 +970,11 @@ es_status_t es_shard_handoff(es_shard_t* s, es_tensor_t* hidden_out, es_tensor_t
   }
   if (logits) {
     logits->data = s->has_head ? s->logits : nullptr; logits->dtype = ES_DTYPE_F32; logits->rank = 2;
-    logits->shape[0] = s->last_B; logits->shape[1] = s->d.vocab; logits->shape[2] = logits->shape[3] = 1;
+    logits->shape[0] = s->last_head_rows; logits->shape[1] = s->d.vocab; logits->shape[2] = logits->shape[3] = 1;
   }
   if (next_ids) {
     next_ids->data = s->has_head ? s->next_ids : nullptr; next_ids->dtype = ES_DTYPE_I32; next_ids->rank = 1;
-    next_ids->shape[0] = s->last_B; next_ids->shape[1] = next_ids->shape[2] = next_ids->shape[3] = 1;
+    next_ids->shape[0] = s->last_head_rows; next_ids->shape[1] = next_ids->shape[2] = next_ids->shape[3] = 1;
   }
   return ES_OK;
 }

@@ -404,6 +404,52 @@ def test_ragged_prompts_and_sequences_that_stop_early(B, tiny, P, split):
             assert rel_err(got, want_l) < TOL
 
 
+@pytest.mark.parametrize("lens,P,split", [([40, 1, 16, 23], 64, None), ([40, 1, 16, 23], 16, 1), ([3, 1, 5], 64, None),
+                                          ([130, 64, 200, 7, 129], 64, 1)])
+def test_packed_prompts_skip_the_padding(B, tiny, lens, P, split):
+    """Prompts of different lengths packed one after the other (no padded rows are computed): the hidden rows, the
+    logits of every sequence's last token and three greedy decode steps must match the oracle run on each
+    sequence alone; with `split` the model runs as two shards handing the packed activation over.  The cases
+    cover the tensor-core and the CUDA-core attention (64- and 16-token pages), prompts that end inside, on and
+    just past a 128-row query tile, and a batch small enough (9 rows) for the weight-streaming kernels."""
+    wd, wh = tiny
+    Bn, total, S = len(lens), sum(lens), 3
+    seqs = [prompt_ids(0, 1, L, TINY.vocab, seed=50 + b)[0] for b, L in enumerate(lens)]
+    packed = torch.cat(seqs).cuda()
+    slots = list(reversed(range(Bn)))
+    kw = dict(max_slots=Bn, max_seq=max(lens) + S, max_tokens=total, max_batch=Bn, kv_page_tokens=P)
+    if split is None:
+        shards = [B.Shard(TINY, 0, 2, wd, **kw)]
+    else:
+        shards = [B.Shard(TINY, 0, split, slice_weights(wd, TINY, 0, split), **kw),
+                  B.Shard(TINY, split, 2, slice_weights(wd, TINY, split, 2), **kw)]
+    x = None
+    for i, sh in enumerate(shards):
+        sh.es_shard_prefill_packed(packed if i == 0 else None, x, Bn, slots, lens)
+        x, logits, nxt = sh.es_shard_handoff()
+    assert x.shape == (1, total, TINY.d_model) and logits.shape == (Bn, TINY.vocab) and nxt.shape == (Bn,)
+    pre_h, all_logits, fed = x[0].clone(), [logits.clone()], []
+    for _ in range(S):
+        fed.append(nxt.clone().cpu())
+        feed, x = nxt.clone(), None
+        for i, sh in enumerate(shards):
+            sh.es_shard_decode_step(feed if i == 0 else None, x, Bn, slots)
+            x, logits, nxt = sh.es_shard_handoff()
+        all_logits.append(logits.clone())
+    for sh in shards:
+        sh.es_shard_device_status()
+        sh.close()
+    row = 0
+    for b, L in enumerate(lens):
+        seq = torch.cat([seqs[b], torch.tensor([int(f[b]) for f in fed], dtype=torch.int32)])
+        want_h, _ = O.shard_forward_full(TINY, wh, 0, 2, ids=seq)
+        assert rel_err(pre_h[row:row + L], want_h[:L]) < TOL, b
+        for s_ in range(S + 1):
+            _, want_l = O.shard_forward_full(TINY, wh, 0, 2, ids=seq[:L + s_])
+            assert rel_err(all_logits[s_][b], want_l) < TOL, (b, s_)
+        row += L
+
+
 def test_pipeline_stage_drives_the_library_on_one_gpu(B, tiny):
     """The multi-device stage object with a single rank: it must drive the real shard (device tensors, greedy
     feedback, several micro-batches in their own KV slots) to the oracle's tokens.  The message flow between ranks
