@@ -450,6 +450,39 @@ def test_packed_prompts_skip_the_padding(B, tiny, lens, P, split):
         row += L
 
 
+def test_packed_prompts_on_7b_layer_shapes(B):
+    """The packed prefill on layer shapes that take the CTA-pair tensor-core products and the tcgen05 attention
+    (two Llama-2-7B-shaped layers, prompts of 300, 128 and 700 tokens = 1128 rows): hidden rows and last-token
+    logits of every sequence against the oracle run on that sequence alone, and against the padded form."""
+    from workload import ModelShape, shard_weights
+    m = ModelShape("7b-2layers", 2, 4096, 32, 32, 128, 11008, 512)
+    wd = shard_weights(12, m, 0, 2, device="cuda")
+    wh = {k: v.cpu() for k, v in wd.items() if k != "layers"}
+    wh["layers"] = [{k: v.cpu() for k, v in lw.items()} for lw in wd["layers"]]
+    lens = [300, 128, 700]
+    Bn, total, T = len(lens), sum(lens), max(lens)
+    seqs = [prompt_ids(12, 1, L, m.vocab, seed=70 + b)[0] for b, L in enumerate(lens)]
+    sh = B.Shard(m, 0, 2, wd, max_slots=Bn, max_seq=T + 2, max_tokens=Bn * T, max_batch=Bn)
+    sh.es_shard_prefill_packed(torch.cat(seqs).cuda(), None, Bn, [0, 1, 2], lens)
+    x, logits, nxt = sh.es_shard_handoff()
+    packed_h, packed_l = x[0].clone(), logits.clone()
+    padded = torch.zeros(Bn, T, dtype=torch.int32)
+    for b, L in enumerate(lens):
+        padded[b, :L] = seqs[b]
+    sh.es_shard_reset_slots(None)
+    sh.es_shard_prefill_ragged(padded.cuda(), None, Bn, T, [0, 1, 2], lens)
+    xp, lp, _ = sh.es_shard_handoff()
+    row = 0
+    for b, L in enumerate(lens):
+        want_h, want_l = O.shard_forward_full(m, wh, 0, 2, ids=seqs[b])
+        assert report_err(f"packed prefill, 7B shapes, sequence of {L}: hidden", rel_err(packed_h[row:row + L], want_h)) < TOL
+        assert report_err(f"packed prefill, 7B shapes, sequence of {L}: logits", rel_err(packed_l[b], want_l)) < TOL
+        assert rel_err(packed_h[row:row + L], xp[b, :L]) < 2e-3 and rel_err(packed_l[b], lp[b]) < 2e-3
+        row += L
+    sh.es_shard_device_status()
+    sh.close()
+
+
 def test_pipeline_stage_drives_the_library_on_one_gpu(B, tiny):
     """The multi-device stage object with a single rank: it must drive the real shard (device tensors, greedy
     feedback, several micro-batches in their own KV slots) to the oracle's tokens.  The message flow between ranks
