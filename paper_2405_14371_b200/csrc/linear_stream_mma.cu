@@ -431,12 +431,7 @@ es_status_t launch_inst(const LinearParams& p, cudaStream_t s, bool pdl) {
     ES_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured = smem;
   }
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    ES_CUDA_CHECK(cudaGetDevice(&dev));
-    ES_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  }
+  const int sms = sm_count();          // of the current device: a process may drive GPUs of different sizes
   int per_sm = 0;
   ES_CUDA_CHECK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, MTHREADS, smem));
   if (per_sm < 1) return fail(ES_ERR_SHAPE, "tensor-core streaming kernel does not fit (K = %d)", p.K);

@@ -305,12 +305,7 @@ es_status_t launch_bn(const TmapSet& maps, const LinearParams& p, int* status, c
     ES_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TileCfg<BN>::SMEM));
     configured = true;
   }
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    ES_CUDA_CHECK(cudaGetDevice(&dev));
-    ES_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  }
+  const int sms = sm_count();          // of the current device: a process may drive GPUs of different sizes
   const int tiles = m_tiles * n_tiles * ((EPI == EPI_F32 && p.k_splits > 1) ? p.k_splits : 1);
   ES_CUDA_CHECK(launch_kernel(kern, dim3(tiles < sms ? tiles : sms), dim3(TC_THREADS), TileCfg<BN>::SMEM, s, pdl, maps, p, status,
                               m_tiles, n_tiles));

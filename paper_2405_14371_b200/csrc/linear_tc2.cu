@@ -291,12 +291,7 @@ es_status_t launch_pair(const TmapSet2& maps, const LinearParams& p, int* status
     ES_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM2));
     configured = true;
   }
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    ES_CUDA_CHECK(cudaGetDevice(&dev));
-    ES_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-  }
+  const int sms = sm_count();          // of the current device: a process may drive GPUs of different sizes
   const int tiles = m_tiles * n_tiles * ((EPI == EPI_F32 && p.k_splits > 1) ? p.k_splits : 1);
   int pairs = sms / 2;
   if (pairs > tiles) pairs = tiles;
