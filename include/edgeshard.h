@@ -233,10 +233,10 @@ ES_API es_status_t es_shard_kernel_timing(es_shard_t *shard, double *total_ms, d
 
 /* Timing from inside a step (Sec. "Profiling" asks what each layer costs on the device; this is the same
  * question one level down, per kernel of a replayed step).  While on, every kernel of a pass records the
- * earliest time any of its CTAs started and the latest time any of its warps finished (%globaltimer,
- * one atomic per CTA / warp) into a slot of the scratch buffer; decode steps are still replayed as graphs
+ * earliest time any of its CTAs started and the latest time the first thread of any of its CTAs finished
+ * (%globaltimer, two atomics per CTA) into a slot of the scratch buffer; decode steps are still replayed as graphs
  * with programmatic dependent launch, so the overlap between consecutive kernels is what it is in a normal
- * step (the stamps cost well under a microsecond per kernel).  Switching it on or off drops the captured
+ * step (measured: a step takes the same time with and without the stamps).  Switching it on or off drops the captured
  * graphs.  es_shard_step_timing synchronises and returns, for each launch of the most recently enqueued
  * pass in launch order (up to `capacity`; *n = how many there were): its category, its start and end in
  * microseconds relative to the first start of the pass, and its algorithmic bytes (as in
